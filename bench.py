@@ -1,0 +1,349 @@
+#!/usr/bin/env python
+"""Benchmark of the hybrid decode-attention hot path on B200.
+
+A step is one pass of the whole path over one batch of synthetic input: hg_attn_partial over the
+GPU-resident KV slice, then hg_attn_merge of the chunk partials with the partials of the host-held
+slice.  Prints ONE JSON line (rank 0).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+N > 1 is launched under torchrun, one rank per GPU; every rank runs its own copy of the workload
+(independent sequences, no data-path collective): weak scaling.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode attention KV tokens/s"
+UNIT = "KV tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the partial kernel, from the ncu
+# captures summarised under profiles/ (None until a capture of that workload exists)
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        rows = [l for t, l in self.lines if t0 - 0.05 <= t <= t1 + 0.2] or [l for _, l in self.lines]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in rows:
+            p = [x.strip() for x in l.split(",")]
+            try:
+                sm.append(float(p[0])); mx.append(float(p[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, p[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample(w, rows_budget, device):
+    """Inputs for the oracle's share of the work: the GPU slice of `rows_budget` (sequence, head) rows."""
+    import numpy as np
+    import torch
+    rows = []
+    for b in range(w.B):
+        for h in range(w.Hq):
+            if len(rows) < rows_budget and w.tok_end[b] > w.tok_begin[b]:
+                rows.append((b, h))
+    bits = lambda t: t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+    qall = w.q()
+    items = []
+    for b, h in rows:
+        g = h // w.G
+        K = bits(w.kv_rows("k", b, g, w.tok_begin[b], w.tok_end[b], device))
+        V = bits(w.kv_rows("v", b, g, w.tok_begin[b], w.tok_end[b], device))
+        items.append((bits(qall[b, h]), K, V, w.tok_begin[b], w.tok_end[b]))
+    tokens = sum(it[4] - it[3] for it in items) / w.Hq     # in units of whole-layer token positions
+    return items, tokens
+
+
+def oracle_pass(w, items, threads):
+    """PARTIAL per chunk over each sampled row's slice, then MERGE (the same work the GPU path does)."""
+    from concurrent.futures import ThreadPoolExecutor
+    from oracle import hg_oracle as O
+    C = w.chunk_tokens
+
+    def one(it):
+        q, K, V, tb, te = it
+        n = te - tb
+        NC = -(-te // C) - tb // C
+        # a row is its own one-sequence, one-head cache whose token 0 is the slice's first token;
+        # the chunk grid is shifted accordingly so that chunks sit on the same absolute boundaries
+        off = tb % C
+        m, l, o = O.chunked_partials(q.reshape(1, 1, -1), _pad(K, off).reshape(1, n + off, 1, -1),
+                                     _pad(V, off).reshape(1, n + off, 1, -1), w.dtype, [off], [n + off], C, NC, threads=1)
+        return O.merge(m[0, 0], l[0, 0], o[0, 0])
+
+    with ThreadPoolExecutor(max_workers=threads) as ex:      # the C calls release the GIL
+        return list(ex.map(one, items))
+
+
+def _pad(a, off):
+    import numpy as np
+    if off == 0:
+        return a
+    return np.concatenate([np.zeros((off, a.shape[1]), dtype=a.dtype), a], axis=0)
+
+
+def time_oracle(w, device, target_core_seconds=20.0):
+    from oracle import hg_oracle as O
+    threads = O.host_threads()
+    per_row = 0.17 * (sum(e - b for b, e in zip(w.tok_begin, w.tok_end)) / max(1, w.B)) / 19660.0 * (w.D / 128.0)
+    budget = max(threads, min(w.B * w.Hq, int(target_core_seconds / max(per_row, 1e-6))))
+    items, tokens = oracle_sample(w, budget, device)
+    t0 = time.perf_counter()
+    oracle_pass(w, items, threads)
+    dt = time.perf_counter() - t0
+    return {"value": tokens / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"{len(items)} of {w.B * w.Hq} (sequence, head) rows, full GPU slice each, "
+                      f"chunked PARTIAL + MERGE in fp64, {dt:.2f} s"}, items, tokens
+
+
+def run_reference(args, rank, world):
+    """--impl reference: the fp64 oracle on the host cores, each step a bounded sample of the workload."""
+    if rank != 0:
+        return
+    import torch
+    from oracle import hg_oracle as O
+    from paper_2604_18529_b200 import workload as W
+    w = W.make_workload(args.workload)
+    dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    threads = O.host_threads()
+    items, tokens = oracle_sample(w, max(threads, 16), dev)
+    for _ in range(min(args.warmup, 1)):
+        oracle_pass(w, items[:threads], threads)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_pass(w, items, threads)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = tokens / dt
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "sample": f"{len(items)} of {w.B * w.Hq} (sequence, head) rows per step"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": f"{len(items)} rows x {args.steps} steps"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="opt13b")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--probe", action="store_true", help="also time the read-probe kernel")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        return run_reference(args, rank, world)
+
+    import torch
+    import torch.distributed as dist
+    import paper_2604_18529_b200 as pkg
+    from paper_2604_18529_b200 import workload as W
+    from paper_2604_18529_b200.problem import DeviceProblem
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    w = W.make_workload(args.workload)
+    prob = DeviceProblem(w, dev)
+    # partials of the host-held slice: produced by the host in the real system; here synthetic values with
+    # the statistics of a real partial (they are inputs of the merge, not results of this library)
+    gen = torch.Generator(device=dev).manual_seed(w.seed)
+    host = [(torch.randn(w.B, w.Hq, 1, w.D, device=dev, generator=gen),
+             torch.randn(w.B, w.Hq, 1, device=dev, generator=gen),
+             torch.rand(w.B, w.Hq, 1, device=dev, generator=gen) + 1.0)]
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        prob.step(host)
+    torch.cuda.synchronize()
+    if int(prob.status.item()) != 0:
+        raise SystemExit(f"device status {int(prob.status.item())} after warm-up")
+
+    # ---- pass A: exactly K steps, device-timed ------------------------------------------------------
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_wall0 = time.time()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        prob.step(host)
+    ev1.record(stream)
+    barrier()
+    t_wall1 = time.time()
+    ms_total = ev0.elapsed_time(ev1)
+
+    # ---- pass B: K more steps with an event around every kernel (roofline of the dominant kernel) --------
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    for e in evs:
+        e[0].record(stream); prob.partial(); e[1].record(stream); prob.merge(host); e[2].record(stream)
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    part_ms = [e[0].elapsed_time(e[1]) for e in evs]
+    merge_ms = [e[1].elapsed_time(e[2]) for e in evs]
+
+    # ---- end to end: per-step data in pinned host memory, results read back ----------------------------------
+    pin = lambda t: t.cpu().pin_memory()
+    q_h, sl_h, tb_h, te_h = pin(prob.q), pin(prob.seq_lens), pin(prob.tok_begin), pin(prob.tok_end)
+    host_h = [tuple(pin(x) for x in src) for src in host]
+    out_h = torch.empty(prob.out.shape, dtype=torch.float32).pin_memory()
+    lse_h = torch.empty(prob.lse.shape, dtype=torch.float32).pin_memory()
+    ws = torch.empty(pkg.hg_attn_workspace_bytes(prob.desc, 1), dtype=torch.uint8, device=dev)
+
+    def e2e_step():
+        pkg.hg_attn_decode_host(q_h, prob.kv["k"], prob.kv["v"], sl_h, tb_h, te_h, host_h, out_h, lse_h, ws, prob.desc)
+        stream.synchronize()            # the caller reads out_h / lse_h after every step
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ee0.record(stream)
+    for _ in range(args.steps):
+        e2e_step()
+    ee1.record(stream)
+    barrier()
+    e2e_ms = ee0.elapsed_time(ee1)
+    same = torch.equal(out_h, prob.out.cpu()) and torch.equal(lse_h, prob.lse.cpu())
+    h2d = sum(t.numel() * t.element_size() for t in (q_h, sl_h, tb_h, te_h)) + \
+        sum(t.numel() * t.element_size() for src in host_h for t in src)
+    d2h = out_h.numel() * 4 + lse_h.numel() * 4
+
+    probe_ms = None
+    if args.probe:
+        sink = torch.zeros(w.B, w.Hkv, prob.NC, dtype=torch.int32, device=dev)
+        pe = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
+        for _ in range(3):
+            pkg.hg_kv_read_probe(prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end, sink, prob.desc)
+        for e in pe:
+            e[0].record(stream)
+            pkg.hg_kv_read_probe(prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end, sink, prob.desc)
+            e[1].record(stream)
+        torch.cuda.synchronize()
+        probe_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in pe)
+
+    times = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms = times.tolist()
+
+    if rank == 0:
+        tokens = w.gpu_tokens
+        ms_step = ms_total / args.steps
+        peak, peak_kind = measured_peak()
+        kv_bytes = w.kv_bytes()
+        nchunks = sum(w.chunk_grid(b)[1] for b in range(w.B))
+        part_alg = kv_bytes + w.B * w.Hq * w.D * 2 + (prob.kv["num_pages"] * 4 if w.paged else 0) + \
+            w.Hq * nchunks * (w.D + 2) * 4
+        part_avg = statistics.mean(part_ms)
+        achieved = part_alg / (part_avg * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": world * tokens / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": args.workload, "batch": w.B, "q_heads": w.Hq, "kv_heads": w.Hkv, "head_dim": w.D,
+                       "kv_dtype": w.dtype, "context": max(w.seq_lens), "gpu_tokens": tokens, "page_size": w.page_size,
+                       "chunk_tokens": w.chunk_tokens, "kv_bytes_per_step": kv_bytes,
+                       "l2": "inputs larger than L2" if kv_bytes > 2 * 126e6 else "inputs fit L2 (launch-bound case)",
+                       "step_gbs": prob.alg_bytes() / (ms_step * 1e-3) / 1e9,
+                       "step_frac_of_8000": prob.alg_bytes() / (ms_step * 1e-3) / 1e9 / 8000.0,
+                       "partial_us": part_avg * 1e3, "merge_us": statistics.mean(merge_ms) * 1e3,
+                       "roofline_timing": "second pass of K steps with CUDA events around each kernel",
+                       "probe_us": None if probe_ms is None else probe_ms * 1e3},
+            "roofline": {"bound": "hbm", "kernel": "partial_kernel", "achieved": achieved, "peak": peak,
+                         "peak_kind": f"{peak_kind} copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
+                         "frac_of_8000": achieved / 8000.0, "alg_bytes_per_launch": part_alg,
+                         "traffic": NCU_TRAFFIC_BYTES.get(args.workload)},
+            "e2e": {"value": world * tokens / (e2e_ms / args.steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps, "matches_device_path": bool(same),
+                    "api": "hg_attn_decode_host (KV pools stay device resident: they are the GPU's slice of the cache)"},
+            "gpu_launches": 2 * args.steps,
+            "clocks": clocks,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = time_oracle(w, dev)[0]
+        elif world == 1:
+            line["cpu_baseline"] = None
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

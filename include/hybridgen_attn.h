@@ -1,0 +1,199 @@
+/*
+ * hybridgen_attn.h - C ABI of the B200 (sm_100a) decode-attention library for CPU-GPU hybrid
+ * attention with the KV cache split along the token axis ("attention logit parallelism",
+ * Section 4.2 of the HybridGen paper).
+ *
+ * The GPU holds a slice [tok_begin, tok_end) of every sequence's KV cache; the host holds the
+ * rest.  Attention logits are independent per token (Section 4.2), so each side can process its
+ * own tokens.  This library does the device side in two calls:
+ *
+ *   hg_attn_partial  per (sequence, query head, KV chunk): the scaled logits
+ *                    s_t = <q, K_t> / sqrt(D) (Section 2.1), the chunk maximum m, the exp-sum
+ *                    l = sum e^{s_t - m} and the un-normalised value aggregate
+ *                    o = sum e^{s_t - m} V_t  (workflow step 4 plus the device-local part of step 5)
+ *   hg_attn_merge    log-sum-exp combination of any number of such partials (GPU chunks and
+ *                    partials for the host-held slice) into softmax(q K^T / sqrt(D)) V and its
+ *                    log-sum-exp.  It stands for the Token Concatenator + softmax + value
+ *                    aggregation of Section 4.2 / workflow step 5 and gives the same result as
+ *                    monolithic attention over the union of the token sets.
+ *
+ * Conventions
+ *   - Plain C linkage; all structs are PODs that start with their own size.
+ *   - "dev" pointers are device memory, "host" pointers ordinary host memory.  The caller owns
+ *     every buffer; except where an entry point says otherwise the library allocates nothing,
+ *     keeps no mutable global state, never synchronises the device and never aborts.
+ *   - Work is enqueued on the given CUDA stream (a cudaStream_t passed as void*; NULL = the
+ *     legacy default stream) and runs asynchronously.
+ *   - Every entry point returns an hg_status.  When validation fails nothing is launched.
+ *   - m and lse are in natural-log units.  An empty chunk is (m, l, o) = (-inf, 0, 0); merging only
+ *     empty sources gives out = 0, lse = -inf.  No NaN is produced for finite inputs.
+ *   - Query head h reads KV head h / (num_q_heads / num_kv_heads) (consecutive grouping).
+ *   - Decode step: the single query of a sequence attends every cached token of its slice; there
+ *     is no mask inside the step (the new token's K, V are appended before attention, Section 2.1).
+ */
+#ifndef HYBRIDGEN_ATTN_H_
+#define HYBRIDGEN_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HG_VERSION 0x00010000u /* major.minor.patch = 0.1.0 */
+
+typedef enum hg_status {
+    HG_OK = 0,
+    HG_ERR_INVALID_ARG = 1, /* null pointer, bad size, misaligned base or stride, struct too small */
+    HG_ERR_UNSUPPORTED = 2, /* valid but not implemented (head_dim, page size, group size ...) */
+    HG_ERR_CUDA = 3,        /* a CUDA call or the launch failed (see cudaGetLastError) */
+    HG_ERR_WORKSPACE = 4    /* caller workspace too small / problem exceeds a fixed scratch limit */
+} hg_status;
+
+typedef enum hg_dtype { HG_DTYPE_F16 = 0, HG_DTYPE_BF16 = 1 } hg_dtype;
+
+/* bits of hg_attn_desc.flags */
+#define HG_FLAG_NONE 0u
+
+/* values the kernels may write to *hg_attn_desc.status (device word, optional) */
+#define HG_DEV_OK 0
+#define HG_DEV_WAIT_TIMEOUT 1 /* a bounded on-chip barrier wait ran out; results are invalid (m_part of
+                                 the affected items is NaN).  While the word holds this value the
+                                 kernels skip their work, so clear it before the next call. */
+#define HG_DEV_BAD_PAGE 2     /* a block-table entry of a resident page was outside [0, num_pages) */
+
+/*
+ * Problem description (host struct).
+ *
+ * KV pool addressing, in elements of the 16-bit dtype, for token t of sequence b, KV head g,
+ * component d (the innermost D elements are contiguous):
+ *     page   = block_table ? block_table[b * max_pages + t / page_size] : b * max_pages + t / page_size
+ *     offset = page * page_stride + g * head_stride + (t % page_size) * tok_stride + d
+ * K and V pools share this addressing.  Only pages that overlap [tok_begin, tok_end) are
+ * dereferenced; other block-table entries may be -1.  Whole resident pages may be read,
+ * including rows outside the slice, but such rows never influence a result.
+ * Requirements: head_dim in {64, 128}; page_size in {16, 32, 64, 128, 256}; pool base addresses
+ * 16-byte aligned; every stride a multiple of 8 elements; chunk_tokens a multiple of 64 and of
+ * page_size, at most 65536.
+ *
+ * Chunk grid: chunks sit on absolute multiples of chunk_tokens.  Chunk c of sequence b covers
+ *     [(tok_begin[b] / chunk_tokens + c) * chunk_tokens, + chunk_tokens)  intersected with
+ *     [tok_begin[b], tok_end[b]),
+ * so nc_b = ceil(tok_end / chunk_tokens) - floor(tok_begin / chunk_tokens) chunks are non-empty
+ * (0 when the slice is empty).  num_chunks must be >= every nc_b; slots c >= nc_b are written as
+ * empty partials.
+ */
+typedef struct hg_attn_desc {
+    uint32_t struct_size;      /* sizeof(hg_attn_desc) as compiled by the caller */
+    int32_t batch;             /* B  >= 1 */
+    int32_t num_q_heads;       /* Hq, a multiple of num_kv_heads */
+    int32_t num_kv_heads;      /* Hkv */
+    int32_t head_dim;          /* D */
+    int32_t dtype;             /* hg_dtype of q, K and V */
+    int32_t page_size;         /* tokens per page */
+    int32_t num_pages;         /* pages in each pool */
+    int64_t page_stride;       /* elements */
+    int64_t head_stride;       /* elements */
+    int64_t tok_stride;        /* elements */
+    const int32_t* block_table; /* dev [B][max_pages], or NULL for identity paging */
+    int32_t max_pages;         /* row length of block_table */
+    int32_t chunk_tokens;      /* C */
+    int32_t num_chunks;        /* NC: chunk slots per (sequence, head) in o/m/l_part */
+    float scale;               /* logit scale; 0 means 1/sqrt(D) */
+    uint32_t flags;            /* HG_FLAG_* */
+    int32_t* status;           /* dev, optional: receives HG_DEV_* if a kernel detects a problem */
+} hg_attn_desc;
+
+/* One source of partials for hg_attn_merge (host struct, dev pointers). */
+typedef struct hg_partial_src {
+    const float* o; /* dev [B][Hq][nc][D] */
+    const float* m; /* dev [B][Hq][nc]    */
+    const float* l; /* dev [B][Hq][nc]    */
+    int32_t nc;     /* partials per (sequence, head) in this source, >= 1 */
+    int32_t reserved;
+} hg_partial_src;
+
+/*
+ * Scaled logits, chunk max, exp-sum and un-normalised P.V for the GPU-resident slice
+ * (Section 2.1 for the logit definition; Section 4.2 and workflow step 4 for the token split).
+ *
+ *   q          dev [B][Hq][D], dtype as desc->dtype, 16-byte aligned
+ *   k_cache    dev K pool, v_cache dev V pool (addressing above)
+ *   seq_lens   dev int32 [B]   cached tokens per sequence
+ *   tok_begin  dev int32 [B]   0 <= tok_begin <= tok_end <= seq_len
+ *   tok_end    dev int32 [B]
+ *   o_part     dev float [B][Hq][NC][D]  out: sum_t e^{s_t - m} V_t
+ *   m_part     dev float [B][Hq][NC]     out: exact fp32 chunk maximum of the scaled logits
+ *   l_part     dev float [B][Hq][NC]     out: sum_t e^{s_t - m}
+ * Ranges are read on the device, so the call never waits for the GPU; a slice that needs more
+ * than num_chunks chunks is truncated to its first num_chunks chunks.
+ * Accumulation is fp32.  For num_q_heads > num_kv_heads the P.V product runs on tensor cores with
+ * P carried as a two-term (hi + lo) 16-bit expansion.
+ * Errors: HG_ERR_INVALID_ARG / HG_ERR_UNSUPPORTED before any launch; HG_ERR_CUDA if the launch fails.
+ */
+hg_status hg_attn_partial(const void* q, const void* k_cache, const void* v_cache, const int32_t* seq_lens,
+                          const int32_t* tok_begin, const int32_t* tok_end, float* o_part, float* m_part,
+                          float* l_part, void* stream, const hg_attn_desc* desc);
+
+/*
+ * Log-sum-exp merge and normalisation (stands for concatenation + softmax + value aggregation of
+ * Section 4.2 / workflow step 5; result identical, up to rounding order, to attention over the
+ * union of the sources' token sets).
+ *
+ *   partials  host array of n_src sources (n_src >= 1); each source's arrays are dev memory
+ *   out       dev float [B][Hq][D]   sum_i w_i o_i / sum_i w_i l_i,  w_i = e^{m_i - max_j m_j}
+ *   lse       dev float [B][Hq]      max_j m_j + ln sum_i w_i l_i   (may be NULL)
+ * Only batch, num_q_heads and head_dim of desc are used.  n_src <= HG_MAX_MERGE_SRC.
+ */
+#define HG_MAX_MERGE_SRC 8
+hg_status hg_attn_merge(const hg_partial_src* partials, int32_t n_src, float* out, float* lse, void* stream,
+                        const hg_attn_desc* desc);
+
+/*
+ * Bytes of device workspace hg_attn_decode / hg_attn_decode_host need for this problem
+ * (chunk partials, plus staging for q, ranges, host partials and results in the _host form).
+ * Returns 0 for an invalid description.
+ */
+size_t hg_attn_workspace_bytes(const hg_attn_desc* desc, int32_t n_host_src);
+
+/*
+ * One pass of the whole path: hg_attn_partial into workspace, then hg_attn_merge of those
+ * chunk partials with n_host_src further sources (partials for the host-held slice, already in
+ * device memory).  workspace: dev, 256-byte aligned, at least hg_attn_workspace_bytes().
+ */
+hg_status hg_attn_decode(const void* q, const void* k_cache, const void* v_cache, const int32_t* seq_lens,
+                         const int32_t* tok_begin, const int32_t* tok_end, const hg_partial_src* host_partials,
+                         int32_t n_host_src, float* out, float* lse, void* workspace, size_t workspace_bytes,
+                         void* stream, const hg_attn_desc* desc);
+
+/*
+ * The same pass for a caller whose per-step data lives in HOST memory: q, the three range arrays,
+ * the host-slice partials (hg_partial_src with HOST pointers here) and the results out / lse are
+ * host buffers (pinned memory makes the copies asynchronous); they are staged through the device
+ * workspace with cudaMemcpyAsync on the stream.  The KV pools and the block table stay device
+ * resident - they are the GPU's slice of the cache, not per-step input.  Returns after enqueuing;
+ * out / lse are valid once the stream has been synchronised.
+ */
+hg_status hg_attn_decode_host(const void* q_host, const void* k_cache, const void* v_cache,
+                              const int32_t* seq_lens_host, const int32_t* tok_begin_host,
+                              const int32_t* tok_end_host, const hg_partial_src* host_partials_host,
+                              int32_t n_host_src, float* out_host, float* lse_host, void* workspace,
+                              size_t workspace_bytes, void* stream, const hg_attn_desc* desc);
+
+/*
+ * Evidence kernel, not part of the attention path: streams the same K and V tiles through the
+ * same TMA pipeline as hg_attn_partial and folds them into one 32-bit checksum per work item
+ * (sink: dev uint32 [B][Hkv][NC]).  Used to measure the read ceiling of the paged access pattern.
+ */
+hg_status hg_kv_read_probe(const void* k_cache, const void* v_cache, const int32_t* seq_lens,
+                           const int32_t* tok_begin, const int32_t* tok_end, uint32_t* sink, void* stream,
+                           const hg_attn_desc* desc);
+
+const char* hg_status_string(hg_status s);
+uint32_t hg_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HYBRIDGEN_ATTN_H_ */

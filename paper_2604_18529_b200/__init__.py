@@ -1,1 +1,22 @@
-"""B200-native hybrid decode attention (partials + LSE merge)."""
+"""B200-native decode attention over the GPU-resident slice of a long KV cache:
+per-chunk softmax partials (``hg_attn_partial``) and their log-sum-exp merge with
+partials for the host-held slice (``hg_attn_merge``).
+
+The arithmetic runs in the CUDA library under ``csrc/``; this package only marshals
+arguments. Importing it does not load the library; the first call does, and raises if
+the library has not been built.
+"""
+from .binding import (  # noqa: F401
+    HgError,
+    lib,
+    lib_path,
+    attn_desc,
+    hg_attn_partial,
+    hg_attn_merge,
+    hg_attn_decode,
+    hg_attn_decode_host,
+    hg_attn_workspace_bytes,
+    hg_status_string,
+    hg_kv_read_probe,
+    hg_version,
+)

@@ -1,0 +1,351 @@
+// Host side of the C ABI declared in include/hybridgen_attn.h: argument validation, TMA tensor-map
+// encoding, launches.  No allocation, no synchronisation, no global mutable state (the cached
+// driver entry point and the per-kernel shared-memory opt-in are idempotent).
+#include "hybridgen_attn.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include "hg_merge.cuh"
+#include "hg_partial.cuh"
+
+namespace hg {
+
+// ---- validation ------------------------------------------------------------------------------------
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int ilog2_exact(int v) {
+    for (int s = 0; s < 31; ++s)
+        if ((1 << s) == v) return s;
+    return -1;
+}
+
+// Checks the fields every entry point relies on.  `need_kv` also checks the KV addressing.
+static hg_status check_desc(const hg_attn_desc* d, bool need_kv) {
+    if (!d || d->struct_size < sizeof(hg_attn_desc)) return HG_ERR_INVALID_ARG;
+    if (d->batch < 1 || d->batch > 65535) return HG_ERR_INVALID_ARG;
+    if (d->num_kv_heads < 1 || d->num_q_heads < 1 || d->num_q_heads % d->num_kv_heads) return HG_ERR_INVALID_ARG;
+    if (d->head_dim <= 0 || d->head_dim % 8) return HG_ERR_INVALID_ARG;
+    if (d->head_dim != 64 && d->head_dim != 128) return HG_ERR_UNSUPPORTED;
+    if (!need_kv) return HG_OK;
+    if (d->dtype != HG_DTYPE_F16 && d->dtype != HG_DTYPE_BF16) return HG_ERR_INVALID_ARG;
+    if (d->page_size < 1 || d->num_pages < 1 || d->max_pages < 1) return HG_ERR_INVALID_ARG;
+    if (d->page_stride < 0 || d->head_stride < 0 || d->tok_stride < d->head_dim) return HG_ERR_INVALID_ARG;
+    if ((d->page_stride | d->head_stride | d->tok_stride) & 7) return HG_ERR_INVALID_ARG;   // 16-byte multiples
+    if (d->chunk_tokens < 1 || d->num_chunks < 1) return HG_ERR_INVALID_ARG;
+    if (!(d->scale >= 0.f) || isinf(d->scale)) return HG_ERR_INVALID_ARG;
+    const int shift = ilog2_exact(d->page_size);
+    if (shift < 4 || shift > 8) return HG_ERR_UNSUPPORTED;                                   // 16 .. 256
+    if (d->chunk_tokens % TILE_T || d->chunk_tokens % d->page_size || d->chunk_tokens > 65536)
+        return HG_ERR_UNSUPPORTED;
+    if (d->chunk_tokens / d->page_size > MAX_CHUNK_PAGES) return HG_ERR_UNSUPPORTED;
+    if ((int64_t)d->num_kv_heads * ((d->num_q_heads / d->num_kv_heads + 7) / 8) > 65535) return HG_ERR_UNSUPPORTED;
+    if (!d->block_table && (int64_t)d->batch * d->max_pages > d->num_pages) return HG_ERR_INVALID_ARG;
+    return HG_OK;
+}
+
+// ---- tensor maps -------------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = []() -> EncodeTiledFn {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &f, 12000, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        return reinterpret_cast<EncodeTiledFn>(f);
+    }();
+    return fn;
+}
+
+// Pool viewed as a 4-D tensor {d, x, y, z} where x, y, z are token-in-page, head and page ordered by
+// ascending stride; one box is 64 d-elements (128 bytes, swizzled) x `rows` tokens.
+static hg_status make_maps(const hg_attn_desc* d, const void* k, const void* v, CUtensorMap* tk, CUtensorMap* tv,
+                           int perm[3]) {
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return HG_ERR_CUDA;
+    const int rows = d->page_size >= TILE_T ? TILE_T : d->page_size;
+    int64_t stride[3] = {d->tok_stride, d->head_stride, d->page_stride};
+    int64_t extent[3] = {d->page_size, d->num_kv_heads, d->num_pages};
+    int order[3] = {0, 1, 2};
+    for (int i = 0; i < 3; ++i)                       // insertion sort, stable
+        for (int j = i; j > 0 && stride[order[j]] < stride[order[j - 1]]; --j) {
+            int t = order[j]; order[j] = order[j - 1]; order[j - 1] = t;
+        }
+    cuuint64_t dims[4] = {(cuuint64_t)d->head_dim, 0, 0, 0};
+    cuuint64_t strides[3];
+    cuuint32_t box[4] = {64, 1, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    for (int i = 0; i < 3; ++i) {
+        dims[1 + i] = (cuuint64_t)extent[order[i]];
+        strides[i] = (cuuint64_t)stride[order[i]] * 2u;
+        if (order[i] == 0) box[1 + i] = (cuuint32_t)rows;
+        perm[i] = order[i];
+    }
+    const CUtensorMapDataType dt = d->dtype == HG_DTYPE_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+    const void* base[2] = {k, v};
+    CUtensorMap* out[2] = {tk, tv};
+    for (int i = 0; i < 2; ++i) {
+        CUresult r = enc(out[i], dt, 4, const_cast<void*>(base[i]), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return HG_ERR_UNSUPPORTED;   // a stride pattern the TMA unit cannot express
+    }
+    return HG_OK;
+}
+
+// ---- launches ---------------------------------------------------------------------------------------
+
+static int env_int(const char* name, int dflt, int lo, int hi) {
+    const char* s = getenv(name);
+    if (!s || !*s) return dflt;
+    int v = atoi(s);
+    return v < lo ? lo : (v > hi ? hi : v);
+}
+
+template <int D, bool BF16, int MODE>
+static hg_status launch_partial_t(const CUtensorMap& tk, const CUtensorMap& tv, const PartialParams& p, dim3 grid,
+                                  cudaStream_t st) {
+    const size_t smem = (size_t)p.stages * (D / 64) * HALF_BYTES + 1024;
+    auto kern = partial_kernel<D, BF16, MODE>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+        cudaGetLastError();
+        return HG_ERR_CUDA;
+    }
+    kern<<<grid, THREADS, smem, st>>>(tk, tv, p);
+    return cudaGetLastError() == cudaSuccess ? HG_OK : HG_ERR_CUDA;
+}
+
+template <int MODE>
+static hg_status launch_partial_m(int D, bool bf16, const CUtensorMap& tk, const CUtensorMap& tv, const PartialParams& p,
+                                  dim3 grid, cudaStream_t st) {
+    if (D == 128) return bf16 ? launch_partial_t<128, true, MODE>(tk, tv, p, grid, st) : launch_partial_t<128, false, MODE>(tk, tv, p, grid, st);
+    return bf16 ? launch_partial_t<64, true, MODE>(tk, tv, p, grid, st) : launch_partial_t<64, false, MODE>(tk, tv, p, grid, st);
+}
+
+static hg_status run_partial(int mode, const void* q, const void* k, const void* v, const int32_t* seq_lens,
+                             const int32_t* tok_begin, const int32_t* tok_end, float* o_part, float* m_part, float* l_part,
+                             uint32_t* sink, void* stream, const hg_attn_desc* d) {
+    hg_status st = check_desc(d, true);
+    if (st != HG_OK) return st;
+    if (!k || !v || !seq_lens || !tok_begin || !tok_end) return HG_ERR_INVALID_ARG;
+    if (mode == MODE_PROBE) {
+        if (!sink) return HG_ERR_INVALID_ARG;
+    } else if (!q || !o_part || !m_part || !l_part) {
+        return HG_ERR_INVALID_ARG;
+    }
+    if (!aligned16(k) || !aligned16(v) || (q && !aligned16(q)) || (o_part && !aligned16(o_part))) return HG_ERR_INVALID_ARG;
+
+    PartialParams p;
+    memset(&p, 0, sizeof p);
+    CUtensorMap tk, tv;
+    int perm[3];
+    st = make_maps(d, k, v, &tk, &tv, perm);
+    if (st != HG_OK) return st;
+    const int G = d->num_q_heads / d->num_kv_heads;
+    if (mode != MODE_PROBE) mode = (G == 1) ? MODE_MHA : MODE_GQA;
+    p.q = q; p.seq_lens = seq_lens; p.tok_begin = tok_begin; p.tok_end = tok_end; p.block_table = d->block_table;
+    p.o_part = o_part; p.m_part = m_part; p.l_part = l_part; p.sink = sink; p.status = d->status;
+    p.B = d->batch; p.Hq = d->num_q_heads; p.Hkv = d->num_kv_heads; p.G = G;
+    p.page_size = d->page_size; p.page_shift = ilog2_exact(d->page_size); p.max_pages = d->max_pages;
+    p.num_pages = d->num_pages; p.C = d->chunk_tokens; p.NC = d->num_chunks;
+    p.head_blocks = (mode == MODE_GQA) ? (G + 7) / 8 : 1;
+    p.perm0 = perm[0]; p.perm1 = perm[1]; p.perm2 = perm[2];
+    const float scale = d->scale > 0.f ? d->scale : 1.0f / sqrtf((float)d->head_dim);
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.stages = env_int("HG_ATTN_STAGES", d->head_dim == 128 ? 4 : 8, 2, MAX_STAGES);
+    dim3 grid((unsigned)d->num_chunks, (unsigned)(d->num_kv_heads * p.head_blocks), (unsigned)d->batch);
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const bool bf16 = d->dtype == HG_DTYPE_BF16;
+    switch (mode) {
+        case MODE_MHA: return launch_partial_m<MODE_MHA>(d->head_dim, bf16, tk, tv, p, grid, cs);
+        case MODE_GQA: return launch_partial_m<MODE_GQA>(d->head_dim, bf16, tk, tv, p, grid, cs);
+        default: return launch_partial_m<MODE_PROBE>(d->head_dim, bf16, tk, tv, p, grid, cs);
+    }
+}
+
+static hg_status run_merge(const hg_partial_src* src, int32_t n_src, float* out, float* lse, void* stream,
+                           const hg_attn_desc* d) {
+    hg_status st = check_desc(d, false);
+    if (st != HG_OK) return st;
+    if (!src || n_src < 1 || n_src > HG_MAX_MERGE_SRC || !out) return HG_ERR_INVALID_ARG;
+    MergeParams p;
+    memset(&p, 0, sizeof p);
+    for (int i = 0; i < n_src; ++i) {
+        if (!src[i].o || !src[i].m || !src[i].l || src[i].nc < 1) return HG_ERR_INVALID_ARG;
+        if (!aligned16(src[i].o)) return HG_ERR_INVALID_ARG;
+        p.o[i] = src[i].o; p.m[i] = src[i].m; p.l[i] = src[i].l; p.nc[i] = src[i].nc;
+        p.total += src[i].nc;
+    }
+    p.n_src = n_src; p.out = out; p.lse = lse;
+
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3((unsigned)(d->batch * d->num_q_heads));
+    cfg.blockDim = dim3(MERGE_THREADS);
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;     // start while the producer of the partials drains
+    cfg.attrs = attr;
+    cfg.numAttrs = env_int("HG_ATTN_PDL", 1, 0, 1);
+    cudaError_t e = d->head_dim == 128 ? cudaLaunchKernelEx(&cfg, merge_kernel<128>, p)
+                                       : cudaLaunchKernelEx(&cfg, merge_kernel<64>, p);
+    if (e != cudaSuccess) { cudaGetLastError(); return HG_ERR_CUDA; }
+    return HG_OK;
+}
+
+// ---- workspace layout for the fused entry points ---------------------------------------------------------
+
+static size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+struct Workspace {
+    size_t o_part, m_part, l_part;           // chunk partials
+    size_t q, seq_lens, tok_begin, tok_end;  // staging (host form only)
+    size_t host_part;                        // staged host partials, n_host_partials * (D + 2) floats per row + slack
+    size_t out, lse;
+    size_t total;
+};
+
+static Workspace plan_workspace(const hg_attn_desc* d, int n_host_partials, int n_host_src) {
+    Workspace w;
+    const size_t rows = (size_t)d->batch * d->num_q_heads;
+    size_t off = 0;
+    w.o_part = off; off += up256(rows * d->num_chunks * d->head_dim * sizeof(float));
+    w.m_part = off; off += up256(rows * d->num_chunks * sizeof(float));
+    w.l_part = off; off += up256(rows * d->num_chunks * sizeof(float));
+    w.q = off; off += up256(rows * d->head_dim * 2);
+    w.seq_lens = off; off += up256((size_t)d->batch * 4);
+    w.tok_begin = off; off += up256((size_t)d->batch * 4);
+    w.tok_end = off; off += up256((size_t)d->batch * 4);
+    w.host_part = off; off += up256(rows * (size_t)n_host_partials * (d->head_dim + 2) * sizeof(float)) + (size_t)n_host_src * 3 * 256;
+    w.out = off; off += up256(rows * d->head_dim * sizeof(float));
+    w.lse = off; off += up256(rows * sizeof(float));
+    w.total = off;
+    return w;
+}
+
+}  // namespace hg
+
+using namespace hg;
+
+extern "C" {
+
+hg_status hg_attn_partial(const void* q, const void* k_cache, const void* v_cache, const int32_t* seq_lens,
+                          const int32_t* tok_begin, const int32_t* tok_end, float* o_part, float* m_part, float* l_part,
+                          void* stream, const hg_attn_desc* desc) {
+    return run_partial(MODE_MHA, q, k_cache, v_cache, seq_lens, tok_begin, tok_end, o_part, m_part, l_part, nullptr,
+                       stream, desc);
+}
+
+hg_status hg_kv_read_probe(const void* k_cache, const void* v_cache, const int32_t* seq_lens, const int32_t* tok_begin,
+                           const int32_t* tok_end, uint32_t* sink, void* stream, const hg_attn_desc* desc) {
+    return run_partial(MODE_PROBE, nullptr, k_cache, v_cache, seq_lens, tok_begin, tok_end, nullptr, nullptr, nullptr,
+                       sink, stream, desc);
+}
+
+hg_status hg_attn_merge(const hg_partial_src* partials, int32_t n_src, float* out, float* lse, void* stream,
+                        const hg_attn_desc* desc) {
+    return run_merge(partials, n_src, out, lse, stream, desc);
+}
+
+size_t hg_attn_workspace_bytes(const hg_attn_desc* desc, int32_t n_host_partials) {
+    if (check_desc(desc, true) != HG_OK || n_host_partials < 0) return 0;
+    return plan_workspace(desc, n_host_partials, HG_MAX_MERGE_SRC).total;
+}
+
+hg_status hg_attn_decode(const void* q, const void* k_cache, const void* v_cache, const int32_t* seq_lens,
+                         const int32_t* tok_begin, const int32_t* tok_end, const hg_partial_src* host_partials,
+                         int32_t n_host_src, float* out, float* lse, void* workspace, size_t workspace_bytes, void* stream,
+                         const hg_attn_desc* desc) {
+    hg_status st = check_desc(desc, true);
+    if (st != HG_OK) return st;
+    if (n_host_src < 0 || n_host_src > HG_MAX_MERGE_SRC - 1 || (n_host_src && !host_partials)) return HG_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HG_ERR_INVALID_ARG;
+    const Workspace w = plan_workspace(desc, 0, 0);
+    if (workspace_bytes < w.q) return HG_ERR_WORKSPACE;          // only the chunk partials are needed here
+    char* ws = static_cast<char*>(workspace);
+    float* o_part = reinterpret_cast<float*>(ws + w.o_part);
+    float* m_part = reinterpret_cast<float*>(ws + w.m_part);
+    float* l_part = reinterpret_cast<float*>(ws + w.l_part);
+    st = run_partial(MODE_MHA, q, k_cache, v_cache, seq_lens, tok_begin, tok_end, o_part, m_part, l_part, nullptr, stream, desc);
+    if (st != HG_OK) return st;
+    hg_partial_src src[HG_MAX_MERGE_SRC];
+    src[0].o = o_part; src[0].m = m_part; src[0].l = l_part; src[0].nc = desc->num_chunks; src[0].reserved = 0;
+    for (int i = 0; i < n_host_src; ++i) src[1 + i] = host_partials[i];
+    return run_merge(src, 1 + n_host_src, out, lse, stream, desc);
+}
+
+hg_status hg_attn_decode_host(const void* q_host, const void* k_cache, const void* v_cache, const int32_t* seq_lens_host,
+                              const int32_t* tok_begin_host, const int32_t* tok_end_host,
+                              const hg_partial_src* host_partials_host, int32_t n_host_src, float* out_host, float* lse_host,
+                              void* workspace, size_t workspace_bytes, void* stream, const hg_attn_desc* desc) {
+    hg_status st = check_desc(desc, true);
+    if (st != HG_OK) return st;
+    if (!q_host || !seq_lens_host || !tok_begin_host || !tok_end_host || !out_host) return HG_ERR_INVALID_ARG;
+    if (n_host_src < 0 || n_host_src > HG_MAX_MERGE_SRC - 1 || (n_host_src && !host_partials_host)) return HG_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HG_ERR_INVALID_ARG;
+    int n_host_partials = 0;
+    for (int i = 0; i < n_host_src; ++i) {
+        const hg_partial_src& s = host_partials_host[i];
+        if (!s.o || !s.m || !s.l || s.nc < 1) return HG_ERR_INVALID_ARG;
+        n_host_partials += s.nc;
+    }
+    const Workspace w = plan_workspace(desc, n_host_partials, n_host_src);
+    if (workspace_bytes < w.total) return HG_ERR_WORKSPACE;
+    char* ws = static_cast<char*>(workspace);
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const size_t rows = (size_t)desc->batch * desc->num_q_heads;
+    const int D = desc->head_dim;
+    bool ok = true;
+    ok &= cudaMemcpyAsync(ws + w.q, q_host, rows * D * 2, cudaMemcpyHostToDevice, cs) == cudaSuccess;
+    ok &= cudaMemcpyAsync(ws + w.seq_lens, seq_lens_host, (size_t)desc->batch * 4, cudaMemcpyHostToDevice, cs) == cudaSuccess;
+    ok &= cudaMemcpyAsync(ws + w.tok_begin, tok_begin_host, (size_t)desc->batch * 4, cudaMemcpyHostToDevice, cs) == cudaSuccess;
+    ok &= cudaMemcpyAsync(ws + w.tok_end, tok_end_host, (size_t)desc->batch * 4, cudaMemcpyHostToDevice, cs) == cudaSuccess;
+    hg_partial_src dev_src[HG_MAX_MERGE_SRC];
+    size_t off = w.host_part;
+    for (int i = 0; i < n_host_src && ok; ++i) {
+        const hg_partial_src& s = host_partials_host[i];
+        const size_t ob = rows * s.nc * D * sizeof(float), mb = rows * s.nc * sizeof(float);
+        dev_src[i].nc = s.nc; dev_src[i].reserved = 0;
+        dev_src[i].o = reinterpret_cast<const float*>(ws + off);
+        ok &= cudaMemcpyAsync(ws + off, s.o, ob, cudaMemcpyHostToDevice, cs) == cudaSuccess; off += up256(ob);
+        dev_src[i].m = reinterpret_cast<const float*>(ws + off);
+        ok &= cudaMemcpyAsync(ws + off, s.m, mb, cudaMemcpyHostToDevice, cs) == cudaSuccess; off += up256(mb);
+        dev_src[i].l = reinterpret_cast<const float*>(ws + off);
+        ok &= cudaMemcpyAsync(ws + off, s.l, mb, cudaMemcpyHostToDevice, cs) == cudaSuccess; off += up256(mb);
+    }
+    if (!ok) { cudaGetLastError(); return HG_ERR_CUDA; }
+    float* out_dev = reinterpret_cast<float*>(ws + w.out);
+    float* lse_dev = reinterpret_cast<float*>(ws + w.lse);
+    st = hg_attn_decode(ws + w.q, k_cache, v_cache, reinterpret_cast<const int32_t*>(ws + w.seq_lens),
+                        reinterpret_cast<const int32_t*>(ws + w.tok_begin), reinterpret_cast<const int32_t*>(ws + w.tok_end),
+                        dev_src, n_host_src, out_dev, lse_dev, workspace, workspace_bytes, stream, desc);
+    if (st != HG_OK) return st;
+    ok &= cudaMemcpyAsync(out_host, out_dev, rows * D * sizeof(float), cudaMemcpyDeviceToHost, cs) == cudaSuccess;
+    if (lse_host) ok &= cudaMemcpyAsync(lse_host, lse_dev, rows * sizeof(float), cudaMemcpyDeviceToHost, cs) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return HG_ERR_CUDA; }
+    return HG_OK;
+}
+
+const char* hg_status_string(hg_status s) {
+    switch (s) {
+        case HG_OK: return "ok";
+        case HG_ERR_INVALID_ARG: return "invalid argument";
+        case HG_ERR_UNSUPPORTED: return "unsupported configuration";
+        case HG_ERR_CUDA: return "CUDA error";
+        case HG_ERR_WORKSPACE: return "workspace too small";
+        default: return "unknown status";
+    }
+}
+
+uint32_t hg_version(void) { return HG_VERSION; }
+
+}  // extern "C"

@@ -1,0 +1,247 @@
+"""GPU path vs the fp64 oracle, element by element, through the C ABI (via the thin binding).
+
+Sizes are small enough for the whole-tensor oracle yet span several 64-token tiles, several chunks
+and ragged first/last tiles.  Tolerances (parity_util): out max-abs 2e-3, rel-L2 1e-3, LSE 1e-4.
+"""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2604_18529_b200 as pkg
+from paper_2604_18529_b200 import binding as hg
+from paper_2604_18529_b200 import workload as W
+from paper_2604_18529_b200.problem import DeviceProblem
+from parity_util import OracleRef, bits, check_output, check_partials
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def run_and_check(w, poison_tail=False, what=None):
+    what = what or w.name
+    ref = OracleRef(w)
+    prob = DeviceProblem(w, DEV, poison_tail=poison_tail)
+    prob.partial()
+    torch.cuda.synchronize()
+    assert int(prob.status.item()) == hg.HG_DEV_OK, what
+    rm, rl, ro = ref.chunk_partials(w.chunk_tokens, prob.NC)
+    check_partials(prob.o_part.reshape(-1, w.D), prob.m_part.reshape(-1), prob.l_part.reshape(-1),
+                   rm.reshape(-1), rl.reshape(-1), ro.reshape(-1, w.D), what)
+    prob.merge(ref.host_partials_device(DEV))
+    torch.cuda.synchronize()
+    return prob, ref, check_output(prob.out, prob.lse, ref.out, ref.lse, what)
+
+
+def wl(**kw):
+    base = dict(name="case", B=2, Hq=4, Hkv=2, D=128, dtype="f16", seq_lens=[700, 333], tok_begin=[130, 5],
+                tok_end=[700, 290], page_size=16, layout="HND", chunk_tokens=128, seed=11)
+    base.update(kw)
+    return W.AttnWorkload(**base)
+
+
+# ---- the five benchmark configurations, scaled down ------------------------------------------------
+
+@pytest.mark.parametrize("name", W.WORKLOADS)
+def test_scaled_down_benchmark_configs(name):
+    full = W.make_workload(name)
+    w = full if name == "tiny" else W.scaled_down(full, 64 if name != "ragged" else 16, max_batch=3)
+    run_and_check(w)
+
+
+# ---- shape sweep: head grouping, head_dim, dtype, page size, layout ----------------------------------
+
+@pytest.mark.parametrize("Hq,Hkv", [(2, 2), (3, 3), (4, 1), (8, 1), (6, 2), (16, 1), (12, 1)])
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+def test_head_grouping_sweep(Hq, Hkv, D, dtype):
+    run_and_check(wl(Hq=Hq, Hkv=Hkv, D=D, dtype=dtype, seed=100 + Hq * 7 + D))
+
+
+@pytest.mark.parametrize("page_size", [16, 32, 64, 128, 256])
+@pytest.mark.parametrize("layout,paged", [("HND", True), ("NHD", True), ("NHD", False)])
+@pytest.mark.parametrize("G", [1, 4])
+def test_page_size_and_layout_sweep(page_size, layout, paged, G):
+    chunk = max(128, page_size)
+    w = wl(Hq=2 * G, Hkv=2, page_size=page_size, layout=layout, paged=paged, chunk_tokens=chunk,
+           seq_lens=[900, 517], tok_begin=[77, 0], tok_end=[900, 400], seed=page_size + G)
+    run_and_check(w)
+
+
+@pytest.mark.parametrize("G", [1, 8])
+@pytest.mark.parametrize("chunk", [64, 192, 256, 1024])
+def test_chunk_sizes(G, chunk):
+    w = wl(Hq=G, Hkv=1, chunk_tokens=chunk, seq_lens=[1500, 64], tok_begin=[333, 0], tok_end=[1500, 64], seed=chunk)
+    run_and_check(w)
+
+
+# ---- edge cases ---------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("G", [1, 4])
+@pytest.mark.parametrize("tb,te,L", [
+    (0, 0, 100),          # empty slice at the start
+    (100, 100, 100),      # empty slice at the end
+    (37, 38, 100),        # one token
+    (64, 128, 300),       # exactly one aligned tile
+    (63, 65, 300),        # two tokens straddling a tile boundary
+    (0, 300, 300),        # everything on the GPU, nothing on the host
+    (17, 29, 300),        # inside one page
+    (127, 129, 130),      # straddles a chunk boundary
+])
+def test_slice_edge_cases(G, tb, te, L):
+    w = wl(B=2, Hq=2 * G, Hkv=2, seq_lens=[L, 200], tok_begin=[tb, 10], tok_end=[te, 150], chunk_tokens=128, seed=tb + te)
+    run_and_check(w, what=f"G{G} [{tb},{te}) of {L}")
+
+
+@pytest.mark.parametrize("G", [1, 4])
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+def test_rows_past_seq_len_never_matter(G, dtype):
+    # the last resident page holds NaN patterns after the sequence's final token
+    w = wl(Hq=2 * G, Hkv=2, dtype=dtype, seq_lens=[701, 333], tok_begin=[130, 5], tok_end=[701, 333], seed=5)
+    run_and_check(w, poison_tail=True)
+
+
+@pytest.mark.parametrize("G", [1, 8])
+def test_outlier_tokens(G):
+    w = wl(B=1, Hq=G, Hkv=1, seq_lens=[3000], tok_begin=[1200], tok_end=[3000], outlier_frac=0.01, chunk_tokens=256, seed=9)
+    run_and_check(w)
+
+
+def test_all_slices_empty_gives_zero_and_minus_inf():
+    w = wl(seq_lens=[50, 60], tok_begin=[50, 0], tok_end=[50, 0])
+    prob = DeviceProblem(w, DEV)
+    prob.partial()
+    prob.merge([])
+    torch.cuda.synchronize()
+    assert (prob.out == 0).all() and torch.isinf(prob.lse).all() and (prob.lse < 0).all()
+    assert torch.isinf(prob.m_part).all() and (prob.l_part == 0).all() and (prob.o_part == 0).all()
+
+
+def test_extra_chunk_slots_are_neutral():
+    w = wl()
+    ref = OracleRef(w)
+    prob = DeviceProblem(w, DEV)
+    NC = prob.NC + 3
+    prob.NC = NC
+    prob.desc = prob.make_desc(w.chunk_tokens, NC)
+    prob.o_part = torch.full((w.B, w.Hq, NC, w.D), 7.0, device=DEV)
+    prob.m_part = torch.full((w.B, w.Hq, NC), 7.0, device=DEV)
+    prob.l_part = torch.full((w.B, w.Hq, NC), 7.0, device=DEV)
+    prob.step(ref.host_partials_device(DEV))
+    torch.cuda.synchronize()
+    n1 = w.chunk_grid(1)[1]
+    assert torch.isinf(prob.m_part[1, :, n1:]).all() and (prob.l_part[1, :, n1:] == 0).all()
+    assert (prob.o_part[1, :, n1:] == 0).all()
+    check_output(prob.out, prob.lse, ref.out, ref.lse)
+
+
+# ---- split invariance and reproducibility on the GPU -----------------------------------------------------
+
+@pytest.mark.parametrize("G", [1, 4])
+def test_merged_result_is_invariant_to_chunking_and_bit_reproducible(G):
+    w = wl(Hq=2 * G, Hkv=2, seq_lens=[2100, 900], tok_begin=[400, 100], tok_end=[2100, 900])
+    ref = OracleRef(w)
+    outs = []
+    for chunk in (64, 128, 512, 2048):
+        wc = dataclasses.replace(w, chunk_tokens=chunk)
+        prob = DeviceProblem(wc, DEV)
+        host = ref.host_partials_device(DEV)
+        prob.step(host)
+        torch.cuda.synchronize()
+        check_output(prob.out, prob.lse, ref.out, ref.lse, f"chunk {chunk}")
+        first = (prob.out.clone(), prob.lse.clone(), prob.o_part.clone())
+        prob.step(host)
+        torch.cuda.synchronize()
+        assert torch.equal(prob.out, first[0]) and torch.equal(prob.lse, first[1]) and torch.equal(prob.o_part, first[2])
+        outs.append(prob.out.double().cpu().numpy())
+    for o in outs[1:]:
+        assert np.abs(o - outs[0]).max() <= 2e-3
+
+
+def test_merge_is_invariant_to_how_host_partials_are_split():
+    w = wl(B=1, Hq=4, Hkv=1, seq_lens=[1200], tok_begin=[800], tok_end=[1200])
+    ref = OracleRef(w)
+    prob = DeviceProblem(w, DEV)
+    prob.partial()
+    # host slice [0, 800) as 1, 2 or 5 partials in a single source, or as separate sources
+    from oracle import hg_oracle as O
+    for cuts in ([0, 800], [0, 300, 800], [0, 100, 101, 400, 799, 800]):
+        parts = [O.chunked_partials(ref.q, ref.K, ref.V, w.dtype, [a], [b], 0, 1) for a, b in zip(cuts[:-1], cuts[1:])]
+        m = np.concatenate([p[0] for p in parts], axis=2); l = np.concatenate([p[1] for p in parts], axis=2)
+        o = np.concatenate([p[2] for p in parts], axis=2)
+        src = tuple(torch.from_numpy(x).float().to(DEV) for x in (o, m, l))
+        prob.merge([src])
+        torch.cuda.synchronize()
+        check_output(prob.out, prob.lse, ref.out, ref.lse, f"one source, cuts {cuts}")
+        if len(parts) <= 5:
+            srcs = [tuple(torch.from_numpy(x).float().to(DEV) for x in (p[2], p[0], p[1])) for p in parts]
+            prob.merge(srcs)
+            torch.cuda.synchronize()
+            check_output(prob.out, prob.lse, ref.out, ref.lse, f"{len(srcs)} sources")
+
+
+# ---- the fused entry points ---------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("G", [1, 4])
+def test_decode_and_decode_host_match_partial_plus_merge(G):
+    w = wl(Hq=2 * G, Hkv=2)
+    ref = OracleRef(w)
+    prob = DeviceProblem(w, DEV)
+    host_dev = ref.host_partials_device(DEV)
+    prob.step(host_dev)
+    torch.cuda.synchronize()
+    want_out, want_lse = prob.out.clone(), prob.lse.clone()
+
+    nbytes = pkg.hg_attn_workspace_bytes(prob.desc, 2)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=DEV)
+    out = torch.empty_like(prob.out); lse = torch.empty_like(prob.lse)
+    pkg.hg_attn_decode(prob.q, prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end, host_dev,
+                       out, lse, ws, prob.desc)
+    torch.cuda.synchronize()
+    assert torch.equal(out, want_out) and torch.equal(lse, want_lse)
+
+    pin = lambda t: t.cpu().pin_memory()
+    host_pinned = [tuple(pin(x) for x in src) for src in host_dev]
+    out_h = torch.empty(prob.out.shape, dtype=torch.float32).pin_memory()
+    lse_h = torch.empty(prob.lse.shape, dtype=torch.float32).pin_memory()
+    pkg.hg_attn_decode_host(pin(prob.q), prob.kv["k"], prob.kv["v"], pin(prob.seq_lens), pin(prob.tok_begin),
+                            pin(prob.tok_end), host_pinned, out_h, lse_h, ws, prob.desc)
+    torch.cuda.synchronize()
+    assert torch.equal(out_h, want_out.cpu()) and torch.equal(lse_h, want_lse.cpu())
+    check_output(out_h, lse_h, ref.out, ref.lse)
+
+
+# ---- the read probe moves exactly the slice's bytes -------------------------------------------------------------
+
+@pytest.mark.parametrize("layout", ["HND", "NHD"])
+def test_read_probe_checksum_is_the_xor_of_the_slice(layout):
+    w = wl(layout=layout, seq_lens=[700, 333], tok_begin=[130, 5], tok_end=[700, 290])
+    prob = DeviceProblem(w, DEV)
+    sink = torch.zeros(w.B, w.Hkv, prob.NC, dtype=torch.int32, device=DEV)
+    pkg.hg_kv_read_probe(prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end, sink, prob.desc)
+    torch.cuda.synchronize()
+    got = sink.cpu().numpy().view(np.uint32)
+    for b in range(w.B):
+        for g in range(w.Hkv):
+            for c in range(prob.NC):
+                lo, hi = w.chunk_range(b, c)
+                want = np.uint32(0)
+                if hi > lo:
+                    for which in ("k", "v"):
+                        words = bits(w.kv_rows(which, b, g, lo, hi)).reshape(-1).view(np.uint32)
+                        want ^= np.bitwise_xor.reduce(words)
+                assert got[b, g, c] == want, (b, g, c)
+
+
+def test_bad_page_id_is_reported_not_dereferenced():
+    w = wl()
+    prob = DeviceProblem(w, DEV)
+    table = prob.kv["block_table"].clone()
+    page = w.tok_begin[0] // w.page_size + 3
+    table[0, page] = prob.kv["num_pages"] + 5          # out of range: the kernel must skip it and flag the call
+    prob.kv = dict(prob.kv, block_table=table)
+    prob.desc = prob.make_desc(w.chunk_tokens, prob.NC)
+    prob.partial()
+    torch.cuda.synchronize()
+    assert int(prob.status.item()) == hg.HG_DEV_BAD_PAGE
