@@ -182,6 +182,37 @@ hg_status hg_attn_decode_host(const void* q_host, const void* k_cache, const voi
                               size_t workspace_bytes, void* stream, const hg_attn_desc* desc);
 
 /*
+ * hg_attn_decode for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this entry point exists for the embedding environment, not for the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a CUDA-graph capture, in a
+ * plugin whose host gives it a fixed memory budget and forbids further allocation, or in a
+ * latency-critical decode loop that must not take the allocator's lock or trigger an implicit
+ * device synchronisation.  Such a caller has the inputs and the output buffers but nowhere to put
+ * the chunk partials that sit between the two kernels.
+ *
+ * Here those partials live in a fixed array inside the library's device image
+ * (HG_STATIC_SCRATCH_BYTES bytes, reserved on every GPU that loads the library for as long as the
+ * process lives).  Arguments and results are those of hg_attn_decode minus the workspace.
+ *
+ *   - Limit: batch * num_q_heads * num_chunks * (head_dim + 2) * 4 bytes (each of the three arrays
+ *     rounded up to 256 bytes) must fit in HG_STATIC_SCRATCH_BYTES; a larger problem is refused with
+ *     HG_ERR_WORKSPACE and nothing is launched.  Use bigger chunks or hg_attn_decode instead.
+ *   - The first call on each device looks up the array's device address (a symbol query, no
+ *     allocation) with that device current.  Make that first call outside any stream capture.
+ *   - Neither this call nor anything it calls uses cudaMalloc, cudaFree or an allocating library.
+ *   - All calls on a device share the one array and it keeps the previous call's contents.  Every
+ *     slot a call reads is first written by that call's own partial kernel, so nothing needs
+ *     clearing; but two calls whose kernels may overlap on the GPU (different streams, no
+ *     dependency between them) race on the array and give undefined results.  Serialise them.
+ */
+#define HG_STATIC_SCRATCH_BYTES (8u << 20)
+hg_status hg_attn_decode_static(const void* q, const void* k_cache, const void* v_cache, const int32_t* seq_lens,
+                                const int32_t* tok_begin, const int32_t* tok_end,
+                                const hg_partial_src* host_partials, int32_t n_host_src, float* out, float* lse,
+                                void* stream, const hg_attn_desc* desc);
+
+/*
  * Evidence kernel, not part of the attention path: streams the same K and V tiles through the
  * same TMA pipeline as hg_attn_partial and folds them into one 32-bit checksum per work item
  * (sink: dev uint32 [B][Hkv][NC]).  Used to measure the read ceiling of the paged access pattern.

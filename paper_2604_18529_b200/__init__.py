@@ -15,6 +15,7 @@ from .binding import (  # noqa: F401
     hg_attn_merge,
     hg_attn_decode,
     hg_attn_decode_host,
+    hg_attn_decode_static,
     hg_attn_workspace_bytes,
     hg_status_string,
     hg_kv_read_probe,

@@ -21,6 +21,7 @@ HG_OK, HG_ERR_INVALID_ARG, HG_ERR_UNSUPPORTED, HG_ERR_CUDA, HG_ERR_WORKSPACE = 0
 HG_DTYPE_F16, HG_DTYPE_BF16 = 0, 1
 HG_DEV_OK, HG_DEV_WAIT_TIMEOUT, HG_DEV_BAD_PAGE = 0, 1, 2
 HG_MAX_MERGE_SRC = 8
+HG_STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class HgError(RuntimeError):
@@ -80,6 +81,8 @@ def lib():
         L.hg_attn_decode.restype = C.c_int
         L.hg_attn_decode_host.argtypes = L.hg_attn_decode.argtypes
         L.hg_attn_decode_host.restype = C.c_int
+        L.hg_attn_decode_static.argtypes = [vp] * 6 + [C.POINTER(HgPartialSrc), i32, vp, vp, vp, C.POINTER(HgAttnDesc)]
+        L.hg_attn_decode_static.restype = C.c_int
         L.hg_kv_read_probe.argtypes = [vp] * 7 + [C.POINTER(HgAttnDesc)]
         L.hg_kv_read_probe.restype = C.c_int
         L.hg_status_string.argtypes = [C.c_int]
@@ -206,6 +209,22 @@ def hg_attn_decode(q, k_cache, v_cache, seq_lens, tok_begin, tok_end, host_parti
                               _dev(workspace, "workspace"), workspace.numel() * workspace.element_size(),
                               _stream(stream), C.byref(desc))
     _check(st, "hg_attn_decode")
+
+
+def hg_attn_decode_static(q, k_cache, v_cache, seq_lens, tok_begin, tok_end, host_partials, out, lse,
+                          desc: HgAttnDesc, stream=None) -> None:
+    """``hg_attn_decode`` for callers that may not allocate device memory (graph capture, fixed-budget
+    plugins, allocator-free decode loops): the chunk partials go to a fixed 8 MiB array inside the
+    library instead of a caller workspace.  Raises ``HgError`` (workspace) if the problem's partials do
+    not fit.  All calls on a device share that array, so calls that could overlap on the GPU must be
+    serialised; make the first call on a device outside any stream capture."""
+    arr = _src_array(host_partials, host=False)
+    st = lib().hg_attn_decode_static(_dev(q, "q"), _dev(k_cache, "k_cache"), _dev(v_cache, "v_cache"),
+                                     _dev(seq_lens, "seq_lens", torch.int32), _dev(tok_begin, "tok_begin", torch.int32),
+                                     _dev(tok_end, "tok_end", torch.int32), arr, len(host_partials),
+                                     _dev(out, "out", torch.float32), _dev(lse, "lse", torch.float32),
+                                     _stream(stream), C.byref(desc))
+    _check(st, "hg_attn_decode_static")
 
 
 def hg_attn_decode_host(q_host, k_cache, v_cache, seq_lens_host, tok_begin_host, tok_end_host, host_partials_host,

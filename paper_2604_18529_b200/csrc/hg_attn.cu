@@ -1,6 +1,7 @@
 // Host side of the C ABI declared in include/hybridgen_attn.h: argument validation, TMA tensor-map
 // encoding, launches.  No allocation, no synchronisation, no global mutable state (the cached
-// driver entry point and the per-kernel shared-memory opt-in are idempotent).
+// driver entry point, the per-kernel shared-memory opt-in and the per-device address of the static
+// scratch array are idempotent).
 #include "hybridgen_attn.h"
 
 #include <cuda.h>
@@ -8,6 +9,8 @@
 #include <math.h>
 #include <stdlib.h>
 #include <string.h>
+
+#include <atomic>
 
 #include "hg_merge.cuh"
 #include "hg_partial.cuh"
@@ -349,3 +352,38 @@ const char* hg_status_string(hg_status s) {
 uint32_t hg_version(void) { return HG_VERSION; }
 
 }  // extern "C"
+
+// ---- decode without any allocation: chunk partials in a fixed array of the device image ----------------
+
+// Scratch for hg_attn_decode_static.  In host code this name is only a handle for the symbol, not a
+// device address: the address is obtained once per device with cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char hg_static_scratch[HG_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+static std::atomic<void*> g_static_scratch_addr[kMaxDevices];
+
+// Device address of the scratch array on the current device (looked up on the first call per device).
+static void* static_scratch_ptr() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return nullptr; }
+    void* p = g_static_scratch_addr[dev].load(std::memory_order_acquire);
+    if (p) return p;
+    void* addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, hg_static_scratch) != cudaSuccess || !addr) { cudaGetLastError(); return nullptr; }
+    g_static_scratch_addr[dev].store(addr, std::memory_order_release);   // every thread would store the same value
+    return addr;
+}
+
+extern "C" hg_status hg_attn_decode_static(const void* q, const void* k_cache, const void* v_cache,
+                                           const int32_t* seq_lens, const int32_t* tok_begin, const int32_t* tok_end,
+                                           const hg_partial_src* host_partials, int32_t n_host_src, float* out,
+                                           float* lse, void* stream, const hg_attn_desc* desc) {
+    hg_status st = hg::check_desc(desc, true);
+    if (st != HG_OK) return st;
+    const hg::Workspace w = hg::plan_workspace(desc, 0, 0);
+    if (w.q > HG_STATIC_SCRATCH_BYTES) return HG_ERR_WORKSPACE;     // chunk partials exceed the fixed scratch
+    void* scratch = static_scratch_ptr();
+    if (!scratch) return HG_ERR_CUDA;
+    return hg_attn_decode(q, k_cache, v_cache, seq_lens, tok_begin, tok_end, host_partials, n_host_src, out, lse,
+                          scratch, HG_STATIC_SCRATCH_BYTES, stream, desc);
+}
