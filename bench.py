@@ -28,7 +28,10 @@ UNIT = "KV tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the partial kernel, from the ncu
 # captures summarised under profiles/ (None until a capture of that workload exists)
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # profiles/partial_kernel_opt13b.md: one sequence captured (402.77 MB read + 4.28 MB written), x 8 sequences
+    "opt13b": 8 * (402_771_456 + 4_281_600),
+}
 
 
 def measured_peak():
@@ -186,6 +189,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="opt13b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=0, help="keep only the first BATCH sequences (small profiling captures)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--probe", action="store_true", help="also time the read-probe kernel")
     args = ap.parse_args()
@@ -211,6 +215,8 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
     w = W.make_workload(args.workload)
+    if args.batch:
+        w = W.first_sequences(w, args.batch)
     prob = DeviceProblem(w, dev)
     # partials of the host-held slice: produced by the host in the real system; here synthetic values with
     # the statistics of a real partial (they are inputs of the merge, not results of this library)
@@ -317,7 +323,7 @@ def main():
             "metric": METRIC, "value": world * tokens / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": args.workload, "batch": w.B, "q_heads": w.Hq, "kv_heads": w.Hkv, "head_dim": w.D,
+            "config": {"workload": w.name, "batch": w.B, "q_heads": w.Hq, "kv_heads": w.Hkv, "head_dim": w.D,
                        "kv_dtype": w.dtype, "context": max(w.seq_lens), "gpu_tokens": tokens, "page_size": w.page_size,
                        "chunk_tokens": w.chunk_tokens, "kv_bytes_per_step": kv_bytes,
                        "l2": "inputs larger than L2" if kv_bytes > 2 * 126e6 else "inputs fit L2 (launch-bound case)",

@@ -163,7 +163,7 @@ static hg_status run_partial(int mode, const void* q, const void* k, const void*
     p.perm0 = perm[0]; p.perm1 = perm[1]; p.perm2 = perm[2];
     const float scale = d->scale > 0.f ? d->scale : 1.0f / sqrtf((float)d->head_dim);
     p.scale_log2 = scale * 1.4426950408889634f;
-    p.stages = env_int("HG_ATTN_STAGES", d->head_dim == 128 ? 4 : 8, 2, MAX_STAGES);
+    p.stages = env_int("HG_ATTN_STAGES", d->head_dim == 128 ? 3 : 6, 2, MAX_STAGES);   // 48 KB of stages: 4 CTAs per SM
     dim3 grid((unsigned)d->num_chunks, (unsigned)(d->num_kv_heads * p.head_blocks), (unsigned)d->batch);
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     const bool bf16 = d->dtype == HG_DTYPE_BF16;
