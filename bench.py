@@ -34,6 +34,22 @@ NCU_TRAFFIC_BYTES = {
 }
 
 
+def max_over_ranks(values, device="cpu"):
+    """Element-wise maximum of `values` over all ranks (identity when not running distributed)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_value(tokens_per_rank, world, ms_per_step):
+    """KV tokens/s of the whole job: every rank processes its own copy of the workload (weak scaling),
+    and the job is as slow as its slowest rank."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3)
+
+
 def measured_peak():
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
@@ -304,10 +320,7 @@ def main():
         torch.cuda.synchronize()
         probe_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in pe)
 
-    times = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms = times.tolist()
+    ms_total, e2e_ms = max_over_ranks([ms_total, e2e_ms], dev)
 
     if rank == 0:
         tokens = w.gpu_tokens
@@ -320,7 +333,7 @@ def main():
         part_avg = statistics.mean(part_ms)
         achieved = part_alg / (part_avg * 1e-3) / 1e9
         line = {
-            "metric": METRIC, "value": world * tokens / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+            "metric": METRIC, "value": whole_job_value(tokens, world, ms_step), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "batch": w.B, "q_heads": w.Hq, "kv_heads": w.Hkv, "head_dim": w.D,
@@ -336,7 +349,7 @@ def main():
                          "peak_kind": f"{peak_kind} copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
                          "frac_of_8000": achieved / 8000.0, "alg_bytes_per_launch": part_alg,
                          "traffic": NCU_TRAFFIC_BYTES.get(args.workload)},
-            "e2e": {"value": world * tokens / (e2e_ms / args.steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "e2e": {"value": whole_job_value(tokens, world, e2e_ms / args.steps), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps, "matches_device_path": bool(same),
                     "api": "hg_attn_decode_host (KV pools stay device resident: they are the GPU's slice of the cache)"},
             "gpu_launches": 2 * args.steps,
