@@ -58,9 +58,9 @@ typedef enum hg_dtype { HG_DTYPE_F16 = 0, HG_DTYPE_BF16 = 1 } hg_dtype;
 
 /* values the kernels may write to *hg_attn_desc.status (device word, optional) */
 #define HG_DEV_OK 0
-#define HG_DEV_WAIT_TIMEOUT 1 /* a bounded on-chip barrier wait ran out; results are invalid (m_part of
-                                 the affected items is NaN).  While the word holds this value the
-                                 kernels skip their work, so clear it before the next call. */
+#define HG_DEV_WAIT_TIMEOUT 1 /* a bounded on-chip barrier wait ran out; the call's results are invalid.
+                                 While the word holds this value the kernels skip their work, so clear
+                                 it before the next call. */
 #define HG_DEV_BAD_PAGE 2     /* a block-table entry of a resident page was outside [0, num_pages) */
 
 /*
@@ -75,7 +75,7 @@ typedef enum hg_dtype { HG_DTYPE_F16 = 0, HG_DTYPE_BF16 = 1 } hg_dtype;
  * including rows outside the slice, but such rows never influence a result.
  * Requirements: head_dim in {64, 128}; page_size in {16, 32, 64, 128, 256}; pool base addresses
  * 16-byte aligned; every stride a multiple of 8 elements; chunk_tokens a multiple of 64 and of
- * page_size, at most 65536.
+ * page_size, at most 512 pages.
  *
  * Chunk grid: chunks sit on absolute multiples of chunk_tokens.  Chunk c of sequence b covers
  *     [(tok_begin[b] / chunk_tokens + c) * chunk_tokens, + chunk_tokens)  intersected with
@@ -103,6 +103,10 @@ typedef struct hg_attn_desc {
     float scale;               /* logit scale; 0 means 1/sqrt(D) */
     uint32_t flags;            /* HG_FLAG_* */
     int32_t* status;           /* dev, optional: receives HG_DEV_* if a kernel detects a problem */
+    int32_t* sched_counter;    /* dev, optional, 4 bytes: when given, hg_attn_partial zeroes it on the stream and
+                                  its CTAs draw work items from it dynamically (better balance on ragged
+                                  batches); NULL: items are dealt round-robin.  Must not be shared by calls
+                                  that may overlap on the GPU.  Present when struct_size covers it. */
 } hg_attn_desc;
 
 /* One source of partials for hg_attn_merge (host struct, dev pointers). */

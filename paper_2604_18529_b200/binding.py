@@ -50,6 +50,7 @@ class HgAttnDesc(C.Structure):
         ("scale", C.c_float),
         ("flags", C.c_uint32),
         ("status", C.c_void_p),
+        ("sched_counter", C.c_void_p),
     ]
 
 
@@ -142,9 +143,10 @@ _DTYPES = {torch.float16: HG_DTYPE_F16, torch.bfloat16: HG_DTYPE_BF16, "f16": HG
 def attn_desc(*, batch: int, num_q_heads: int, num_kv_heads: int, head_dim: int, dtype, page_size: int,
               num_pages: int, page_stride: int, head_stride: int, tok_stride: int,
               block_table: Optional[torch.Tensor], max_pages: int, chunk_tokens: int, num_chunks: int,
-              scale: float = 0.0, status: Optional[torch.Tensor] = None, flags: int = 0) -> HgAttnDesc:
-    """Fill an ``hg_attn_desc``.  ``block_table`` (int32 CUDA [B][max_pages]) and ``status`` (int32 CUDA
-    scalar) are kept alive by the returned object."""
+              scale: float = 0.0, status: Optional[torch.Tensor] = None, flags: int = 0,
+              sched_counter: Optional[torch.Tensor] = None) -> HgAttnDesc:
+    """Fill an ``hg_attn_desc``.  ``block_table`` (int32 CUDA [B][max_pages]), ``status`` and
+    ``sched_counter`` (int32 CUDA scalars) are kept alive by the returned object."""
     d = HgAttnDesc()
     d.struct_size = C.sizeof(HgAttnDesc)
     d.batch, d.num_q_heads, d.num_kv_heads, d.head_dim = batch, num_q_heads, num_kv_heads, head_dim
@@ -155,7 +157,8 @@ def attn_desc(*, batch: int, num_q_heads: int, num_kv_heads: int, head_dim: int,
     d.max_pages, d.chunk_tokens, d.num_chunks = max_pages, chunk_tokens, num_chunks
     d.scale, d.flags = scale, flags
     d.status = _dev(status, "status", torch.int32)
-    d._keep = (block_table, status)
+    d.sched_counter = _dev(sched_counter, "sched_counter", torch.int32)
+    d._keep = (block_table, status, sched_counter)
     return d
 
 

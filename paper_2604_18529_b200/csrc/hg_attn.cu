@@ -7,6 +7,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <math.h>
+#include <stddef.h>
 #include <stdlib.h>
 #include <string.h>
 
@@ -21,6 +22,11 @@ namespace hg {
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// The optional trailing field, for callers compiled against a shorter struct.
+static int32_t* desc_sched(const hg_attn_desc* d) {
+    return d->struct_size >= sizeof(hg_attn_desc) ? d->sched_counter : nullptr;
+}
+
 static int ilog2_exact(int v) {
     for (int s = 0; s < 31; ++s)
         if ((1 << s) == v) return s;
@@ -29,7 +35,7 @@ static int ilog2_exact(int v) {
 
 // Checks the fields every entry point relies on.  `need_kv` also checks the KV addressing.
 static hg_status check_desc(const hg_attn_desc* d, bool need_kv) {
-    if (!d || d->struct_size < sizeof(hg_attn_desc)) return HG_ERR_INVALID_ARG;
+    if (!d || d->struct_size < offsetof(hg_attn_desc, sched_counter)) return HG_ERR_INVALID_ARG;
     if (d->batch < 1 || d->batch > 65535) return HG_ERR_INVALID_ARG;
     if (d->num_kv_heads < 1 || d->num_q_heads < 1 || d->num_q_heads % d->num_kv_heads) return HG_ERR_INVALID_ARG;
     if (d->head_dim <= 0 || d->head_dim % 8) return HG_ERR_INVALID_ARG;
@@ -46,6 +52,7 @@ static hg_status check_desc(const hg_attn_desc* d, bool need_kv) {
     if (d->chunk_tokens % TILE_T || d->chunk_tokens % d->page_size || d->chunk_tokens > 65536)
         return HG_ERR_UNSUPPORTED;
     if (d->chunk_tokens / d->page_size > MAX_CHUNK_PAGES) return HG_ERR_UNSUPPORTED;
+    if (desc_sched(d) && (reinterpret_cast<uintptr_t>(desc_sched(d)) & 3u)) return HG_ERR_INVALID_ARG;
     if ((int64_t)d->num_kv_heads * ((d->num_q_heads / d->num_kv_heads + 7) / 8) > 65535) return HG_ERR_UNSUPPORTED;
     if (!d->block_table && (int64_t)d->batch * d->max_pages > d->num_pages) return HG_ERR_INVALID_ARG;
     return HG_OK;
@@ -69,35 +76,28 @@ static EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// Pool viewed as a 4-D tensor {d, x, y, z} where x, y, z are token-in-page, head and page ordered by
-// ascending stride; one box is 64 d-elements (128 bytes, swizzled) x `rows` tokens.
-static hg_status make_maps(const hg_attn_desc* d, const void* k, const void* v, CUtensorMap* tk, CUtensorMap* tv,
-                           int perm[3]) {
+// Pool viewed as a 5-D tensor {d within a 64-element half, token in page, half, head, page}; one box is a
+// whole page of one head: [half][rows][64 elements = 128 bytes, swizzled].  The half dimension sits
+// behind the token dimension (its stride, 128 bytes, is the smaller one) so that the box lands in
+// shared memory as two 128-byte-wide column blocks, the layout ldmatrix reads without bank conflicts.
+static hg_status make_maps(const hg_attn_desc* d, const void* k, const void* v, CUtensorMap* tk, CUtensorMap* tv) {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return HG_ERR_CUDA;
     const int rows = d->page_size >= TILE_T ? TILE_T : d->page_size;
-    int64_t stride[3] = {d->tok_stride, d->head_stride, d->page_stride};
-    int64_t extent[3] = {d->page_size, d->num_kv_heads, d->num_pages};
-    int order[3] = {0, 1, 2};
-    for (int i = 0; i < 3; ++i)                       // insertion sort, stable
-        for (int j = i; j > 0 && stride[order[j]] < stride[order[j - 1]]; --j) {
-            int t = order[j]; order[j] = order[j - 1]; order[j - 1] = t;
-        }
-    cuuint64_t dims[4] = {(cuuint64_t)d->head_dim, 0, 0, 0};
-    cuuint64_t strides[3];
-    cuuint32_t box[4] = {64, 1, 1, 1};
-    cuuint32_t estr[4] = {1, 1, 1, 1};
-    for (int i = 0; i < 3; ++i) {
-        dims[1 + i] = (cuuint64_t)extent[order[i]];
-        strides[i] = (cuuint64_t)stride[order[i]] * 2u;
-        if (order[i] == 0) box[1 + i] = (cuuint32_t)rows;
-        perm[i] = order[i];
-    }
+    const int halves = d->head_dim / 64;
+    cuuint64_t dims[5] = {64, (cuuint64_t)d->page_size, (cuuint64_t)halves, (cuuint64_t)d->num_kv_heads,
+                          (cuuint64_t)d->num_pages};
+    cuuint64_t strides[4] = {(cuuint64_t)d->tok_stride * 2u, 128u, (cuuint64_t)d->head_stride * 2u,
+                             (cuuint64_t)d->page_stride * 2u};
+    if (d->num_kv_heads == 1) strides[2] = strides[0];     // unused dimensions still need a legal stride
+    if (d->num_pages == 1) strides[3] = strides[0];
+    cuuint32_t box[5] = {64, (cuuint32_t)rows, (cuuint32_t)halves, 1, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     const CUtensorMapDataType dt = d->dtype == HG_DTYPE_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
     const void* base[2] = {k, v};
     CUtensorMap* out[2] = {tk, tv};
     for (int i = 0; i < 2; ++i) {
-        CUresult r = enc(out[i], dt, 4, const_cast<void*>(base[i]), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+        CUresult r = enc(out[i], dt, 5, const_cast<void*>(base[i]), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return HG_ERR_UNSUPPORTED;   // a stride pattern the TMA unit cannot express
     }
@@ -114,13 +114,27 @@ static int env_int(const char* name, int dflt, int lo, int hi) {
 }
 
 template <int D, bool BF16, int MODE>
-static hg_status launch_partial_t(const CUtensorMap& tk, const CUtensorMap& tv, const PartialParams& p, dim3 grid,
-                                  cudaStream_t st) {
-    const size_t smem = (size_t)p.stages * (D / 64) * HALF_BYTES + 1024;
+static hg_status launch_partial_t(const CUtensorMap& tk, const CUtensorMap& tv, PartialParams p, cudaStream_t st) {
+    const size_t smem = (size_t)p.stages * 2 * TILE_T * D * 2 + 1024;     // K + V tile per stage
     auto kern = partial_kernel<D, BF16, MODE>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
         cudaGetLastError();
         return HG_ERR_CUDA;
+    }
+    const int Y = p.Hkv * p.head_blocks;
+    dim3 grid((unsigned)p.NC, (unsigned)Y, (unsigned)p.B);
+    if (p.persistent) {
+        // one wave of resident CTAs; each takes items round-robin
+        int dev = 0, sms = 0, per_sm = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, THREADS, smem) != cudaSuccess || per_sm < 1) {
+            cudaGetLastError();
+            return HG_ERR_CUDA;
+        }
+        per_sm = env_int("HG_ATTN_CTAS_PER_SM", per_sm, 1, per_sm);
+        const long long slots = (long long)p.NC * Y * p.B;
+        const long long resident = (long long)sms * per_sm;
+        grid = dim3((unsigned)(slots < resident ? slots : resident), 1, 1);
     }
     kern<<<grid, THREADS, smem, st>>>(tk, tv, p);
     return cudaGetLastError() == cudaSuccess ? HG_OK : HG_ERR_CUDA;
@@ -128,9 +142,9 @@ static hg_status launch_partial_t(const CUtensorMap& tk, const CUtensorMap& tv, 
 
 template <int MODE>
 static hg_status launch_partial_m(int D, bool bf16, const CUtensorMap& tk, const CUtensorMap& tv, const PartialParams& p,
-                                  dim3 grid, cudaStream_t st) {
-    if (D == 128) return bf16 ? launch_partial_t<128, true, MODE>(tk, tv, p, grid, st) : launch_partial_t<128, false, MODE>(tk, tv, p, grid, st);
-    return bf16 ? launch_partial_t<64, true, MODE>(tk, tv, p, grid, st) : launch_partial_t<64, false, MODE>(tk, tv, p, grid, st);
+                                  cudaStream_t st) {
+    if (D == 128) return bf16 ? launch_partial_t<128, true, MODE>(tk, tv, p, st) : launch_partial_t<128, false, MODE>(tk, tv, p, st);
+    return bf16 ? launch_partial_t<64, true, MODE>(tk, tv, p, st) : launch_partial_t<64, false, MODE>(tk, tv, p, st);
 }
 
 static hg_status run_partial(int mode, const void* q, const void* k, const void* v, const int32_t* seq_lens,
@@ -149,8 +163,7 @@ static hg_status run_partial(int mode, const void* q, const void* k, const void*
     PartialParams p;
     memset(&p, 0, sizeof p);
     CUtensorMap tk, tv;
-    int perm[3];
-    st = make_maps(d, k, v, &tk, &tv, perm);
+    st = make_maps(d, k, v, &tk, &tv);
     if (st != HG_OK) return st;
     const int G = d->num_q_heads / d->num_kv_heads;
     if (mode != MODE_PROBE) mode = (G == 1) ? MODE_MHA : MODE_GQA;
@@ -160,17 +173,23 @@ static hg_status run_partial(int mode, const void* q, const void* k, const void*
     p.page_size = d->page_size; p.page_shift = ilog2_exact(d->page_size); p.max_pages = d->max_pages;
     p.num_pages = d->num_pages; p.C = d->chunk_tokens; p.NC = d->num_chunks;
     p.head_blocks = (mode == MODE_GQA) ? (G + 7) / 8 : 1;
-    p.perm0 = perm[0]; p.perm1 = perm[1]; p.perm2 = perm[2];
     const float scale = d->scale > 0.f ? d->scale : 1.0f / sqrtf((float)d->head_dim);
     p.scale_log2 = scale * 1.4426950408889634f;
-    p.stages = env_int("HG_ATTN_STAGES", d->head_dim == 128 ? 3 : 6, 2, MAX_STAGES);   // 48 KB of stages: 4 CTAs per SM
-    dim3 grid((unsigned)d->num_chunks, (unsigned)(d->num_kv_heads * p.head_blocks), (unsigned)d->batch);
+    p.stages = env_int("HG_ATTN_STAGES", d->head_dim == 128 ? 3 : 6, 2, MAX_STAGES);   // 96 KB of ring: 2 CTAs per SM
+    // persistent schedule unless the batch or the chunk's page list exceeds what the kernel keeps in shared memory
+    p.persistent = (d->batch <= PERSIST_MAX_BATCH && d->chunk_tokens / d->page_size <= PERSIST_CHUNK_PAGES)
+                       ? env_int("HG_ATTN_PERSISTENT", 1, 0, 1) : 0;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    p.sched = p.persistent && env_int("HG_ATTN_DYNAMIC", 1, 0, 1) ? desc_sched(d) : nullptr;
+    if (p.sched && cudaMemsetAsync(p.sched, 0, sizeof(int32_t), cs) != cudaSuccess) {
+        cudaGetLastError();
+        return HG_ERR_CUDA;
+    }
     const bool bf16 = d->dtype == HG_DTYPE_BF16;
     switch (mode) {
-        case MODE_MHA: return launch_partial_m<MODE_MHA>(d->head_dim, bf16, tk, tv, p, grid, cs);
-        case MODE_GQA: return launch_partial_m<MODE_GQA>(d->head_dim, bf16, tk, tv, p, grid, cs);
-        default: return launch_partial_m<MODE_PROBE>(d->head_dim, bf16, tk, tv, p, grid, cs);
+        case MODE_MHA: return launch_partial_m<MODE_MHA>(d->head_dim, bf16, tk, tv, p, cs);
+        case MODE_GQA: return launch_partial_m<MODE_GQA>(d->head_dim, bf16, tk, tv, p, cs);
+        default: return launch_partial_m<MODE_PROBE>(d->head_dim, bf16, tk, tv, p, cs);
     }
 }
 
@@ -211,6 +230,7 @@ static size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct Workspace {
     size_t o_part, m_part, l_part;           // chunk partials
+    size_t sched;                            // work counter of the partial kernel
     size_t q, seq_lens, tok_begin, tok_end;  // staging (host form only)
     size_t host_part;                        // staged host partials, n_host_partials * (D + 2) floats per row + slack
     size_t out, lse;
@@ -224,6 +244,7 @@ static Workspace plan_workspace(const hg_attn_desc* d, int n_host_partials, int 
     w.o_part = off; off += up256(rows * d->num_chunks * d->head_dim * sizeof(float));
     w.m_part = off; off += up256(rows * d->num_chunks * sizeof(float));
     w.l_part = off; off += up256(rows * d->num_chunks * sizeof(float));
+    w.sched = off; off += 256;
     w.q = off; off += up256(rows * d->head_dim * 2);
     w.seq_lens = off; off += up256((size_t)d->batch * 4);
     w.tok_begin = off; off += up256((size_t)d->batch * 4);
@@ -278,7 +299,12 @@ hg_status hg_attn_decode(const void* q, const void* k_cache, const void* v_cache
     float* o_part = reinterpret_cast<float*>(ws + w.o_part);
     float* m_part = reinterpret_cast<float*>(ws + w.m_part);
     float* l_part = reinterpret_cast<float*>(ws + w.l_part);
-    st = run_partial(MODE_MHA, q, k_cache, v_cache, seq_lens, tok_begin, tok_end, o_part, m_part, l_part, nullptr, stream, desc);
+    hg_attn_desc dd;
+    memset(&dd, 0, sizeof dd);
+    memcpy(&dd, desc, desc->struct_size < sizeof dd ? desc->struct_size : sizeof dd);
+    dd.struct_size = sizeof dd;
+    dd.sched_counter = reinterpret_cast<int32_t*>(ws + w.sched);       // the workspace provides the work counter
+    st = run_partial(MODE_MHA, q, k_cache, v_cache, seq_lens, tok_begin, tok_end, o_part, m_part, l_part, nullptr, stream, &dd);
     if (st != HG_OK) return st;
     hg_partial_src src[HG_MAX_MERGE_SRC];
     src[0].o = o_part; src[0].m = m_part; src[0].l = l_part; src[0].nc = desc->num_chunks; src[0].reserved = 0;

@@ -82,15 +82,15 @@ __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* tm) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tm)) : "memory");
 }
 
-// One tiled 4-D tensor load, global -> this CTA's shared memory, completion counted in bytes on `bar`.
-// c0 (innermost coordinate, 16-bit elements) must be a multiple of 8: every call site passes 0 or 64.
-__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* tm, uint64_t* bar, int c0, int c1, int c2,
-                                            int c3, uint64_t policy) {
+// One tiled 5-D tensor load, global -> this CTA's shared memory, completion counted in bytes on `bar`.
+// c0 (innermost coordinate, 16-bit elements) must be a multiple of 8: every call site passes 0.
+__device__ __forceinline__ void tma_load_5d(void* dst, const CUtensorMap* tm, uint64_t* bar, int c0, int c1, int c2,
+                                            int c3, int c4, uint64_t policy) {
     asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
-        " [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
+        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%3, %4, %5, %6, %7}], [%2], %8;"
         ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(tm)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2),
-          "r"(c3), "l"(policy)
+          "r"(c3), "r"(c4), "l"(policy)
         : "memory");
 }
 

@@ -1,11 +1,15 @@
 // Split-KV decode attention partials over a paged 16-bit KV pool (sm_100a).
 //
-// One CTA per work item (sequence b, KV head g [, block of 8 query heads], chunk c).  A producer
-// warp streams the item's K and V tiles (64 tokens x D, 128-byte-swizzled) from HBM into a ring of
-// shared-memory stages with TMA tensor loads; four consumer warps each own 16 token rows of every
-// tile and keep a private online-softmax state (running max, exp-sum, un-normalised output), which
-// is merged across warps once at the end.  K_j and V_j alternate in the ring, so the logits never
-// leave the chip.
+// A work item is (sequence b, KV head g [, block of 8 query heads], chunk c).  Persistent CTAs take
+// items from the list of non-empty items, dynamically through a global counter when the caller
+// provides one, else round-robin; the producer warp is the only scheduler, and every filled stage
+// carries a descriptor telling the consumers what it holds.  Within a CTA the producer streams, per
+// 64-token step, the K tile and the V tile of the item (64 x D each) from HBM into one stage of a
+// shared-memory ring with TMA tensor loads - one 5-D box per (page, tensor), 128-byte swizzled - and
+// runs ahead across item boundaries, so the ring never drains between items.  Four consumer warps
+// each own 16 token rows of every tile and keep a private online-softmax state (running max,
+// exp-sum, un-normalised output); the states are merged once per item, using the item's last stage
+// as scratch before it is handed back to the producer.  The logits never leave the chip.
 //
 //   MODE_MHA    one query head per KV head: dot products on CUDA cores, fp32 throughout.
 //   MODE_GQA    up to 8 query heads share the KV head: S^T = K q^T and O^T = V^T P^T on warp-level
@@ -13,6 +17,14 @@
 //               for a group of 8).  P is fed as hi + lo 16-bit terms, so its rounding error is ~2^-17
 //               (bf16) / ~2^-22 (fp16) instead of one 16-bit ulp.
 //   MODE_PROBE  same loads, no attention math: folds the slice's bytes into a checksum.
+//
+// With p.persistent == 0 the grid is (NC, Hkv * head_blocks, B) and every CTA handles the one item
+// its block index names (used for batches or chunks too large for the in-kernel item scan).
+//
+// Why the stage is a K+V pair and the box a whole page: issuing one TMA tensor load costs the
+// producer ~250 cycles plus ~50 per further lane of the same instruction, and every mbarrier
+// hand-shake costs another few hundred; at ~50 GB/s per SM that only works if each producer
+// iteration moves tens of KB.
 #pragma once
 
 #include "hg_device.cuh"
@@ -23,9 +35,10 @@ constexpr int TILE_T = 64;             // tokens per tile
 constexpr int CONSUMER_WARPS = 4;
 constexpr int CONSUMER_THREADS = CONSUMER_WARPS * 32;
 constexpr int THREADS = CONSUMER_THREADS + 32;
-constexpr int MAX_STAGES = 12;
-constexpr int MAX_CHUNK_PAGES = 1024;
-constexpr int HALF_BYTES = TILE_T * 128;  // one 64-element (128-byte) column half of a tile
+constexpr int MAX_STAGES = 8;
+constexpr int MAX_CHUNK_PAGES = 512;       // chunk_tokens / page_size, any schedule
+constexpr int PERSIST_CHUNK_PAGES = 256;   // ... for the persistent schedule (page ids are double-buffered)
+constexpr int PERSIST_MAX_BATCH = 512;     // sequences the in-kernel item scan handles
 
 enum { MODE_MHA = 0, MODE_GQA = 1, MODE_PROBE = 2 };
 
@@ -43,21 +56,32 @@ struct PartialParams {
     int B, Hq, Hkv, G;
     int page_size, page_shift, max_pages, num_pages;
     int C, NC, stages, head_blocks;
-    int perm0, perm1, perm2;  // tensor-map dim 1+i carries logical coordinate perm_i: 0 = token-in-page, 1 = head, 2 = page
+    int persistent;
+    int32_t* sched;           // zeroed work counter: items are handed out dynamically (NULL: round-robin)
     float scale_log2;         // logit scale * log2(e)
 };
 
 struct Control {
     uint64_t full[MAX_STAGES];
     uint64_t empty[MAX_STAGES];
+    uint64_t cbar;                       // barrier among the consumer warps (one arrival per warp)
+    int2 sdesc[MAX_STAGES];              // what a filled stage holds: x = item index (-1: no more work), y = tile in item
     int abort_flag;
-    uint32_t probe_acc;
-    int pages[MAX_CHUNK_PAGES];
+    int pages[MAX_CHUNK_PAGES];          // persistent schedule: two buffers, at 0 and at MAX_CHUNK_PAGES / 2
     float red_m[32];
     float red_l[32];
+    int cum[PERSIST_MAX_BATCH + 1];      // cum[b] = number of items of sequences < b
+    int tb[PERSIST_MAX_BATCH];           // clamped slice of every sequence
+    int te[PERSIST_MAX_BATCH];
 };
+static_assert(PERSIST_CHUNK_PAGES <= MAX_CHUNK_PAGES / 2, "page-id double buffer");
 
-__device__ __forceinline__ int pick3(int k, int a, int b, int c) { return k == 0 ? a : (k == 1 ? b : c); }
+// One work item, decoded identically by the producer and by every consumer warp.
+struct Item {
+    int b, y, c;        // sequence, KV head * head_blocks + head block, chunk slot
+    int lo, hi;         // token range
+    int tile0, ntiles;  // 64-token tiles covering it
+};
 
 // All lanes wait; the verdict is made warp-uniform so that no lane leaves a loop alone.
 __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
@@ -65,14 +89,50 @@ __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volati
     return __all_sync(0xffffffffu, ok);
 }
 
+// Clamped slice [tb, te) of sequence b and its number of chunk slots in use.
+__device__ __forceinline__ int seq_chunks(const PartialParams& p, int b, int& tb, int& te) {
+    tb = max(p.tok_begin[b], 0);
+    te = min(p.tok_end[b], p.seq_lens[b]);
+    if (te <= tb) return 0;
+    return min((te + p.C - 1) / p.C - tb / p.C, p.NC);
+}
+
+__device__ __forceinline__ void set_range(const PartialParams& p, Item& it, int tb, int te) {
+    const int first = tb / p.C;
+    it.lo = max((first + it.c) * p.C, tb);
+    it.hi = min((first + it.c + 1) * p.C, te);
+    it.tile0 = it.lo / TILE_T;
+    it.ntiles = it.hi > it.lo ? (it.hi + TILE_T - 1) / TILE_T - it.tile0 : 0;
+}
+
+// Item i of the persistent schedule: items are ordered by (b, y, c); everything it needs is in shared memory.
+__device__ __forceinline__ Item decode_item(const PartialParams& p, const Control& ctl, int i) {
+    int lo = 0, hi = p.B;                 // largest b with cum[b] <= i
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (ctl.cum[mid] <= i) lo = mid; else hi = mid;
+    }
+    Item it;
+    it.b = lo;
+    const int tb = ctl.tb[lo], te = ctl.te[lo];
+    const int nc = max(te > tb ? min((te + p.C - 1) / p.C - tb / p.C, p.NC) : 0, 1);
+    const int r = i - ctl.cum[lo];
+    it.y = r / nc;
+    it.c = r - it.y * nc;
+    set_range(p, it, tb, te);
+    return it;
+}
+
 template <int D, bool BF16, int MODE>
 __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant__ CUtensorMap tmK,
                                                           const __grid_constant__ CUtensorMap tmV,
                                                           const PartialParams p) {
     constexpr int HALVES = D / 64;
-    constexpr int STAGE_BYTES = HALVES * HALF_BYTES;
+    constexpr int TILE_BYTES = TILE_T * D * 2;
+    constexpr int STAGE_BYTES = 2 * TILE_BYTES;   // K tile, then V tile
     constexpr int NV = 8 * HALVES;     // MHA: d-components owned by a lane
     constexpr int KSTEPS = D / 16;     // GQA: 16-wide steps along d
+    constexpr float LN2 = 0.6931471805599453f;
     const float NEG_INF = __int_as_float(0xff800000);
 
     extern __shared__ uint8_t smem_raw[];
@@ -84,408 +144,580 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
     cudaTriggerProgrammaticLaunchCompletion();   // a dependent merge launch may be scheduled while this grid drains
 #endif
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int c = blockIdx.x;
-    const int g = blockIdx.y / p.head_blocks, hb = blockIdx.y % p.head_blocks;
-    const int b = blockIdx.z;
-
-    // ---- the item's token range --------------------------------------------------------------
-    const int L = p.seq_lens[b];
-    const int tb = max(p.tok_begin[b], 0);
-    const int te = min(p.tok_end[b], L);
-    const int first = tb / p.C;
-    const int lo = max((first + c) * p.C, tb);
-    const int hi = min((first + c + 1) * p.C, te);
-
-    const int nheads = (MODE == MODE_GQA) ? min(8, p.G - hb * 8) : 1;
-    const int h0 = (MODE == MODE_GQA) ? g * p.G + hb * 8 : g;   // first query head of this item
-
-    if (te <= tb || lo >= hi) {            // empty chunk slot: neutral element
-        if constexpr (MODE == MODE_PROBE) {
-            if (tid == 0) p.sink[((size_t)b * p.Hkv + g) * p.NC + c] = 0u;
-        } else {
-            for (int i = tid; i < nheads * D; i += THREADS)
-                p.o_part[(((size_t)b * p.Hq + h0 + i / D) * p.NC + c) * D + i % D] = 0.f;
-            if (tid < nheads) {
-                p.m_part[((size_t)b * p.Hq + h0 + tid) * p.NC + c] = NEG_INF;
-                p.l_part[((size_t)b * p.Hq + h0 + tid) * p.NC + c] = 0.f;
-            }
-        }
-        return;
-    }
+    const int Y = p.Hkv * p.head_blocks;
 
     // a wait already timed out in this call (or the caller left the word set): do not queue behind it
-    if (p.status && *reinterpret_cast<volatile int32_t*>(p.status) == HG_DEV_WAIT_TIMEOUT) {
-        if constexpr (MODE != MODE_PROBE) {
-            if (tid < nheads) p.m_part[((size_t)b * p.Hq + h0 + tid) * p.NC + c] = __int_as_float(0x7fc00000);
-        }
-        return;
-    }
+    if (p.status && *reinterpret_cast<volatile int32_t*>(p.status) == HG_DEV_WAIT_TIMEOUT) return;
 
-    const int tile0 = lo / TILE_T;
-    const int ntiles = (hi + TILE_T - 1) / TILE_T - tile0;
-    const int page0 = (tile0 * TILE_T) >> p.page_shift;
-    const int npages = (((tile0 + ntiles) * TILE_T - 1) >> p.page_shift) + 1 - page0;
-    const int n_iter = 2 * ntiles;   // K_0, V_0, K_1, V_1, ...
-
-    // ---- set-up: barriers and the physical page ids of this chunk -------------------------------
+    // ---- set-up: barriers, and for the persistent schedule the item counts per sequence ---------------
     if (tid == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(&ctl.full[s], 1);
             mbar_init(&ctl.empty[s], CONSUMER_WARPS);
         }
+        mbar_init(&ctl.cbar, CONSUMER_WARPS);
         ctl.abort_flag = 0;
-        ctl.probe_acc = 0u;
         fence_barrier_init();
     }
-    for (int i = tid; i < npages && i < MAX_CHUNK_PAGES; i += THREADS) {
-        const int pg = page0 + i;
-        int phys = -1;
-        if (pg * p.page_size < hi && (pg + 1) * p.page_size > lo) {
-            if (pg < p.max_pages)
-                phys = p.block_table ? p.block_table[(size_t)b * p.max_pages + pg] : b * p.max_pages + pg;
-            if (phys < 0 || phys >= p.num_pages) {
-                if (p.status) atomicMax(p.status, HG_DEV_BAD_PAGE);
-                phys = -1;
+    int n_items = 1, item_step = 1, item_first = 0;
+    if (p.persistent) {
+        // cum[b+1] = sum_{b' <= b} nc_b' * Y : one warp, each lane a contiguous block of sequences
+        if (warp == 0) {
+            const int per = (p.B + 31) / 32;
+            const int b0 = min(p.B, lane * per), b1 = min(p.B, b0 + per);
+            int sum = 0;
+            for (int b = b0; b < b1; ++b) { int tb, te; sum += seq_chunks(p, b, tb, te) * Y; }
+            int incl = sum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            int run = incl - sum;
+            if (lane == 0) ctl.cum[0] = 0;
+            for (int b = b0; b < b1; ++b) {
+                int tb, te;
+                run += seq_chunks(p, b, tb, te) * Y;
+                ctl.cum[b + 1] = run; ctl.tb[b] = tb; ctl.te[b] = te;
             }
         }
-        ctl.pages[i] = phys;
+        __syncthreads();
+        n_items = ctl.cum[p.B];
+        // use only as many CTAs as keeps every CTA's item count equal (+-1); the others only help with the
+        // empty slots below
+        const int rounds = (n_items + (int)gridDim.x - 1) / (int)gridDim.x;
+        item_step = rounds > 0 ? (n_items + rounds - 1) / rounds : 1;
+        item_first = blockIdx.x;
+
+        // empty chunk slots (c >= nc_b): neutral elements, spread over all CTAs
+        for (int s = blockIdx.x; s < p.B * Y; s += gridDim.x) {
+            const int b = s / Y, y = s - b * Y;
+            int tb, te;
+            const int nc = seq_chunks(p, b, tb, te);
+            const int ne = p.NC - nc;                 // empty slots per head
+            if (ne <= 0) continue;
+            if constexpr (MODE == MODE_PROBE) {
+                for (int i = tid; i < ne; i += THREADS) p.sink[((size_t)b * p.Hkv + y) * p.NC + nc + i] = 0u;
+            } else {
+                const int hb = y % p.head_blocks, g = y / p.head_blocks;
+                const int nh = (MODE == MODE_GQA) ? min(8, p.G - hb * 8) : 1;
+                const int hq0 = (MODE == MODE_GQA) ? g * p.G + hb * 8 : g;
+                for (int i = tid; i < nh * ne * D; i += THREADS) {
+                    const int sl = i / D, hh = sl / ne, cc = nc + sl % ne;
+                    p.o_part[(((size_t)b * p.Hq + hq0 + hh) * p.NC + cc) * D + i % D] = 0.f;
+                }
+                for (int i = tid; i < nh * ne; i += THREADS) {
+                    const int hh = i / ne, cc = nc + i % ne;
+                    p.m_part[((size_t)b * p.Hq + hq0 + hh) * p.NC + cc] = NEG_INF;
+                    p.l_part[((size_t)b * p.Hq + hq0 + hh) * p.NC + cc] = 0.f;
+                }
+            }
+        }
+        if (n_items == 0 || (!p.sched && (int)blockIdx.x >= item_step)) return;
+    } else {
+        __syncthreads();
     }
-    __syncthreads();
 
     volatile int* abort_flag = &ctl.abort_flag;
+    auto get_item = [&](int i) -> Item {
+        if (p.persistent) return decode_item(p, ctl, i);
+        Item it;
+        it.b = blockIdx.z; it.y = blockIdx.y; it.c = blockIdx.x;
+        int tb, te;
+        seq_chunks(p, it.b, tb, te);
+        if (te <= tb) { it.lo = it.hi = it.tile0 = it.ntiles = 0; } else set_range(p, it, tb, te);
+        return it;
+    };
 
-    // consumer state (only the active mode's survives compilation); parked in shared memory after the loop
-    float mha_m = NEG_INF, mha_l = 0.f, mha_o[NV];
-    float gqa_m[2] = {NEG_INF, NEG_INF}, gqa_l[2] = {0.f, 0.f}, gqa_o[KSTEPS][4];
-    uint32_t probe_x = 0u;
-#pragma unroll
-    for (int i = 0; i < NV; ++i) mha_o[i] = 0.f;
-#pragma unroll
-    for (int i = 0; i < KSTEPS; ++i) { gqa_o[i][0] = gqa_o[i][1] = gqa_o[i][2] = gqa_o[i][3] = 0.f; }
+    if (!p.persistent) {
+        // this CTA's only item may be an empty chunk slot: neutral element, nothing to stream
+        const Item it = get_item(0);
+        if (it.ntiles == 0) {
+            if constexpr (MODE == MODE_PROBE) {
+                if (tid == 0) p.sink[((size_t)it.b * p.Hkv + it.y) * p.NC + it.c] = 0u;
+            } else {
+                const int hb = it.y % p.head_blocks, g = it.y / p.head_blocks;
+                const int nh = (MODE == MODE_GQA) ? min(8, p.G - hb * 8) : 1;
+                const int hq0 = (MODE == MODE_GQA) ? g * p.G + hb * 8 : g;
+                for (int i = tid; i < nh * D; i += THREADS)
+                    p.o_part[(((size_t)it.b * p.Hq + hq0 + i / D) * p.NC + it.c) * D + i % D] = 0.f;
+                if (tid < nh) {
+                    p.m_part[((size_t)it.b * p.Hq + hq0 + tid) * p.NC + it.c] = NEG_INF;
+                    p.l_part[((size_t)it.b * p.Hq + hq0 + tid) * p.NC + it.c] = 0.f;
+                }
+            }
+            return;
+        }
+    }
+
+    // ---- tile geometry in shared memory ---------------------------------------------------------------
+    // A tile is 64/R boxes of R token rows (R = min(page_size, 64)); a box is [half][row][128 bytes], the
+    // 16-byte chunks of a row XOR-swizzled with (row & 7).
+    const int rshift = min(p.page_shift, 6);
+    const int R = 1 << rshift;
+    const uint32_t half_stride = 128u << rshift;
+    const uint32_t box_bytes = (uint32_t)(HALVES * 128) << rshift;
+    auto row_off = [&](int r) -> uint32_t { return (uint32_t)(r >> rshift) * box_bytes + (uint32_t)(r & (R - 1)) * 128u; };
 
     const int row0 = warp * 16;                  // a consumer warp's rows within every tile
     const int gi = lane >> 3, li = lane & 7;     // MHA: 8 lanes share a token row; 4 row groups per warp
     const int quad = lane >> 2, tq = lane & 3;   // GQA: MMA fragment coordinates
 
     if (warp == CONSUMER_WARPS) {
-        // ======================= producer warp =======================
+        // =============================== producer warp ===============================
         prefetch_tensormap(&tmK);
         prefetch_tensormap(&tmV);
         const uint64_t policy = l2_evict_first_policy();
-        const int rows = p.page_size >= TILE_T ? TILE_T : p.page_size;
-        const int nbox = p.page_size >= TILE_T ? 1 : (TILE_T >> p.page_shift);
-        const int j = lane / HALVES, h = lane % HALVES;
-        int issued = 0;
-        for (int it = 0; it < n_iter; ++it) {
-            const int s = it % p.stages;
-            const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
+        const int nbox = TILE_T >> rshift;           // boxes per tile: 4, 2 or 1
+        const int j = lane & (nbox - 1);             // this lane's box
+        const int isv = lane >> (6 - rshift);        // 0: K tile, 1: V tile (lanes >= 2 * nbox idle)
+        constexpr int PER_LANE = PERSIST_CHUNK_PAGES / 32;
+        const bool dynamic = p.persistent && p.sched != nullptr;
+
+        // block-table entry of logical page pg of the item's sequence if the page overlaps [lo, hi), else -2
+        // (the value is only loaded here; check_page() validates it once it is needed)
+        auto lookup = [&](const Item& it, int pg) -> int {
+            if (pg * p.page_size < it.hi && (pg + 1) * p.page_size > it.lo && pg < p.max_pages)
+                return p.block_table ? __ldg(p.block_table + (size_t)it.b * p.max_pages + pg) : it.b * p.max_pages + pg;
+            return -2;                                   // no token of the item on this page
+        };
+        auto check_page = [&](int phys) -> int {
+            if (phys == -2) return -1;
+            if (phys < 0 || phys >= p.num_pages) {
+                if (p.status) atomicMax(p.status, HG_DEV_BAD_PAGE);
+                return -1;
+            }
+            return phys;
+        };
+        auto first_page = [&](const Item& it) { return (it.tile0 * TILE_T) >> p.page_shift; };
+        auto num_pages_of = [&](const Item& it) {
+            return it.ntiles ? (((it.tile0 + it.ntiles) * TILE_T - 1) >> p.page_shift) + 1 - first_page(it) : 0;
+        };
+        // Index of the k-th item this CTA takes.  With the dynamic schedule lane 0 holds the counter's answer
+        // in `raw` until it is needed, so that the atomic's round trip overlaps the current item's loads.
+        auto request = [&](int k) -> int {
+            if (!p.persistent) return k == 0 ? 0 : n_items;
+            if (dynamic) return lane == 0 ? atomicAdd(p.sched, 1) : 0;
+            return (int)blockIdx.x + k * item_step;
+        };
+        auto settle = [&](int raw) -> int { return dynamic ? __shfl_sync(0xffffffffu, raw, 0) : raw; };
+
+        int s = 0, issued = 0, k = 0;                // ring position, stages armed so far, items taken so far
+        uint32_t ph = 0;
+        bool alive = true;
+        int i_cur = settle(request(0));
+        int raw_nxt = request(1);
+        Item cur;
+        if (i_cur < n_items) {                       // page ids of the first item
+            cur = get_item(i_cur);
+            const int page0 = first_page(cur), npages = num_pages_of(cur);
+            for (int i = lane; i < npages && i < MAX_CHUNK_PAGES; i += 32) ctl.pages[i] = check_page(lookup(cur, page0 + i));
+            __syncwarp();
+        }
+        while (i_cur < n_items && alive) {
+            const int page0 = first_page(cur);
+            const int* const pages = &ctl.pages[(k & 1) * (MAX_CHUNK_PAGES / 2)];
+            // the next item: its index was requested one item ago; request the one after it, and start fetching
+            // the next item's page ids (parked in shared memory after this item's loads have been issued)
+            const int i_nxt = settle(raw_nxt);
+            raw_nxt = request(k + 2);
+            const bool has_next = i_nxt < n_items;
+            Item nxt = cur;
+            int nxt_ids[PER_LANE];
+            int nxt_npages = 0;
+            if (has_next) {
+                nxt = get_item(i_nxt);
+                const int np0 = first_page(nxt);
+                nxt_npages = min(num_pages_of(nxt), PERSIST_CHUNK_PAGES);
+#pragma unroll
+                for (int u = 0; u < PER_LANE; ++u) {
+                    const int idx = u * 32 + lane;
+                    nxt_ids[u] = idx < nxt_npages ? lookup(nxt, np0 + idx) : -2;
+                }
+            }
+            const int g = cur.y / p.head_blocks;
+            for (int it = 0; it < cur.ntiles; ++it) {              // one stage = K tile + V tile of 64 tokens
+                int okw = 1;
+                if (lane == 0) okw = mbar_wait(&ctl.empty[s], ph ^ 1u, abort_flag) ? 1 : 0;
+                okw = __shfl_sync(0xffffffffu, okw, 0);
+                if (!okw) { alive = false; break; }
+                const int t0j = (cur.tile0 + it) * TILE_T + j * R;
+                int phys = -1;
+                if (isv < 2 && t0j < cur.hi && t0j + R > cur.lo) phys = pages[(t0j >> p.page_shift) - page0];
+                const uint32_t nvalid = __popc(__ballot_sync(0xffffffffu, phys >= 0));   // K and V boxes
+                if (lane == 0) {
+                    ctl.sdesc[s] = make_int2(i_cur, it);
+                    mbar_arrive_expect_tx(&ctl.full[s], nvalid * box_bytes);
+                }
+                __syncwarp();
+                if (phys >= 0) {
+                    uint8_t* dst = stage0_ptr + (size_t)s * STAGE_BYTES + isv * TILE_BYTES + j * box_bytes;
+                    tma_load_5d(dst, isv ? &tmV : &tmK, &ctl.full[s], 0, t0j & (p.page_size - 1), 0, g, phys, policy);
+                }
+                ++issued;
+                if (++s == p.stages) { s = 0; ph ^= 1u; }
+            }
+            if (!has_next) break;
+            int* const dstp = &ctl.pages[((k + 1) & 1) * (MAX_CHUNK_PAGES / 2)];
+#pragma unroll
+            for (int u = 0; u < PER_LANE; ++u) {
+                const int idx = u * 32 + lane;
+                if (idx < nxt_npages) dstp[idx] = check_page(nxt_ids[u]);
+            }
+            __syncwarp();
+            cur = nxt;
+            i_cur = i_nxt;
+            ++k;
+        }
+        if (alive) {
+            // no more work: one last, empty stage tells the consumers
             int okw = 1;
             if (lane == 0) okw = mbar_wait(&ctl.empty[s], ph ^ 1u, abort_flag) ? 1 : 0;
             okw = __shfl_sync(0xffffffffu, okw, 0);
-            if (!okw) break;
-            const int tokbase = (tile0 + (it >> 1)) * TILE_T;
-            const int t0j = tokbase + j * rows;
-            int phys = -1;
-            if (j < nbox && t0j < hi && t0j + rows > lo) phys = ctl.pages[(t0j >> p.page_shift) - page0];
-            const uint32_t nvalid = __popc(__ballot_sync(0xffffffffu, phys >= 0 && h == 0));
-            if (lane == 0) mbar_arrive_expect_tx(&ctl.full[s], nvalid * (uint32_t)rows * 128u * HALVES);
-            __syncwarp();
-            if (phys >= 0) {
-                const int tin = t0j & (p.page_size - 1);
-                uint8_t* dst = stage0_ptr + (size_t)s * STAGE_BYTES + h * HALF_BYTES + j * rows * 128;
-                tma_load_4d(dst, (it & 1) ? &tmV : &tmK, &ctl.full[s], h * 64, pick3(p.perm0, tin, g, phys),
-                            pick3(p.perm1, tin, g, phys), pick3(p.perm2, tin, g, phys), policy);
+            if (okw && lane == 0) {
+                ctl.sdesc[s] = make_int2(-1, 0);
+                mbar_arrive_expect_tx(&ctl.full[s], 0u);
             }
-            issued = it + 1;
         }
         if (*abort_flag && lane == 0) {
             // unwinding: do not leave the CTA while copies into its shared memory may still land
-            for (int it = max(0, issued - p.stages); it < issued; ++it) {
+            for (int g2 = max(0, issued - p.stages); g2 < issued; ++g2) {
                 int dummy = 0;
-                mbar_wait(&ctl.full[it % p.stages], (uint32_t)(it / p.stages) & 1u, &dummy);
+                mbar_wait(&ctl.full[g2 % p.stages], (uint32_t)(g2 / p.stages) & 1u, &dummy);
             }
-        }
-    } else if constexpr (MODE == MODE_PROBE) {
-        // ======================= probe consumers =======================
-        for (int it = 0; it < n_iter; ++it) {
-            const int s = it % p.stages;
-            if (!warp_wait(&ctl.full[s], (uint32_t)(it / p.stages) & 1u, abort_flag)) break;
-            const uint32_t base = stage0 + s * STAGE_BYTES;
-            const int tokbase = (tile0 + (it >> 1)) * TILE_T;
-#pragma unroll
-            for (int i = 0; i < 4 * HALVES; ++i) {
-                // 16 rows x HALVES x 8 chunks per warp; a quarter-warp reads one 128-byte row segment
-                const int idx = i * 32 + lane;
-                const int r = row0 + (idx >> 3) % 16, hh = (idx >> 3) / 16;
-                const int t = tokbase + r;
-                if (t >= lo && t < hi) {
-                    uint4 v = lds128(base + hh * HALF_BYTES + r * 128 + ((idx & 7) << 4));
-                    probe_x ^= v.x ^ v.y ^ v.z ^ v.w;
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&ctl.empty[s]);
-        }
-    } else if constexpr (MODE == MODE_MHA) {
-        // ======================= MHA consumers (CUDA cores) =======================
-        float qf[NV];
-        {
-            const uint16_t* qrow = reinterpret_cast<const uint16_t*>(p.q) + ((size_t)b * p.Hq + h0) * D;
-#pragma unroll
-            for (int hh = 0; hh < HALVES; ++hh) {
-                uint4 raw = *reinterpret_cast<const uint4*>(qrow + hh * 64 + li * 8);
-                float2 a = unpack2<BF16>(raw.x), bb = unpack2<BF16>(raw.y), cc = unpack2<BF16>(raw.z),
-                       dd = unpack2<BF16>(raw.w);
-                qf[hh * 8 + 0] = a.x; qf[hh * 8 + 1] = a.y; qf[hh * 8 + 2] = bb.x; qf[hh * 8 + 3] = bb.y;
-                qf[hh * 8 + 4] = cc.x; qf[hh * 8 + 5] = cc.y; qf[hh * 8 + 6] = dd.x; qf[hh * 8 + 7] = dd.y;
-            }
-        }
-        const int rbase = row0 + gi * 4;      // this lane group's 4 rows
-        for (int jt = 0; jt < ntiles; ++jt) {
-            const int tokbase = (tile0 + jt) * TILE_T;
-            bool valid[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) { const int t = tokbase + rbase + k; valid[k] = t >= lo && t < hi; }
-
-            // ---- K tile: 4 logits per lane group ----
-            int it = 2 * jt, s = it % p.stages;
-            if (!warp_wait(&ctl.full[s], (uint32_t)(it / p.stages) & 1u, abort_flag)) break;
-            uint32_t base = stage0 + s * STAGE_BYTES;
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const int r = rbase + k;
-#pragma unroll
-                for (int hh = 0; hh < HALVES; ++hh) {
-                    uint4 raw = lds128(base + hh * HALF_BYTES + r * 128 + ((li ^ (r & 7)) << 4));
-                    float2 a = unpack2<BF16>(raw.x), bb = unpack2<BF16>(raw.y), cc = unpack2<BF16>(raw.z),
-                           dd = unpack2<BF16>(raw.w);
-                    const float* qq = &qf[hh * 8];
-                    acc[k] = fmaf(a.x, qq[0], acc[k]); acc[k] = fmaf(a.y, qq[1], acc[k]);
-                    acc[k] = fmaf(bb.x, qq[2], acc[k]); acc[k] = fmaf(bb.y, qq[3], acc[k]);
-                    acc[k] = fmaf(cc.x, qq[4], acc[k]); acc[k] = fmaf(cc.y, qq[5], acc[k]);
-                    acc[k] = fmaf(dd.x, qq[6], acc[k]); acc[k] = fmaf(dd.y, qq[7], acc[k]);
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&ctl.empty[s]);
-            float s2[4], mx = NEG_INF;
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                float v = acc[k];
-                v += __shfl_xor_sync(0xffffffffu, v, 1);
-                v += __shfl_xor_sync(0xffffffffu, v, 2);
-                v += __shfl_xor_sync(0xffffffffu, v, 4);
-                s2[k] = valid[k] ? v * p.scale_log2 : NEG_INF;
-                mx = fmaxf(mx, s2[k]);
-            }
-            const float m_new = fmaxf(mha_m, mx);
-            const float m_safe = (m_new == NEG_INF) ? 0.f : m_new;
-            const float corr = fast_exp2(mha_m - m_safe);
-            float pk[4], psum = 0.f;
-#pragma unroll
-            for (int k = 0; k < 4; ++k) { pk[k] = fast_exp2(s2[k] - m_safe); psum += pk[k]; }
-            mha_l = mha_l * corr + psum;
-            mha_m = m_new;
-
-            // ---- V tile: o = o * corr + sum_k p_k V_k ----
-            it = 2 * jt + 1; s = it % p.stages;
-            if (!warp_wait(&ctl.full[s], (uint32_t)(it / p.stages) & 1u, abort_flag)) break;
-            base = stage0 + s * STAGE_BYTES;
-#pragma unroll
-            for (int i = 0; i < NV; ++i) mha_o[i] *= corr;
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const int r = rbase + k;
-#pragma unroll
-                for (int hh = 0; hh < HALVES; ++hh) {
-                    uint4 raw = make_uint4(0u, 0u, 0u, 0u);      // rows outside the slice never enter the sum
-                    if (valid[k]) raw = lds128(base + hh * HALF_BYTES + r * 128 + ((li ^ (r & 7)) << 4));
-                    float2 a = unpack2<BF16>(raw.x), bb = unpack2<BF16>(raw.y), cc = unpack2<BF16>(raw.z),
-                           dd = unpack2<BF16>(raw.w);
-                    float* oo = &mha_o[hh * 8];
-                    oo[0] = fmaf(pk[k], a.x, oo[0]); oo[1] = fmaf(pk[k], a.y, oo[1]);
-                    oo[2] = fmaf(pk[k], bb.x, oo[2]); oo[3] = fmaf(pk[k], bb.y, oo[3]);
-                    oo[4] = fmaf(pk[k], cc.x, oo[4]); oo[5] = fmaf(pk[k], cc.y, oo[5]);
-                    oo[6] = fmaf(pk[k], dd.x, oo[6]); oo[7] = fmaf(pk[k], dd.y, oo[7]);
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&ctl.empty[s]);
         }
     } else {
-        // ======================= GQA consumers (tensor cores) =======================
-        // q^T as the B operand of S^T = K q^T: b0 = q[head quad][16 ks + 2 tq + {0,1}], b1 = the same + 8
-        uint32_t qb[KSTEPS][2];
-        {
-            const bool live = hb * 8 + quad < p.G;
-            const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
-                reinterpret_cast<const uint16_t*>(p.q) + ((size_t)b * p.Hq + (live ? h0 + quad : h0)) * D);
-#pragma unroll
-            for (int ks = 0; ks < KSTEPS; ++ks) {
-                qb[ks][0] = live ? qrow[ks * 8 + tq] : 0u;
-                qb[ks][1] = live ? qrow[ks * 8 + 4 + tq] : 0u;
-            }
-        }
-        // ldmatrix row addresses (within a tile) for this lane
-        const int a_row = row0 + (lane & 7) + ((lane >> 3) & 1) * 8;   // K: matrices (rows, rows+8) x (k lo, k hi)
-        const int a_kc = lane >> 4;
-        const int v_row = row0 + (lane & 7) + (lane >> 4) * 8;         // V^T: matrices (d lo, d hi) x (tok, tok+8)
-        const int v_dc = (lane >> 3) & 1;
-
-        for (int jt = 0; jt < ntiles; ++jt) {
-            const int tokbase = (tile0 + jt) * TILE_T;
-            const int tA = tokbase + row0 + quad, tB = tA + 8;
-            const bool vA = tA >= lo && tA < hi, vB = tB >= lo && tB < hi;
-            const bool edge = tokbase < lo || tokbase + TILE_T > hi;
-
-            // ---- S^T (16 tokens x 8 heads) ----
-            int it = 2 * jt, s = it % p.stages;
-            if (!warp_wait(&ctl.full[s], (uint32_t)(it / p.stages) & 1u, abort_flag)) break;
-            uint32_t base = stage0 + s * STAGE_BYTES;
-            float sc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int ks = 0; ks < KSTEPS; ++ks) {
-                const int ch = 2 * ks + a_kc;   // 16-byte chunk index along d
-                uint32_t a[4];
-                ldmatrix_x4(a, base + (ch >> 3) * HALF_BYTES + a_row * 128 + (((ch & 7) ^ (a_row & 7)) << 4));
-                mma_16816<BF16>(sc, a, qb[ks][0], qb[ks][1]);
-            }
+        // =============================== consumer warps ===============================
+        int cs = 0;                // ring position and phase of the next stage to consume
+        uint32_t cph = 0;
+        // Barrier among the four consumer warps with a bounded wait (false: give up, the CTA is unwinding).
+        uint32_t cphase = 0;
+        auto consumer_sync = [&]() -> bool {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl.cbar);
+            const bool ok = warp_wait(&ctl.cbar, cphase, abort_flag);
+            cphase ^= 1u;
+            return ok;
+        };
+        // Hands a consumed stage back to the producer.  `wrote` tells that this warp stored to the stage
+        // through the generic proxy, which must be ordered before the next TMA write into it.
+        auto release = [&](int s, bool wrote) {
+            if (wrote) fence_proxy_async();
             __syncwarp();
             if (lane == 0) mbar_arrive(&ctl.empty[s]);
+        };
+        // Waits for the next filled stage; returns its ring position, or -1 when there is no more work (or the
+        // CTA is unwinding).  d receives the stage's descriptor.
+        auto next_stage = [&](int2& d) -> int {
+            const int s = cs;
+            if (!warp_wait(&ctl.full[s], cph, abort_flag)) return -1;
+            if (++cs == p.stages) { cs = 0; cph ^= 1u; }
+            d = ctl.sdesc[s];
+            return d.x < 0 ? -1 : s;
+        };
 
-            // sc[0], sc[1]: token tA, heads 2tq, 2tq+1; sc[2], sc[3]: token tB
-            float s2[4];
-            s2[0] = vA ? sc[0] * p.scale_log2 : NEG_INF; s2[1] = vA ? sc[1] * p.scale_log2 : NEG_INF;
-            s2[2] = vB ? sc[2] * p.scale_log2 : NEG_INF; s2[3] = vB ? sc[3] * p.scale_log2 : NEG_INF;
-            float mx[2] = {fmaxf(s2[0], s2[2]), fmaxf(s2[1], s2[3])};
-#pragma unroll
-            for (int o = 4; o <= 16; o <<= 1) {
-                mx[0] = fmaxf(mx[0], __shfl_xor_sync(0xffffffffu, mx[0], o));
-                mx[1] = fmaxf(mx[1], __shfl_xor_sync(0xffffffffu, mx[1], o));
-            }
-            float corr[2], msafe[2];
-#pragma unroll
-            for (int hc = 0; hc < 2; ++hc) {
-                const float m_new = fmaxf(gqa_m[hc], mx[hc]);
-                msafe[hc] = (m_new == NEG_INF) ? 0.f : m_new;
-                corr[hc] = fast_exp2(gqa_m[hc] - msafe[hc]);
-                gqa_m[hc] = m_new;
-            }
-            float pr[4];
-            pr[0] = fast_exp2(s2[0] - msafe[0]); pr[1] = fast_exp2(s2[1] - msafe[1]);
-            pr[2] = fast_exp2(s2[2] - msafe[0]); pr[3] = fast_exp2(s2[3] - msafe[1]);
-            gqa_l[0] = gqa_l[0] * corr[0] + pr[0] + pr[2];   // per-lane sums over its own two token rows
-            gqa_l[1] = gqa_l[1] * corr[1] + pr[1] + pr[3];
+        Item cur;
+        cur.b = cur.y = cur.c = cur.lo = cur.hi = cur.tile0 = cur.ntiles = 0;
+        int hb = 0, nheads = 1, h0 = 0;
+        auto begin_item = [&](int i) {
+            cur = get_item(i);
+            hb = cur.y % p.head_blocks;
+            const int g = cur.y / p.head_blocks;
+            nheads = (MODE == MODE_GQA) ? min(8, p.G - hb * 8) : 1;
+            h0 = (MODE == MODE_GQA) ? g * p.G + hb * 8 : g;      // first query head of this item
+        };
 
-            // P^T as the B operand of O^T += V^T P^T, as hi + lo 16-bit terms
-            const uint32_t hiA = pack2<BF16>(pr[0], pr[1]), hiB = pack2<BF16>(pr[2], pr[3]);
-            const float2 fA = unpack2<BF16>(hiA), fB = unpack2<BF16>(hiB);
-            const uint32_t loA = pack2<BF16>(pr[0] - fA.x, pr[1] - fA.y), loB = pack2<BF16>(pr[2] - fB.x, pr[3] - fB.y);
-            const uint32_t bh0 = movmatrix_trans(hiA), bh1 = movmatrix_trans(hiB);
-            const uint32_t bl0 = movmatrix_trans(loA), bl1 = movmatrix_trans(loB);
-
-            // ---- O^T ----
-            it = 2 * jt + 1; s = it % p.stages;
-            if (!warp_wait(&ctl.full[s], (uint32_t)(it / p.stages) & 1u, abort_flag)) break;
-            base = stage0 + s * STAGE_BYTES;
-            if (edge) {
-                // rows outside the slice may hold anything (even NaN patterns): clear this warp's copies
-                for (int i = lane; i < 16 * 8 * HALVES; i += 32) {
-                    const int r = row0 + (i / (8 * HALVES)), ch = i % (8 * HALVES);
-                    const int t = tokbase + r;
-                    if (t < lo || t >= hi) sts128_zero(base + (ch >> 3) * HALF_BYTES + r * 128 + ((ch & 7) << 4));
-                }
-                __syncwarp();
-            }
-#pragma unroll
-            for (int mt = 0; mt < KSTEPS; ++mt) {
-                gqa_o[mt][0] *= corr[0]; gqa_o[mt][1] *= corr[1]; gqa_o[mt][2] *= corr[0]; gqa_o[mt][3] *= corr[1];
-                const int ch = 2 * mt + v_dc;
-                uint32_t a[4];
-                ldmatrix_x4_trans(a, base + (ch >> 3) * HALF_BYTES + v_row * 128 + (((ch & 7) ^ (v_row & 7)) << 4));
-                mma_16816<BF16>(gqa_o[mt], a, bh0, bh1);
-                mma_16816<BF16>(gqa_o[mt], a, bl0, bl1);
-            }
-            if (edge) fence_proxy_async();   // the generic-proxy stores above precede the next TMA write to this stage
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&ctl.empty[s]);
-        }
-#pragma unroll
-        for (int o = 4; o <= 16; o <<= 1) {
-            gqa_l[0] += __shfl_xor_sync(0xffffffffu, gqa_l[0], o);
-            gqa_l[1] += __shfl_xor_sync(0xffffffffu, gqa_l[1], o);
-        }
-    }
-
-    // ---- every issued tile has landed and been read: the stage memory becomes the reduction buffer ----
-    __syncthreads();
-    float* const red_o = reinterpret_cast<float*>(stage0_ptr);
-    if (warp < CONSUMER_WARPS && !*abort_flag) {
         if constexpr (MODE == MODE_PROBE) {
+            uint32_t probe_x = 0u;
+            for (;;) {
+                int2 d;
+                const int s = next_stage(d);
+                if (s < 0) break;
+                if (d.y == 0) { begin_item(d.x); probe_x = 0u; }
+                const uint32_t base = stage0 + s * STAGE_BYTES;
+                const int tokbase = (cur.tile0 + d.y) * TILE_T;
 #pragma unroll
-            for (int o = 16; o; o >>= 1) probe_x ^= __shfl_xor_sync(0xffffffffu, probe_x, o);
-            if (lane == 0) atomicXor(&ctl.probe_acc, probe_x);
+                for (int u = 0; u < 8 * HALVES; ++u) {
+                    // K and V: 16 rows x HALVES x 8 chunks each per warp; a quarter-warp reads one 128-byte row segment
+                    const int idx = u * 32 + lane;
+                    const int r = row0 + (idx >> 3) % 16, hh = ((idx >> 3) / 16) % HALVES, kv = (idx >> 3) / (16 * HALVES);
+                    const int t = tokbase + r;
+                    if (t >= cur.lo && t < cur.hi) {
+                        uint4 v = lds128(base + kv * TILE_BYTES + row_off(r) + hh * half_stride + ((idx & 7) << 4));
+                        probe_x ^= v.x ^ v.y ^ v.z ^ v.w;
+                    }
+                }
+                if (d.y + 1 < cur.ntiles) { release(s, false); continue; }
+                // item epilogue, with the item's last stage as scratch
+#pragma unroll
+                for (int o = 16; o; o >>= 1) probe_x ^= __shfl_xor_sync(0xffffffffu, probe_x, o);
+                uint32_t* red = reinterpret_cast<uint32_t*>(stage0_ptr + (size_t)s * STAGE_BYTES);
+                if (!consumer_sync()) break;                      // every warp has read the last stage
+                if (lane == 0) red[warp] = probe_x;
+                if (!consumer_sync()) break;
+                if (tid == 0) p.sink[((size_t)cur.b * p.Hkv + cur.y) * p.NC + cur.c] = red[0] ^ red[1] ^ red[2] ^ red[3];
+                release(s, true);
+            }
         } else if constexpr (MODE == MODE_MHA) {
-            const int slot = warp * 4 + gi;                       // red_o [16 row groups][D]
-            if (li == 0) { ctl.red_m[slot] = mha_m; ctl.red_l[slot] = mha_l; }
+            // ----------------------- MHA (CUDA cores) -----------------------
+            float qf[NV], m_run = NEG_INF, l_run = 0.f, o[NV];
+            const int rbase = row0 + gi * 4;                      // this lane group's 4 rows
+            uint32_t roff[4];
 #pragma unroll
-            for (int hh = 0; hh < HALVES; ++hh) {
-                float4* dst = reinterpret_cast<float4*>(red_o + slot * D + hh * 64 + li * 8);
-                dst[0] = make_float4(mha_o[hh * 8 + 0], mha_o[hh * 8 + 1], mha_o[hh * 8 + 2], mha_o[hh * 8 + 3]);
-                dst[1] = make_float4(mha_o[hh * 8 + 4], mha_o[hh * 8 + 5], mha_o[hh * 8 + 6], mha_o[hh * 8 + 7]);
+            for (int k = 0; k < 4; ++k) roff[k] = row_off(rbase + k) + (uint32_t)((li ^ ((rbase + k) & 7)) << 4);
+
+            for (;;) {
+                int2 d;
+                const int s = next_stage(d);
+                if (s < 0) break;
+                if (d.y == 0) {
+                    begin_item(d.x);
+                    const uint16_t* qrow = reinterpret_cast<const uint16_t*>(p.q) + ((size_t)cur.b * p.Hq + h0) * D;
+#pragma unroll
+                    for (int hh = 0; hh < HALVES; ++hh) {
+                        uint4 raw = *reinterpret_cast<const uint4*>(qrow + hh * 64 + li * 8);
+                        float2 a = unpack2<BF16>(raw.x), bb = unpack2<BF16>(raw.y), cc = unpack2<BF16>(raw.z),
+                               dd = unpack2<BF16>(raw.w);
+                        qf[hh * 8 + 0] = a.x; qf[hh * 8 + 1] = a.y; qf[hh * 8 + 2] = bb.x; qf[hh * 8 + 3] = bb.y;
+                        qf[hh * 8 + 4] = cc.x; qf[hh * 8 + 5] = cc.y; qf[hh * 8 + 6] = dd.x; qf[hh * 8 + 7] = dd.y;
+                    }
+                    m_run = NEG_INF; l_run = 0.f;
+#pragma unroll
+                    for (int u = 0; u < NV; ++u) o[u] = 0.f;
+                }
+                const int tokbase = (cur.tile0 + d.y) * TILE_T;
+                bool valid[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) { const int t = tokbase + rbase + k; valid[k] = t >= cur.lo && t < cur.hi; }
+                const uint32_t kbase = stage0 + s * STAGE_BYTES, vbase = kbase + TILE_BYTES;
+
+                // ---- K tile: 4 logits per lane group ----
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+#pragma unroll
+                    for (int hh = 0; hh < HALVES; ++hh) {
+                        uint4 raw = lds128(kbase + roff[k] + hh * half_stride);
+                        float2 a = unpack2<BF16>(raw.x), bb = unpack2<BF16>(raw.y), cc = unpack2<BF16>(raw.z),
+                               dd = unpack2<BF16>(raw.w);
+                        const float* qq = &qf[hh * 8];
+                        acc[k] = fmaf(a.x, qq[0], acc[k]); acc[k] = fmaf(a.y, qq[1], acc[k]);
+                        acc[k] = fmaf(bb.x, qq[2], acc[k]); acc[k] = fmaf(bb.y, qq[3], acc[k]);
+                        acc[k] = fmaf(cc.x, qq[4], acc[k]); acc[k] = fmaf(cc.y, qq[5], acc[k]);
+                        acc[k] = fmaf(dd.x, qq[6], acc[k]); acc[k] = fmaf(dd.y, qq[7], acc[k]);
+                    }
+                }
+                float s2[4], mx = NEG_INF;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    float v = acc[k];
+                    v += __shfl_xor_sync(0xffffffffu, v, 1);
+                    v += __shfl_xor_sync(0xffffffffu, v, 2);
+                    v += __shfl_xor_sync(0xffffffffu, v, 4);
+                    s2[k] = valid[k] ? v * p.scale_log2 : NEG_INF;
+                    mx = fmaxf(mx, s2[k]);
+                }
+                const float m_new = fmaxf(m_run, mx);
+                const float m_safe = (m_new == NEG_INF) ? 0.f : m_new;
+                const float corr = fast_exp2(m_run - m_safe);
+                float pk[4], psum = 0.f;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) { pk[k] = fast_exp2(s2[k] - m_safe); psum += pk[k]; }
+                l_run = l_run * corr + psum;
+                m_run = m_new;
+
+                // ---- V tile: o = o * corr + sum_k p_k V_k ----
+#pragma unroll
+                for (int u = 0; u < NV; ++u) o[u] *= corr;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+#pragma unroll
+                    for (int hh = 0; hh < HALVES; ++hh) {
+                        uint4 raw = make_uint4(0u, 0u, 0u, 0u);      // rows outside the slice never enter the sum
+                        if (valid[k]) raw = lds128(vbase + roff[k] + hh * half_stride);
+                        float2 a = unpack2<BF16>(raw.x), bb = unpack2<BF16>(raw.y), cc = unpack2<BF16>(raw.z),
+                               dd = unpack2<BF16>(raw.w);
+                        float* oo = &o[hh * 8];
+                        oo[0] = fmaf(pk[k], a.x, oo[0]); oo[1] = fmaf(pk[k], a.y, oo[1]);
+                        oo[2] = fmaf(pk[k], bb.x, oo[2]); oo[3] = fmaf(pk[k], bb.y, oo[3]);
+                        oo[4] = fmaf(pk[k], cc.x, oo[4]); oo[5] = fmaf(pk[k], cc.y, oo[5]);
+                        oo[6] = fmaf(pk[k], dd.x, oo[6]); oo[7] = fmaf(pk[k], dd.y, oo[7]);
+                    }
+                }
+                if (d.y + 1 < cur.ntiles) { release(s, false); continue; }
+
+                // ---- item epilogue: merge the 16 row-group states (the item's last stage is the scratch) ----
+                float* red_o = reinterpret_cast<float*>(stage0_ptr + (size_t)s * STAGE_BYTES);   // [16 row groups][D]
+                if (!consumer_sync()) break;                      // every warp has read the last stage
+                const int slot = warp * 4 + gi;
+                if (li == 0) { ctl.red_m[slot] = m_run; ctl.red_l[slot] = l_run; }
+#pragma unroll
+                for (int hh = 0; hh < HALVES; ++hh) {
+                    float4* dst = reinterpret_cast<float4*>(red_o + slot * D + hh * 64 + li * 8);
+                    dst[0] = make_float4(o[hh * 8 + 0], o[hh * 8 + 1], o[hh * 8 + 2], o[hh * 8 + 3]);
+                    dst[1] = make_float4(o[hh * 8 + 4], o[hh * 8 + 5], o[hh * 8 + 6], o[hh * 8 + 7]);
+                }
+                if (!consumer_sync()) break;
+                if (tid < D) {
+                    float M = NEG_INF;
+#pragma unroll
+                    for (int sidx = 0; sidx < 16; ++sidx) M = fmaxf(M, ctl.red_m[sidx]);
+                    float accv = 0.f, lsum = 0.f;
+#pragma unroll
+                    for (int sidx = 0; sidx < 16; ++sidx) {
+                        const float w = fast_exp2(ctl.red_m[sidx] - M);      // -inf states weigh 0; M is finite
+                        accv = fmaf(w, red_o[sidx * D + tid], accv);
+                        lsum = fmaf(w, ctl.red_l[sidx], lsum);
+                    }
+                    const size_t oslot = ((size_t)cur.b * p.Hq + h0) * p.NC + cur.c;
+                    p.o_part[oslot * D + tid] = accv;
+                    if (tid == 0) { p.m_part[oslot] = M * LN2; p.l_part[oslot] = lsum; }
+                }
+                release(s, true);
             }
         } else {
-            if (quad == 0) {                                      // red_o [4 warps][8 heads][D]
-                ctl.red_m[warp * 8 + 2 * tq] = gqa_m[0]; ctl.red_m[warp * 8 + 2 * tq + 1] = gqa_m[1];
-                ctl.red_l[warp * 8 + 2 * tq] = gqa_l[0]; ctl.red_l[warp * 8 + 2 * tq + 1] = gqa_l[1];
-            }
-            float* w = red_o + (size_t)warp * 8 * D;
+            // ----------------------- GQA (tensor cores) -----------------------
+            uint32_t qb[KSTEPS][2];      // q^T as the B operand of S^T = K q^T
+            float m_run[2] = {NEG_INF, NEG_INF}, l_run[2] = {0.f, 0.f}, oacc[KSTEPS][4];
+            // ldmatrix row addresses for this lane
+            const int a_row = row0 + (lane & 7) + ((lane >> 3) & 1) * 8;   // K: matrices (rows, rows+8) x (k lo, k hi)
+            const int a_kc = lane >> 4;
+            const int v_row = row0 + (lane & 7) + (lane >> 4) * 8;         // V^T: matrices (d lo, d hi) x (tok, tok+8)
+            const int v_dc = (lane >> 3) & 1;
+            const uint32_t a_off = row_off(a_row), v_off = row_off(v_row);
+
+            for (;;) {
+                int2 d;
+                const int s = next_stage(d);
+                if (s < 0) break;
+                if (d.y == 0) {
+                    begin_item(d.x);
+                    // b0 = q[head quad][16 ks + 2 tq + {0,1}], b1 = the same + 8; heads past the group read as zero
+                    const bool live = hb * 8 + quad < p.G;
+                    const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
+                        reinterpret_cast<const uint16_t*>(p.q) + ((size_t)cur.b * p.Hq + (live ? h0 + quad : h0)) * D);
 #pragma unroll
-            for (int mt = 0; mt < KSTEPS; ++mt) {
-                const int d0 = mt * 16 + quad;
-                w[(2 * tq) * D + d0] = gqa_o[mt][0];
-                w[(2 * tq + 1) * D + d0] = gqa_o[mt][1];
-                w[(2 * tq) * D + d0 + 8] = gqa_o[mt][2];
-                w[(2 * tq + 1) * D + d0 + 8] = gqa_o[mt][3];
+                    for (int ks = 0; ks < KSTEPS; ++ks) {
+                        qb[ks][0] = live ? qrow[ks * 8 + tq] : 0u;
+                        qb[ks][1] = live ? qrow[ks * 8 + 4 + tq] : 0u;
+                    }
+                    m_run[0] = m_run[1] = NEG_INF; l_run[0] = l_run[1] = 0.f;
+#pragma unroll
+                    for (int u = 0; u < KSTEPS; ++u) { oacc[u][0] = oacc[u][1] = oacc[u][2] = oacc[u][3] = 0.f; }
+                }
+                const int tokbase = (cur.tile0 + d.y) * TILE_T;
+                const int tA = tokbase + row0 + quad, tB = tA + 8;
+                const bool vA = tA >= cur.lo && tA < cur.hi, vB = tB >= cur.lo && tB < cur.hi;
+                const bool edge = tokbase < cur.lo || tokbase + TILE_T > cur.hi;
+                const uint32_t kbase = stage0 + s * STAGE_BYTES, vbase = kbase + TILE_BYTES;
+
+                // ---- S^T (16 tokens x 8 heads) ----
+                float sc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int ks = 0; ks < KSTEPS; ++ks) {
+                    const int ch = 2 * ks + a_kc;   // 16-byte chunk index along d
+                    uint32_t a[4];
+                    ldmatrix_x4(a, kbase + a_off + (ch >> 3) * half_stride + (((ch & 7) ^ (a_row & 7)) << 4));
+                    mma_16816<BF16>(sc, a, qb[ks][0], qb[ks][1]);
+                }
+                // sc[0], sc[1]: token tA, heads 2tq, 2tq+1; sc[2], sc[3]: token tB
+                float s2[4];
+                s2[0] = vA ? sc[0] * p.scale_log2 : NEG_INF; s2[1] = vA ? sc[1] * p.scale_log2 : NEG_INF;
+                s2[2] = vB ? sc[2] * p.scale_log2 : NEG_INF; s2[3] = vB ? sc[3] * p.scale_log2 : NEG_INF;
+                float mx[2] = {fmaxf(s2[0], s2[2]), fmaxf(s2[1], s2[3])};
+#pragma unroll
+                for (int o = 4; o <= 16; o <<= 1) {
+                    mx[0] = fmaxf(mx[0], __shfl_xor_sync(0xffffffffu, mx[0], o));
+                    mx[1] = fmaxf(mx[1], __shfl_xor_sync(0xffffffffu, mx[1], o));
+                }
+                float corr[2], msafe[2];
+#pragma unroll
+                for (int hc = 0; hc < 2; ++hc) {
+                    const float m_new = fmaxf(m_run[hc], mx[hc]);
+                    msafe[hc] = (m_new == NEG_INF) ? 0.f : m_new;
+                    corr[hc] = fast_exp2(m_run[hc] - msafe[hc]);
+                    m_run[hc] = m_new;
+                }
+                float pr[4];
+                pr[0] = fast_exp2(s2[0] - msafe[0]); pr[1] = fast_exp2(s2[1] - msafe[1]);
+                pr[2] = fast_exp2(s2[2] - msafe[0]); pr[3] = fast_exp2(s2[3] - msafe[1]);
+                l_run[0] = l_run[0] * corr[0] + pr[0] + pr[2];   // per-lane sums over its own two token rows
+                l_run[1] = l_run[1] * corr[1] + pr[1] + pr[3];
+
+                // P^T as the B operand of O^T += V^T P^T, as hi + lo 16-bit terms
+                const uint32_t hiA = pack2<BF16>(pr[0], pr[1]), hiB = pack2<BF16>(pr[2], pr[3]);
+                const float2 fA = unpack2<BF16>(hiA), fB = unpack2<BF16>(hiB);
+                const uint32_t loA = pack2<BF16>(pr[0] - fA.x, pr[1] - fA.y), loB = pack2<BF16>(pr[2] - fB.x, pr[3] - fB.y);
+                const uint32_t bh0 = movmatrix_trans(hiA), bh1 = movmatrix_trans(hiB);
+                const uint32_t bl0 = movmatrix_trans(loA), bl1 = movmatrix_trans(loB);
+
+                // ---- O^T ----
+                if (edge) {
+                    // rows outside the slice may hold anything (even NaN patterns): clear this warp's copies
+                    for (int u = lane; u < 16 * 8 * HALVES; u += 32) {
+                        const int r = row0 + (u / (8 * HALVES)), ch = u % (8 * HALVES);
+                        const int t = tokbase + r;
+                        if (t < cur.lo || t >= cur.hi) sts128_zero(vbase + row_off(r) + (ch >> 3) * half_stride + ((ch & 7) << 4));
+                    }
+                    __syncwarp();
+                }
+#pragma unroll
+                for (int mt = 0; mt < KSTEPS; ++mt) {
+                    oacc[mt][0] *= corr[0]; oacc[mt][1] *= corr[1]; oacc[mt][2] *= corr[0]; oacc[mt][3] *= corr[1];
+                    const int ch = 2 * mt + v_dc;
+                    uint32_t a[4];
+                    ldmatrix_x4_trans(a, vbase + v_off + (ch >> 3) * half_stride + (((ch & 7) ^ (v_row & 7)) << 4));
+                    mma_16816<BF16>(oacc[mt], a, bh0, bh1);
+                    mma_16816<BF16>(oacc[mt], a, bl0, bl1);
+                }
+                if (d.y + 1 < cur.ntiles) { release(s, edge); continue; }
+
+                // ---- item epilogue: merge the 4 warp states (the item's last stage is the scratch) ----
+#pragma unroll
+                for (int o = 4; o <= 16; o <<= 1) {
+                    l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], o);
+                    l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], o);
+                }
+                float* red_o = reinterpret_cast<float*>(stage0_ptr + (size_t)s * STAGE_BYTES);   // [4 warps][8 heads][D]
+                if (!consumer_sync()) break;                          // every warp has read the last stage
+                if (quad == 0) {
+                    ctl.red_m[warp * 8 + 2 * tq] = m_run[0]; ctl.red_m[warp * 8 + 2 * tq + 1] = m_run[1];
+                    ctl.red_l[warp * 8 + 2 * tq] = l_run[0]; ctl.red_l[warp * 8 + 2 * tq + 1] = l_run[1];
+                }
+                float* wdst = red_o + (size_t)warp * 8 * D;
+#pragma unroll
+                for (int mt = 0; mt < KSTEPS; ++mt) {
+                    const int d0 = mt * 16 + quad;
+                    wdst[(2 * tq) * D + d0] = oacc[mt][0];
+                    wdst[(2 * tq + 1) * D + d0] = oacc[mt][1];
+                    wdst[(2 * tq) * D + d0 + 8] = oacc[mt][2];
+                    wdst[(2 * tq + 1) * D + d0 + 8] = oacc[mt][3];
+                }
+                if (!consumer_sync()) break;
+                for (int u = tid; u < nheads * D; u += CONSUMER_THREADS) {
+                    const int hh = u / D, dd = u % D;
+                    float M = NEG_INF;
+#pragma unroll
+                    for (int w2 = 0; w2 < CONSUMER_WARPS; ++w2) M = fmaxf(M, ctl.red_m[w2 * 8 + hh]);
+                    float accv = 0.f, lsum = 0.f;
+#pragma unroll
+                    for (int w2 = 0; w2 < CONSUMER_WARPS; ++w2) {
+                        const float w = fast_exp2(ctl.red_m[w2 * 8 + hh] - M);     // M is finite: the item has tokens
+                        accv = fmaf(w, red_o[(w2 * 8 + hh) * D + dd], accv);
+                        lsum = fmaf(w, ctl.red_l[w2 * 8 + hh], lsum);
+                    }
+                    const size_t oslot = ((size_t)cur.b * p.Hq + h0 + hh) * p.NC + cur.c;
+                    p.o_part[oslot * D + dd] = accv;
+                    if (dd == 0) { p.m_part[oslot] = M * LN2; p.l_part[oslot] = lsum; }
+                }
+                release(s, true);
             }
         }
     }
+
+    // ---- all roles meet; report a timed-out wait ---------------------------------------------------------
     __syncthreads();
-
-    if (*abort_flag) {
-        if (p.status && tid == 0) atomicMax(p.status, HG_DEV_WAIT_TIMEOUT);
-        if constexpr (MODE != MODE_PROBE) {
-            if (tid < nheads) p.m_part[((size_t)b * p.Hq + h0 + tid) * p.NC + c] = __int_as_float(0x7fc00000);
-        }
-        return;
-    }
-
-    if constexpr (MODE == MODE_PROBE) {
-        if (tid == 0) p.sink[((size_t)b * p.Hkv + g) * p.NC + c] = ctl.probe_acc;
-    } else {
-        constexpr int NSRC = (MODE == MODE_MHA) ? 16 : CONSUMER_WARPS;       // states to merge per head
-        constexpr int HSTRIDE = (MODE == MODE_MHA) ? 0 : D;                  // red_o: [src][head][D]
-        constexpr int SSTRIDE = (MODE == MODE_MHA) ? D : 8 * D;
-        constexpr float LN2 = 0.6931471805599453f;
-        for (int i = tid; i < nheads * D; i += THREADS) {
-            const int hh = i / D, d = i % D;
-            float M = NEG_INF;
-#pragma unroll
-            for (int sidx = 0; sidx < NSRC; ++sidx) M = fmaxf(M, ctl.red_m[(MODE == MODE_MHA) ? sidx : sidx * 8 + hh]);
-            float accv = 0.f, lsum = 0.f;
-#pragma unroll
-            for (int sidx = 0; sidx < NSRC; ++sidx) {
-                const int mi = (MODE == MODE_MHA) ? sidx : sidx * 8 + hh;
-                const float w = fast_exp2(ctl.red_m[mi] - M);      // -inf states weigh 0; M is finite here
-                accv = fmaf(w, red_o[sidx * SSTRIDE + hh * HSTRIDE + d], accv);
-                lsum = fmaf(w, ctl.red_l[mi], lsum);
-            }
-            const size_t slot = ((size_t)b * p.Hq + h0 + hh) * p.NC + c;
-            p.o_part[slot * D + d] = accv;
-            if (d == 0) { p.m_part[slot] = M * LN2; p.l_part[slot] = lsum; }
-        }
-    }
+    if (*abort_flag && p.status && tid == 0) atomicMax(p.status, HG_DEV_WAIT_TIMEOUT);
 }
 
 }  // namespace hg

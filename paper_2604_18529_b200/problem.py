@@ -24,6 +24,7 @@ class DeviceProblem:
         self.tok_begin = torch.tensor(w.tok_begin, dtype=torch.int32, device=dev)
         self.tok_end = torch.tensor(w.tok_end, dtype=torch.int32, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.sched = torch.zeros(1, dtype=torch.int32, device=dev)
         self.NC = w.num_chunks
         self.desc = self.make_desc(w.chunk_tokens, self.NC)
         B, Hq, D, NC = w.B, w.Hq, w.D, self.NC
@@ -39,7 +40,7 @@ class DeviceProblem:
                             page_size=w.page_size, num_pages=kv["num_pages"], page_stride=kv["page_stride"],
                             head_stride=kv["head_stride"], tok_stride=kv["tok_stride"], block_table=kv["block_table"],
                             max_pages=kv["max_pages"], chunk_tokens=chunk_tokens, num_chunks=num_chunks, scale=scale,
-                            status=self.status)
+                            status=self.status, sched_counter=self.sched)
 
     def partial(self, stream=None):
         hg.hg_attn_partial(self.q, self.kv["k"], self.kv["v"], self.seq_lens, self.tok_begin, self.tok_end,

@@ -46,7 +46,8 @@ def test_desc_struct_matches_the_c_layout():
     # offsets follow natural C alignment of the header's field order
     f = {n: getattr(hg.HgAttnDesc, n).offset for n, _ in hg.HgAttnDesc._fields_}
     assert f["struct_size"] == 0 and f["num_pages"] == 28 and f["page_stride"] == 32 and f["block_table"] == 56
-    assert f["max_pages"] == 64 and f["flags"] == 80 and f["status"] == 88 and C.sizeof(hg.HgAttnDesc) == 96
+    assert f["max_pages"] == 64 and f["flags"] == 80 and f["status"] == 88 and f["sched_counter"] == 96
+    assert C.sizeof(hg.HgAttnDesc) == 104
     assert C.sizeof(hg.HgPartialSrc) == 32
 
 
@@ -116,6 +117,15 @@ def test_merge_and_decode_reject_bad_arguments(lib):
     assert lib.hg_attn_decode(*args, FAKE + 16, 1 << 30, None, C.byref(d)) == hg.HG_ERR_INVALID_ARG
     assert lib.hg_attn_decode(*args, FAKE, 1024, None, C.byref(d)) == hg.HG_ERR_WORKSPACE
     assert lib.hg_attn_decode_host(*args, FAKE, 1024, None, C.byref(d)) == hg.HG_ERR_WORKSPACE
+
+
+def test_shorter_struct_without_the_trailing_field_is_accepted(lib):
+    d = good_desc()
+    d.struct_size = 96                       # a caller compiled before sched_counter existed
+    d.sched_counter = 0x3                    # garbage behind the declared size must be ignored
+    assert call_partial(lib, d, q=None) == hg.HG_ERR_INVALID_ARG      # gets as far as the pointer checks
+    d.struct_size = 104
+    assert call_partial(lib, d) == hg.HG_ERR_INVALID_ARG              # now the misaligned counter is seen
 
 
 def test_workspace_bytes(lib):
