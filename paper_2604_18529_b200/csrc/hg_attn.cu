@@ -115,7 +115,7 @@ static int env_int(const char* name, int dflt, int lo, int hi) {
 
 template <int D, bool BF16, int MODE>
 static hg_status launch_partial_t(const CUtensorMap& tk, const CUtensorMap& tv, PartialParams p, cudaStream_t st) {
-    const size_t smem = (size_t)p.stages * 2 * TILE_T * D * 2 + 1024;     // K + V tile per stage
+    const size_t smem = (size_t)p.stages * (2 * TILE_T * D * 2 + 8 * D * 2) + 1024;     // per stage: K tile, V tile, q rows
     auto kern = partial_kernel<D, BF16, MODE>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
         cudaGetLastError();
@@ -211,15 +211,19 @@ static hg_status run_merge(const hg_partial_src* src, int32_t n_src, float* out,
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3((unsigned)(d->batch * d->num_q_heads));
-    cfg.blockDim = dim3(MERGE_THREADS);
+    const bool wide = p.total > 64;                              // long rows: 32 warps per row
+    cfg.blockDim = dim3(wide ? 1024 : 256);
     cfg.stream = static_cast<cudaStream_t>(stream);
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;     // start while the producer of the partials drains
     cfg.attrs = attr;
     cfg.numAttrs = env_int("HG_ATTN_PDL", 1, 0, 1);
-    cudaError_t e = d->head_dim == 128 ? cudaLaunchKernelEx(&cfg, merge_kernel<128>, p)
-                                       : cudaLaunchKernelEx(&cfg, merge_kernel<64>, p);
+    cudaError_t e;
+    if (d->head_dim == 128)
+        e = wide ? cudaLaunchKernelEx(&cfg, merge_kernel<128, 1024>, p) : cudaLaunchKernelEx(&cfg, merge_kernel<128, 256>, p);
+    else
+        e = wide ? cudaLaunchKernelEx(&cfg, merge_kernel<64, 1024>, p) : cudaLaunchKernelEx(&cfg, merge_kernel<64, 256>, p);
     if (e != cudaSuccess) { cudaGetLastError(); return HG_ERR_CUDA; }
     return HG_OK;
 }

@@ -68,8 +68,8 @@ struct Control {
     int2 sdesc[MAX_STAGES];              // what a filled stage holds: x = item index (-1: no more work), y = tile in item
     int abort_flag;
     int pages[MAX_CHUNK_PAGES];          // persistent schedule: two buffers, at 0 and at MAX_CHUNK_PAGES / 2
-    float red_m[32];
-    float red_l[32];
+    float red_m[2][32];                  // per-warp running maxima / exp-sums of an item, double-buffered by item parity
+    float red_l[2][32];
     int cum[PERSIST_MAX_BATCH + 1];      // cum[b] = number of items of sequences < b
     int tb[PERSIST_MAX_BATCH];           // clamped slice of every sequence
     int te[PERSIST_MAX_BATCH];
@@ -129,7 +129,8 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                                                           const PartialParams p) {
     constexpr int HALVES = D / 64;
     constexpr int TILE_BYTES = TILE_T * D * 2;
-    constexpr int STAGE_BYTES = 2 * TILE_BYTES;   // K tile, then V tile
+    constexpr int Q_BYTES = 8 * D * 2;            // the item's query rows (up to 8 heads), present in an item's first stage
+    constexpr int STAGE_BYTES = 2 * TILE_BYTES + Q_BYTES;   // K tile, V tile, q
     constexpr int NV = 8 * HALVES;     // MHA: d-components owned by a lane
     constexpr int KSTEPS = D / 16;     // GQA: 16-wide steps along d
     constexpr float LN2 = 0.6931471805599453f;
@@ -336,6 +337,8 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 }
             }
             const int g = cur.y / p.head_blocks;
+            const int q_heads = (MODE == MODE_GQA) ? min(8, p.G - (cur.y % p.head_blocks) * 8) : 1;
+            const int q_head0 = (MODE == MODE_GQA) ? g * p.G + (cur.y % p.head_blocks) * 8 : g;
             for (int it = 0; it < cur.ntiles; ++it) {              // one stage = K tile + V tile of 64 tokens
                 int okw = 1;
                 if (lane == 0) okw = mbar_wait(&ctl.empty[s], ph ^ 1u, abort_flag) ? 1 : 0;
@@ -345,11 +348,15 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 int phys = -1;
                 if (isv < 2 && t0j < cur.hi && t0j + R > cur.lo) phys = pages[(t0j >> p.page_shift) - page0];
                 const uint32_t nvalid = __popc(__ballot_sync(0xffffffffu, phys >= 0));   // K and V boxes
+                const uint32_t qbytes = (MODE != MODE_PROBE && it == 0) ? (uint32_t)q_heads * D * 2u : 0u;
                 if (lane == 0) {
                     ctl.sdesc[s] = make_int2(i_cur, it);
-                    mbar_arrive_expect_tx(&ctl.full[s], nvalid * box_bytes);
+                    mbar_arrive_expect_tx(&ctl.full[s], nvalid * box_bytes + qbytes);
                 }
                 __syncwarp();
+                if (qbytes && lane == 31)        // the item's query rows travel with its first stage
+                    bulk_load(stage0_ptr + (size_t)s * STAGE_BYTES + 2 * TILE_BYTES,
+                              reinterpret_cast<const uint16_t*>(p.q) + ((size_t)cur.b * p.Hq + q_head0) * D, qbytes, &ctl.full[s]);
                 if (phys >= 0) {
                     uint8_t* dst = stage0_ptr + (size_t)s * STAGE_BYTES + isv * TILE_BYTES + j * box_bytes;
                     tma_load_5d(dst, isv ? &tmV : &tmK, &ctl.full[s], 0, t0j & (p.page_size - 1), 0, g, phys, policy);
@@ -406,6 +413,12 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
             __syncwarp();
             if (lane == 0) mbar_arrive(&ctl.empty[s]);
         };
+        // Scratch of the item epilogue: consumer warp w2 parks its state in the memory of its own 16 K rows of
+        // the item's last stage (nobody else reads those rows): 2 KB per 64-element column half.
+        auto warp_scratch = [&](int s, int w2, int float_idx) -> float* {
+            return reinterpret_cast<float*>(stage0_ptr + (size_t)s * STAGE_BYTES + row_off(16 * w2) +
+                                            (uint32_t)(float_idx >> 9) * half_stride) + (float_idx & 511);
+        };
         // Waits for the next filled stage; returns its ring position, or -1 when there is no more work (or the
         // CTA is unwinding).  d receives the stage's descriptor.
         auto next_stage = [&](int2& d) -> int {
@@ -418,9 +431,10 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
 
         Item cur;
         cur.b = cur.y = cur.c = cur.lo = cur.hi = cur.tile0 = cur.ntiles = 0;
-        int hb = 0, nheads = 1, h0 = 0;
+        int hb = 0, nheads = 1, h0 = 0, par = 1;
         auto begin_item = [&](int i) {
             cur = get_item(i);
+            par ^= 1;
             hb = cur.y % p.head_blocks;
             const int g = cur.y / p.head_blocks;
             nheads = (MODE == MODE_GQA) ? min(8, p.G - hb * 8) : 1;
@@ -451,12 +465,13 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 // item epilogue, with the item's last stage as scratch
 #pragma unroll
                 for (int o = 16; o; o >>= 1) probe_x ^= __shfl_xor_sync(0xffffffffu, probe_x, o);
-                uint32_t* red = reinterpret_cast<uint32_t*>(stage0_ptr + (size_t)s * STAGE_BYTES);
-                if (!consumer_sync()) break;                      // every warp has read the last stage
-                if (lane == 0) red[warp] = probe_x;
+                if (lane == 0) ctl.red_l[par][warp] = __uint_as_float(probe_x);
                 if (!consumer_sync()) break;
-                if (tid == 0) p.sink[((size_t)cur.b * p.Hkv + cur.y) * p.NC + cur.c] = red[0] ^ red[1] ^ red[2] ^ red[3];
-                release(s, true);
+                if (tid == 0)
+                    p.sink[((size_t)cur.b * p.Hkv + cur.y) * p.NC + cur.c] =
+                        __float_as_uint(ctl.red_l[par][0]) ^ __float_as_uint(ctl.red_l[par][1]) ^
+                        __float_as_uint(ctl.red_l[par][2]) ^ __float_as_uint(ctl.red_l[par][3]);
+                release(s, false);
             }
         } else if constexpr (MODE == MODE_MHA) {
             // ----------------------- MHA (CUDA cores) -----------------------
@@ -472,10 +487,10 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 if (s < 0) break;
                 if (d.y == 0) {
                     begin_item(d.x);
-                    const uint16_t* qrow = reinterpret_cast<const uint16_t*>(p.q) + ((size_t)cur.b * p.Hq + h0) * D;
+                    const uint32_t qs = stage0 + s * STAGE_BYTES + 2 * TILE_BYTES;
 #pragma unroll
                     for (int hh = 0; hh < HALVES; ++hh) {
-                        uint4 raw = *reinterpret_cast<const uint4*>(qrow + hh * 64 + li * 8);
+                        uint4 raw = lds128(qs + hh * 128 + li * 16);
                         float2 a = unpack2<BF16>(raw.x), bb = unpack2<BF16>(raw.y), cc = unpack2<BF16>(raw.z),
                                dd = unpack2<BF16>(raw.w);
                         qf[hh * 8 + 0] = a.x; qf[hh * 8 + 1] = a.y; qf[hh * 8 + 2] = bb.x; qf[hh * 8 + 3] = bb.y;
@@ -546,14 +561,12 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 }
                 if (d.y + 1 < cur.ntiles) { release(s, false); continue; }
 
-                // ---- item epilogue: merge the 16 row-group states (the item's last stage is the scratch) ----
-                float* red_o = reinterpret_cast<float*>(stage0_ptr + (size_t)s * STAGE_BYTES);   // [16 row groups][D]
-                if (!consumer_sync()) break;                      // every warp has read the last stage
+                // ---- item epilogue: merge the 16 row-group states (parked in the item's last stage) ----
                 const int slot = warp * 4 + gi;
-                if (li == 0) { ctl.red_m[slot] = m_run; ctl.red_l[slot] = l_run; }
+                if (li == 0) { ctl.red_m[par][slot] = m_run; ctl.red_l[par][slot] = l_run; }
 #pragma unroll
                 for (int hh = 0; hh < HALVES; ++hh) {
-                    float4* dst = reinterpret_cast<float4*>(red_o + slot * D + hh * 64 + li * 8);
+                    float4* dst = reinterpret_cast<float4*>(warp_scratch(s, warp, gi * D + hh * 64 + li * 8));
                     dst[0] = make_float4(o[hh * 8 + 0], o[hh * 8 + 1], o[hh * 8 + 2], o[hh * 8 + 3]);
                     dst[1] = make_float4(o[hh * 8 + 4], o[hh * 8 + 5], o[hh * 8 + 6], o[hh * 8 + 7]);
                 }
@@ -561,13 +574,13 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 if (tid < D) {
                     float M = NEG_INF;
 #pragma unroll
-                    for (int sidx = 0; sidx < 16; ++sidx) M = fmaxf(M, ctl.red_m[sidx]);
+                    for (int sidx = 0; sidx < 16; ++sidx) M = fmaxf(M, ctl.red_m[par][sidx]);
                     float accv = 0.f, lsum = 0.f;
 #pragma unroll
                     for (int sidx = 0; sidx < 16; ++sidx) {
-                        const float w = fast_exp2(ctl.red_m[sidx] - M);      // -inf states weigh 0; M is finite
-                        accv = fmaf(w, red_o[sidx * D + tid], accv);
-                        lsum = fmaf(w, ctl.red_l[sidx], lsum);
+                        const float w = fast_exp2(ctl.red_m[par][sidx] - M);      // -inf states weigh 0; M is finite
+                        accv = fmaf(w, *warp_scratch(s, sidx >> 2, (sidx & 3) * D + tid), accv);
+                        lsum = fmaf(w, ctl.red_l[par][sidx], lsum);
                     }
                     const size_t oslot = ((size_t)cur.b * p.Hq + h0) * p.NC + cur.c;
                     p.o_part[oslot * D + tid] = accv;
@@ -594,12 +607,11 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                     begin_item(d.x);
                     // b0 = q[head quad][16 ks + 2 tq + {0,1}], b1 = the same + 8; heads past the group read as zero
                     const bool live = hb * 8 + quad < p.G;
-                    const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
-                        reinterpret_cast<const uint16_t*>(p.q) + ((size_t)cur.b * p.Hq + (live ? h0 + quad : h0)) * D);
+                    const uint32_t qs = stage0 + s * STAGE_BYTES + 2 * TILE_BYTES + quad * (D * 2);
 #pragma unroll
                     for (int ks = 0; ks < KSTEPS; ++ks) {
-                        qb[ks][0] = live ? qrow[ks * 8 + tq] : 0u;
-                        qb[ks][1] = live ? qrow[ks * 8 + 4 + tq] : 0u;
+                        qb[ks][0] = live ? lds32(qs + (ks * 8 + tq) * 4) : 0u;
+                        qb[ks][1] = live ? lds32(qs + (ks * 8 + 4 + tq) * 4) : 0u;
                     }
                     m_run[0] = m_run[1] = NEG_INF; l_run[0] = l_run[1] = 0.f;
 #pragma unroll
@@ -678,33 +690,30 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                     l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], o);
                     l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], o);
                 }
-                float* red_o = reinterpret_cast<float*>(stage0_ptr + (size_t)s * STAGE_BYTES);   // [4 warps][8 heads][D]
-                if (!consumer_sync()) break;                          // every warp has read the last stage
                 if (quad == 0) {
-                    ctl.red_m[warp * 8 + 2 * tq] = m_run[0]; ctl.red_m[warp * 8 + 2 * tq + 1] = m_run[1];
-                    ctl.red_l[warp * 8 + 2 * tq] = l_run[0]; ctl.red_l[warp * 8 + 2 * tq + 1] = l_run[1];
+                    ctl.red_m[par][warp * 8 + 2 * tq] = m_run[0]; ctl.red_m[par][warp * 8 + 2 * tq + 1] = m_run[1];
+                    ctl.red_l[par][warp * 8 + 2 * tq] = l_run[0]; ctl.red_l[par][warp * 8 + 2 * tq + 1] = l_run[1];
                 }
-                float* wdst = red_o + (size_t)warp * 8 * D;
 #pragma unroll
-                for (int mt = 0; mt < KSTEPS; ++mt) {
+                for (int mt = 0; mt < KSTEPS; ++mt) {               // this warp's [8 heads][D] into its own rows
                     const int d0 = mt * 16 + quad;
-                    wdst[(2 * tq) * D + d0] = oacc[mt][0];
-                    wdst[(2 * tq + 1) * D + d0] = oacc[mt][1];
-                    wdst[(2 * tq) * D + d0 + 8] = oacc[mt][2];
-                    wdst[(2 * tq + 1) * D + d0 + 8] = oacc[mt][3];
+                    *warp_scratch(s, warp, (2 * tq) * D + d0) = oacc[mt][0];
+                    *warp_scratch(s, warp, (2 * tq + 1) * D + d0) = oacc[mt][1];
+                    *warp_scratch(s, warp, (2 * tq) * D + d0 + 8) = oacc[mt][2];
+                    *warp_scratch(s, warp, (2 * tq + 1) * D + d0 + 8) = oacc[mt][3];
                 }
                 if (!consumer_sync()) break;
                 for (int u = tid; u < nheads * D; u += CONSUMER_THREADS) {
                     const int hh = u / D, dd = u % D;
                     float M = NEG_INF;
 #pragma unroll
-                    for (int w2 = 0; w2 < CONSUMER_WARPS; ++w2) M = fmaxf(M, ctl.red_m[w2 * 8 + hh]);
+                    for (int w2 = 0; w2 < CONSUMER_WARPS; ++w2) M = fmaxf(M, ctl.red_m[par][w2 * 8 + hh]);
                     float accv = 0.f, lsum = 0.f;
 #pragma unroll
                     for (int w2 = 0; w2 < CONSUMER_WARPS; ++w2) {
-                        const float w = fast_exp2(ctl.red_m[w2 * 8 + hh] - M);     // M is finite: the item has tokens
-                        accv = fmaf(w, red_o[(w2 * 8 + hh) * D + dd], accv);
-                        lsum = fmaf(w, ctl.red_l[w2 * 8 + hh], lsum);
+                        const float w = fast_exp2(ctl.red_m[par][w2 * 8 + hh] - M);     // M is finite: the item has tokens
+                        accv = fmaf(w, *warp_scratch(s, w2, u), accv);
+                        lsum = fmaf(w, ctl.red_l[par][w2 * 8 + hh], lsum);
                     }
                     const size_t oslot = ((size_t)cur.b * p.Hq + h0 + hh) * p.NC + cur.c;
                     p.o_part[oslot * D + dd] = accv;
