@@ -29,8 +29,10 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the partial kernel, from the ncu
 # captures summarised under profiles/ (None until a capture of that workload exists)
 NCU_TRAFFIC_BYTES = {
-    # profiles/partial_kernel_opt13b.md: one sequence captured (402.77 MB read + 4.28 MB written), x 8 sequences
-    "opt13b": 8 * (402_771_456 + 4_281_600),
+    # profiles/partial_kernel_opt13b.md: two sequences captured (805.54 MB read + 4.74 MB written), x 4
+    "opt13b": 4 * (805_537_024 + 4_742_400),
+    # profiles/partial_kernel_llama70b.md: the full launch captured
+    "llama70b": 1_718_222_000 + 6_867_968,
 }
 
 

@@ -55,6 +55,9 @@ typedef enum hg_dtype { HG_DTYPE_F16 = 0, HG_DTYPE_BF16 = 1 } hg_dtype;
 
 /* bits of hg_attn_desc.flags */
 #define HG_FLAG_NONE 0u
+#define HG_FLAG_TEST_STALL 1u /* testing aid: the loader of hg_attn_partial / hg_kv_read_probe never fills a
+                                 stage, so every wait runs into its time limit (about 2 s); the call then
+                                 reports HG_DEV_WAIT_TIMEOUT through *status and returns normally */
 
 /* values the kernels may write to *hg_attn_desc.status (device word, optional) */
 #define HG_DEV_OK 0

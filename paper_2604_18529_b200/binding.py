@@ -21,6 +21,7 @@ HG_OK, HG_ERR_INVALID_ARG, HG_ERR_UNSUPPORTED, HG_ERR_CUDA, HG_ERR_WORKSPACE = 0
 HG_DTYPE_F16, HG_DTYPE_BF16 = 0, 1
 HG_DEV_OK, HG_DEV_WAIT_TIMEOUT, HG_DEV_BAD_PAGE = 0, 1, 2
 HG_MAX_MERGE_SRC = 8
+HG_FLAG_TEST_STALL = 1
 HG_STATIC_SCRATCH_BYTES = 8 << 20
 
 

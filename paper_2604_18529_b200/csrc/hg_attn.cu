@@ -179,6 +179,7 @@ static hg_status run_partial(int mode, const void* q, const void* k, const void*
     // persistent schedule unless the batch or the chunk's page list exceeds what the kernel keeps in shared memory
     p.persistent = (d->batch <= PERSIST_MAX_BATCH && d->chunk_tokens / d->page_size <= PERSIST_CHUNK_PAGES)
                        ? env_int("HG_ATTN_PERSISTENT", 1, 0, 1) : 0;
+    p.test_stall = (d->flags & HG_FLAG_TEST_STALL) ? 1 : 0;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     p.sched = p.persistent && env_int("HG_ATTN_DYNAMIC", 1, 0, 1) ? desc_sched(d) : nullptr;
     if (p.sched && cudaMemsetAsync(p.sched, 0, sizeof(int32_t), cs) != cudaSuccess) {

@@ -57,6 +57,7 @@ struct PartialParams {
     int page_size, page_shift, max_pages, num_pages;
     int C, NC, stages, head_blocks;
     int persistent;
+    int test_stall;           // HG_FLAG_TEST_STALL: the producer never fills a stage
     int32_t* sched;           // zeroed work counter: items are handed out dynamically (NULL: round-robin)
     float scale_log2;         // logit scale * log2(e)
 };
@@ -306,7 +307,7 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
         int s = 0, issued = 0, k = 0;                // ring position, stages armed so far, items taken so far
         uint32_t ph = 0;
         bool alive = true;
-        int i_cur = settle(request(0));
+        int i_cur = p.test_stall ? n_items : settle(request(0));
         int raw_nxt = request(1);
         Item cur;
         if (i_cur < n_items) {                       // page ids of the first item
@@ -376,7 +377,7 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
             i_cur = i_nxt;
             ++k;
         }
-        if (alive) {
+        if (alive && !p.test_stall) {
             // no more work: one last, empty stage tells the consumers
             int okw = 1;
             if (lane == 0) okw = mbar_wait(&ctl.empty[s], ph ^ 1u, abort_flag) ? 1 : 0;

@@ -245,3 +245,86 @@ def test_bad_page_id_is_reported_not_dereferenced():
     prob.partial()
     torch.cuda.synchronize()
     assert int(prob.status.item()) == hg.HG_DEV_BAD_PAGE
+
+
+# ---- schedules: persistent-dynamic, persistent-static and one-CTA-per-item give the same bits --------------------
+
+@pytest.mark.parametrize("G", [1, 4])
+def test_result_does_not_depend_on_the_schedule(G, monkeypatch):
+    w = wl(B=3, Hq=2 * G, Hkv=2, seq_lens=[2100, 900, 333], tok_begin=[400, 100, 333], tok_end=[2100, 900, 333],
+           chunk_tokens=128)
+    ref = OracleRef(w)
+    results = []
+    for env in ({}, {"HG_ATTN_DYNAMIC": "0"}, {"HG_ATTN_PERSISTENT": "0"}, {"HG_ATTN_STAGES": "2"},
+                {"HG_ATTN_CTAS_PER_SM": "1", "HG_ATTN_STAGES": "5"}):
+        for k in ("HG_ATTN_DYNAMIC", "HG_ATTN_PERSISTENT", "HG_ATTN_STAGES", "HG_ATTN_CTAS_PER_SM"):
+            monkeypatch.delenv(k, raising=False)
+        for k, v in env.items():
+            monkeypatch.setenv(k, v)
+        prob = DeviceProblem(w, DEV)
+        prob.step(ref.host_partials_device(DEV))
+        torch.cuda.synchronize()
+        assert int(prob.status.item()) == hg.HG_DEV_OK
+        check_output(prob.out, prob.lse, ref.out, ref.lse, str(env))
+        results.append((prob.o_part.clone(), prob.m_part.clone(), prob.l_part.clone(), prob.out.clone()))
+    for r in results[1:]:
+        for a, b in zip(results[0], r):
+            assert torch.equal(a, b)
+
+
+def test_without_a_work_counter_items_are_dealt_round_robin():
+    w = wl(Hq=8, Hkv=2)
+    ref = OracleRef(w)
+    prob = DeviceProblem(w, DEV)
+    prob.sched = None
+    prob.desc = prob.make_desc(w.chunk_tokens, prob.NC)
+    assert not prob.desc.sched_counter
+    prob.step(ref.host_partials_device(DEV))
+    torch.cuda.synchronize()
+    check_output(prob.out, prob.lse, ref.out, ref.lse)
+
+
+# ---- shapes beyond what the persistent schedule keeps in shared memory fall back to one CTA per item ------------
+
+def test_large_batch_uses_the_per_item_grid():
+    B = 530                                              # more sequences than the in-kernel item scan handles
+    lens = [40 + (7 * i) % 150 for i in range(B)]
+    tb = [(3 * i) % 30 for i in range(B)]
+    w = wl(B=B, Hq=2, Hkv=1, D=64, seq_lens=lens, tok_begin=tb, tok_end=lens, chunk_tokens=64, seed=77)
+    run_and_check(w)
+
+
+def test_chunks_with_many_pages_use_the_per_item_grid():
+    # 8192-token chunks of 16-token pages: 512 page ids per chunk, beyond the double-buffered page list
+    w = wl(B=1, Hq=4, Hkv=1, seq_lens=[9000], tok_begin=[100], tok_end=[9000], chunk_tokens=8192, seed=78)
+    run_and_check(w)
+
+
+# ---- bounded waits: a stalled pipeline ends with a status code, not a hang -----------------------------------------
+
+@pytest.mark.parametrize("G", [1, 4])
+def test_stalled_loader_times_out_with_a_status_and_the_context_stays_usable(G):
+    import time
+    w = wl(B=1, Hq=2 * G, Hkv=2, seq_lens=[300], tok_begin=[0], tok_end=[300])
+    ref = OracleRef(w)
+    prob = DeviceProblem(w, DEV)
+    prob.desc.flags = hg.HG_FLAG_TEST_STALL          # nothing ever fills a stage: every consumer wait must run out
+    torch.cuda.synchronize()
+    t0 = time.time()
+    prob.partial()
+    torch.cuda.synchronize()
+    dt = time.time() - t0
+    assert int(prob.status.item()) == hg.HG_DEV_WAIT_TIMEOUT
+    assert 1.0 < dt < 30.0
+    # while the word is set, later launches return at once instead of queueing behind a broken pipeline
+    prob.desc.flags = 0
+    t0 = time.time()
+    prob.partial()
+    torch.cuda.synchronize()
+    assert time.time() - t0 < 1.0 and int(prob.status.item()) == hg.HG_DEV_WAIT_TIMEOUT
+    # cleared: the same context computes correct results again
+    prob.status.zero_()
+    prob.step(ref.host_partials_device(DEV))
+    torch.cuda.synchronize()
+    assert int(prob.status.item()) == hg.HG_DEV_OK
+    check_output(prob.out, prob.lse, ref.out, ref.lse)
