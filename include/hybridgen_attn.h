@@ -220,6 +220,41 @@ hg_status hg_attn_decode_static(const void* q, const void* k_cache, const void* 
                                 void* stream, const hg_attn_desc* desc);
 
 /*
+ * Problem description of hg_attn_partial_from_logits (host struct).
+ */
+typedef struct hg_logits_desc {
+    uint32_t struct_size;  /* sizeof(hg_logits_desc) */
+    int32_t batch;         /* B */
+    int32_t num_q_heads;   /* Hq, a multiple of num_kv_heads */
+    int32_t num_kv_heads;  /* Hkv */
+    int32_t head_dim;      /* D in {64, 128} */
+    int32_t dtype;         /* hg_dtype of the V rows */
+    int32_t max_selected;  /* K: row length of logits / v_rows (selected-token slots per sequence) */
+    int32_t chunk_tokens;  /* slots per partial, a multiple of 32, at most 1024 */
+    int32_t num_chunks;    /* NC >= ceil(K / chunk_tokens): partials per (sequence, head) */
+} hg_logits_desc;
+
+/*
+ * Softmax partials from host-computed logits and the matching V rows: the device side of the paper's
+ * hand-off (Section 4.2, CPU-side support: the host's Logits Calculator sends the logits of its
+ * selected tokens, "a compact vector", and the corresponding V vectors; workflow steps 2, 3 and 5).
+ * The result plugs into hg_attn_merge as one more source, which stands for concatenating host and
+ * device logits and V rows and taking one softmax over them.
+ *
+ *   logits   dev float [B][Hq][K]      scaled logits s = q.k / sqrt(D) of the selected tokens, natural units;
+ *                                      a slot holding -inf is ignored (its V row is never used)
+ *   v_rows   dev 16-bit [B][Hkv][K][D] V rows of those tokens, slot for slot; the query heads of a group share
+ *                                      their KV head's rows; 16-byte aligned
+ *   n_sel    dev int32 [B]             slots in use per sequence (clamped to [0, K])
+ *   o_part, m_part, l_part             dev float [B][Hq][NC][D] / [B][Hq][NC]: chunk c covers slots
+ *                                      [c * chunk_tokens, (c+1) * chunk_tokens) below n_sel; empty chunks are
+ *                                      (m, l, o) = (-inf, 0, 0)
+ * Token order and token indices do not matter for the result and are not passed.
+ */
+hg_status hg_attn_partial_from_logits(const float* logits, const void* v_rows, const int32_t* n_sel, float* o_part,
+                                      float* m_part, float* l_part, void* stream, const hg_logits_desc* desc);
+
+/*
  * Evidence kernel, not part of the attention path: streams the same K and V tiles through the
  * same TMA pipeline as hg_attn_partial and folds them into one 32-bit checksum per work item
  * (sink: dev uint32 [B][Hkv][NC]).  Used to measure the read ceiling of the paged access pattern.

@@ -15,6 +15,8 @@
  *   MERGE       log-sum-exp combination of partials over disjoint token sets; by Section 4.2's
  *               exactness claim (outputs identical to monolithic execution) it must equal
  *               FULL of the union
+ *   PARTIAL from logits  the same triple from host-computed logits and gathered V rows (the device side of
+ *               the paper's hand-off)
  *   LITERAL     the paper's own hand-off (Section 4.2 / workflow steps 2-5): each device computes
  *               raw logits for its own tokens, the logits and V rows are concatenated and put
  *               back in original token order, one softmax, one value aggregation
@@ -98,6 +100,26 @@ void hgo_partial(const uint16_t* q, const uint16_t* K, const uint16_t* V, int64_
         for (int d = 0; d < D; ++d) o[d] += p * dec(row[d], dtype);
     }
     free(s);
+    *m_out = m; *l_out = l;
+}
+
+/* ---- PARTIAL from given logits: the device side of the paper's hand-off (Section 4.2, CPU-side support /
+ *      workflow steps 2-5): the host ships the logits s_i of n selected tokens and their V rows
+ *      Vsel[i] (row i at Vsel + i * row_stride); the result is the same (m, l, o) a PARTIAL over those
+ *      tokens gives.  Logits of -inf mark unselected slots; all -inf (or n = 0) is the empty partial. */
+void hgo_partial_from_logits(const double* s, const uint16_t* Vsel, int64_t row_stride, int D, int dtype, int64_t n,
+                             double* m_out, double* l_out, double* o) {
+    for (int d = 0; d < D; ++d) o[d] = 0.0;
+    double m = -INFINITY;
+    for (int64_t i = 0; i < n; ++i) if (s[i] > m) m = s[i];
+    if (m == -INFINITY) { *m_out = -INFINITY; *l_out = 0.0; return; }
+    double l = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        if (s[i] == -INFINITY) continue;
+        double p = exp(s[i] - m);
+        l += p;
+        for (int d = 0; d < D; ++d) o[d] += p * dec(Vsel[i * row_stride + d], dtype);
+    }
     *m_out = m; *l_out = l;
 }
 

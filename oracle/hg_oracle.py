@@ -51,6 +51,8 @@ def lib():
             L.hgo_decode.argtypes = [_p, _i64, _int, _p]
             L.hgo_logits.argtypes = [_p, _p, _i64, _int, _int, _dbl, _p, _i64, _i64, _p]
             L.hgo_partial.argtypes = [_p, _p, _p, _i64, _int, _int, _dbl, _p, _i64, _i64, _p, _p, _p]
+            L.hgo_partial_from_logits.argtypes = [_p, _p, _i64, _int, _int, _i64, _p, _p, _p]
+            L.hgo_partial_from_logits.restype = None
             L.hgo_full.argtypes = [_p, _p, _p, _i64, _int, _int, _dbl, _p, _i64, _i64, _p, _p]
             L.hgo_merge.argtypes = [_i64, _p, _p, _p, _int, _p, _p]
             L.hgo_literal.argtypes = [_p, _p, _p, _i64, _int, _int, _dbl, _p, _i64, _p, _i64, _p, _p]
@@ -119,6 +121,16 @@ def partial(q, K, V, dtype: str, scale: float = 0.0, idx=None, t0: int = 0, n: i
     D = q.shape[-1]
     m, l, o = _dbl(), _dbl(), np.empty(D, dtype=np.float64)
     lib().hgo_partial(_ptr(q), _ptr(K), _ptr(V), ts, D, DTYPES[dtype], scale, ip, t0, n, C.byref(m), C.byref(l), _ptr(o))
+    return m.value, l.value, o
+
+
+def partial_from_logits(s, Vsel, dtype: str):
+    """PARTIAL from n given logits s[n] (fp64) and the matching V rows Vsel [n][D] -> (m, l, o[D])."""
+    s = np.ascontiguousarray(s, dtype=np.float64)
+    Vsel, rs = _rows(Vsel)
+    D = Vsel.shape[1]
+    m, l, o = _dbl(), _dbl(), np.empty(D, dtype=np.float64)
+    lib().hgo_partial_from_logits(_ptr(s), _ptr(Vsel), rs, D, DTYPES[dtype], len(s), C.byref(m), C.byref(l), _ptr(o))
     return m.value, l.value, o
 
 

@@ -13,6 +13,8 @@ from .binding import (  # noqa: F401
     attn_desc,
     hg_attn_partial,
     hg_attn_merge,
+    hg_attn_partial_from_logits,
+    logits_desc,
     hg_attn_decode,
     hg_attn_decode_host,
     hg_attn_decode_static,

@@ -55,6 +55,20 @@ class HgAttnDesc(C.Structure):
     ]
 
 
+class HgLogitsDesc(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32),
+        ("batch", C.c_int32),
+        ("num_q_heads", C.c_int32),
+        ("num_kv_heads", C.c_int32),
+        ("head_dim", C.c_int32),
+        ("dtype", C.c_int32),
+        ("max_selected", C.c_int32),
+        ("chunk_tokens", C.c_int32),
+        ("num_chunks", C.c_int32),
+    ]
+
+
 class HgPartialSrc(C.Structure):
     _fields_ = [("o", C.c_void_p), ("m", C.c_void_p), ("l", C.c_void_p), ("nc", C.c_int32), ("reserved", C.c_int32)]
 
@@ -85,6 +99,8 @@ def lib():
         L.hg_attn_decode_host.restype = C.c_int
         L.hg_attn_decode_static.argtypes = [vp] * 6 + [C.POINTER(HgPartialSrc), i32, vp, vp, vp, C.POINTER(HgAttnDesc)]
         L.hg_attn_decode_static.restype = C.c_int
+        L.hg_attn_partial_from_logits.argtypes = [vp] * 7 + [C.POINTER(HgLogitsDesc)]
+        L.hg_attn_partial_from_logits.restype = C.c_int
         L.hg_kv_read_probe.argtypes = [vp] * 7 + [C.POINTER(HgAttnDesc)]
         L.hg_kv_read_probe.restype = C.c_int
         L.hg_status_string.argtypes = [C.c_int]
@@ -185,6 +201,26 @@ def hg_attn_partial(q, k_cache, v_cache, seq_lens, tok_begin, tok_end, o_part, m
                                _dev(m_part, "m_part", torch.float32), _dev(l_part, "l_part", torch.float32),
                                _stream(stream), C.byref(desc))
     _check(st, "hg_attn_partial")
+
+
+def logits_desc(*, batch: int, num_q_heads: int, num_kv_heads: int, head_dim: int, dtype, max_selected: int,
+                chunk_tokens: int = 256, num_chunks: int = 0) -> HgLogitsDesc:
+    d = HgLogitsDesc()
+    d.struct_size = C.sizeof(HgLogitsDesc)
+    d.batch, d.num_q_heads, d.num_kv_heads, d.head_dim = batch, num_q_heads, num_kv_heads, head_dim
+    d.dtype = _DTYPES[dtype]
+    d.max_selected, d.chunk_tokens = max_selected, chunk_tokens
+    d.num_chunks = num_chunks or -(-max_selected // chunk_tokens)
+    return d
+
+
+def hg_attn_partial_from_logits(logits, v_rows, n_sel, o_part, m_part, l_part, desc: HgLogitsDesc, stream=None) -> None:
+    """Partials (o, m, l) from host-computed logits [B][Hq][K] (fp32) and the matching V rows [B][Hkv][K][D]."""
+    st = lib().hg_attn_partial_from_logits(_dev(logits, "logits", torch.float32), _dev(v_rows, "v_rows"),
+                                           _dev(n_sel, "n_sel", torch.int32), _dev(o_part, "o_part", torch.float32),
+                                           _dev(m_part, "m_part", torch.float32), _dev(l_part, "l_part", torch.float32),
+                                           _stream(stream), C.byref(desc))
+    _check(st, "hg_attn_partial_from_logits")
 
 
 def hg_attn_merge(partials, out, lse, desc: HgAttnDesc, stream=None) -> None:

@@ -10,7 +10,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libhybridgen_attn.so")
 SOURCES = [os.path.join(CSRC, "hg_attn.cu")]
-DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("hg_device.cuh", "hg_partial.cuh", "hg_merge.cuh")] + [
+DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("hg_device.cuh", "hg_partial.cuh", "hg_merge.cuh", "hg_logits.cuh")] + [
     os.path.join(ROOT, "include", "hybridgen_attn.h")]
 
 

@@ -13,6 +13,7 @@
 
 #include <atomic>
 
+#include "hg_logits.cuh"
 #include "hg_merge.cuh"
 #include "hg_partial.cuh"
 
@@ -283,6 +284,40 @@ hg_status hg_kv_read_probe(const void* k_cache, const void* v_cache, const int32
 hg_status hg_attn_merge(const hg_partial_src* partials, int32_t n_src, float* out, float* lse, void* stream,
                         const hg_attn_desc* desc) {
     return run_merge(partials, n_src, out, lse, stream, desc);
+}
+
+hg_status hg_attn_partial_from_logits(const float* logits, const void* v_rows, const int32_t* n_sel, float* o_part,
+                                      float* m_part, float* l_part, void* stream, const hg_logits_desc* d) {
+    if (!d || d->struct_size < sizeof(hg_logits_desc)) return HG_ERR_INVALID_ARG;
+    if (d->batch < 1 || d->batch > 65535 || d->num_kv_heads < 1 || d->num_kv_heads > 65535 || d->num_q_heads < 1 ||
+        d->num_q_heads % d->num_kv_heads)
+        return HG_ERR_INVALID_ARG;
+    if (d->head_dim <= 0 || d->head_dim % 8) return HG_ERR_INVALID_ARG;
+    if (d->head_dim != 64 && d->head_dim != 128) return HG_ERR_UNSUPPORTED;
+    if (d->dtype != HG_DTYPE_F16 && d->dtype != HG_DTYPE_BF16) return HG_ERR_INVALID_ARG;
+    if (d->max_selected < 1 || d->chunk_tokens < 32 || d->chunk_tokens % 32 || d->num_chunks < 1) return HG_ERR_INVALID_ARG;
+    if (d->chunk_tokens > LG_MAX_CHUNK) return HG_ERR_UNSUPPORTED;
+    if ((int64_t)d->num_chunks * d->chunk_tokens < d->max_selected) return HG_ERR_INVALID_ARG;
+    if (!logits || !v_rows || !n_sel || !o_part || !m_part || !l_part) return HG_ERR_INVALID_ARG;
+    if (!aligned16(v_rows) || !aligned16(o_part)) return HG_ERR_INVALID_ARG;
+    LogitsParams p;
+    p.logits = logits; p.v_rows = v_rows; p.n_sel = n_sel; p.o_part = o_part; p.m_part = m_part; p.l_part = l_part;
+    p.B = d->batch; p.Hq = d->num_q_heads; p.Hkv = d->num_kv_heads; p.G = p.Hq / p.Hkv; p.K = d->max_selected;
+    p.chunk = d->chunk_tokens; p.NC = d->num_chunks;
+    const size_t smem = ((size_t)8 * p.chunk + (size_t)LG_WARPS * 8 * d->head_dim) * sizeof(float);
+    dim3 grid((unsigned)p.NC, (unsigned)p.Hkv, (unsigned)p.B);
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const bool bf16 = d->dtype == HG_DTYPE_BF16;
+    auto launch = [&](auto kern) -> hg_status {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+            cudaGetLastError();
+            return HG_ERR_CUDA;
+        }
+        kern<<<grid, LG_THREADS, smem, cs>>>(p);
+        return cudaGetLastError() == cudaSuccess ? HG_OK : HG_ERR_CUDA;
+    };
+    if (d->head_dim == 128) return bf16 ? launch(logits_partial_kernel<128, true>) : launch(logits_partial_kernel<128, false>);
+    return bf16 ? launch(logits_partial_kernel<64, true>) : launch(logits_partial_kernel<64, false>);
 }
 
 size_t hg_attn_workspace_bytes(const hg_attn_desc* desc, int32_t n_host_partials) {

@@ -1,0 +1,113 @@
+"""The paper's literal CPU -> GPU hand-off on the GPU: the host sends logits of its (selected) tokens and
+their V rows, hg_attn_partial_from_logits turns them into partials, hg_attn_merge combines them with the
+partials of the GPU-resident slice.  Checked against the oracle: chunk partials one by one, and the merged
+result against monolithic attention over exactly the tokens that took part."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2604_18529_b200 as pkg
+from oracle import hg_oracle as O
+from paper_2604_18529_b200 import workload as W
+from paper_2604_18529_b200.problem import DeviceProblem
+from parity_util import LSE_ABS, OUT_MAX_ABS, OUT_REL_L2, bits, check_partials
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def handoff_case(w, keep, chunk, seed=0):
+    """keep: fraction of the host slice the host selects (top logits of the group's first head, per KV head)."""
+    rng = np.random.default_rng(seed)
+    q, K, V = bits(w.q()), bits(w.kv_logical("k")), bits(w.kv_logical("v"))
+    G = w.G
+    n_host = [tb for tb in w.tok_begin]                           # the host holds [0, tok_begin)
+    Ksel = max(1, max(int(np.ceil(keep * n)) for n in n_host))
+    Kpad = Ksel + 5                                               # a few slots that are never used
+    logits = np.full((w.B, w.Hq, Kpad), -np.inf)
+    vrows = np.zeros((w.B, w.Hkv, Kpad, w.D), dtype=np.uint16)
+    vrows[:] = 0x7E00                                             # NaN patterns in unused slots must not matter
+    n_sel = np.zeros(w.B, dtype=np.int32)
+    chosen = {}
+    for b in range(w.B):
+        k = int(np.ceil(keep * n_host[b])) if n_host[b] else 0
+        n_sel[b] = k
+        for g in range(w.Hkv):
+            Kr, Vr = np.ascontiguousarray(K[b, :, g]), np.ascontiguousarray(V[b, :, g])
+            if k == 0:
+                chosen[(b, g)] = np.zeros(0, dtype=np.int64)
+                continue
+            s0 = O.logits(q[b, g * G], Kr, w.dtype, t0=0, n=n_host[b])
+            idx = np.sort(np.argsort(-s0)[:k]) if keep < 1.0 else np.arange(n_host[b])
+            idx = rng.permutation(idx)                            # slot order is arbitrary
+            chosen[(b, g)] = idx
+            vrows[b, g, :k] = Vr[idx]
+            for hh in range(G):
+                logits[b, g * G + hh, :k] = O.logits(q[b, g * G + hh], Kr, w.dtype, idx=idx)
+    if w.B > 1 and n_sel[1] > 3:                                  # head 0 of sequence 1 drops some of its slots
+        logits[1, 0, 1:n_sel[1]:3] = -np.inf
+    return q, K, V, logits, vrows, n_sel, chosen, Kpad
+
+
+@pytest.mark.parametrize("G,D,dtype", [(1, 128, "f16"), (4, 128, "f16"), (8, 64, "bf16"), (12, 128, "bf16")])
+@pytest.mark.parametrize("keep,chunk", [(1.0, 256), (0.25, 64), (0.05, 32)])
+def test_handoff_partials_and_merged_result(G, D, dtype, keep, chunk):
+    w = W.AttnWorkload("handoff", 3, 2 * G, 2, D, dtype, [900, 400, 130], [500, 333, 0], [900, 400, 130],
+                       page_size=16, chunk_tokens=128, seed=41 + G)
+    q, K, V, logits, vrows, n_sel, chosen, Kpad = handoff_case(w, keep, chunk)
+    NCs = -(-Kpad // chunk)
+    desc = pkg.logits_desc(batch=w.B, num_q_heads=w.Hq, num_kv_heads=w.Hkv, head_dim=D, dtype=dtype,
+                           max_selected=Kpad, chunk_tokens=chunk, num_chunks=NCs)
+    lg = torch.from_numpy(logits).float().to(DEV)
+    vr = torch.from_numpy(vrows.view(np.int16)).to(DEV)
+    ns = torch.from_numpy(n_sel).to(DEV)
+    ho = torch.full((w.B, w.Hq, NCs, D), 5.0, device=DEV); hm = torch.full((w.B, w.Hq, NCs), 5.0, device=DEV)
+    hl = torch.full((w.B, w.Hq, NCs), 5.0, device=DEV)
+    pkg.hg_attn_partial_from_logits(lg, vr, ns, ho, hm, hl, desc)
+
+    # chunk partials against the oracle, fed with the fp32 logits the GPU saw
+    lg32 = lg.double().cpu().numpy()
+    rm = np.full((w.B, w.Hq, NCs), -np.inf); rl = np.zeros((w.B, w.Hq, NCs)); ro = np.zeros((w.B, w.Hq, NCs, D))
+    for b in range(w.B):
+        for h in range(w.Hq):
+            for c in range(NCs):
+                a, e = c * chunk, min((c + 1) * chunk, int(n_sel[b]))
+                if e > a:
+                    rm[b, h, c], rl[b, h, c], ro[b, h, c] = O.partial_from_logits(lg32[b, h, a:e], vrows[b, h // w.G, a:e], dtype)
+    torch.cuda.synchronize()
+    check_partials(ho.reshape(-1, D), hm.reshape(-1), hl.reshape(-1), rm.reshape(-1), rl.reshape(-1), ro.reshape(-1, D))
+
+    # merged with the GPU slice's partials: monolithic attention over the GPU slice plus the selected host tokens
+    prob = DeviceProblem(w, DEV)
+    prob.partial()
+    prob.merge([(ho, hm, hl)])
+    torch.cuda.synchronize()
+    out, lse = prob.out.double().cpu().numpy(), prob.lse.double().cpu().numpy()
+    ref_out = np.zeros_like(out); ref_lse = np.zeros_like(lse)
+    for b in range(w.B):
+        for h in range(w.Hq):
+            g = h // w.G
+            host = chosen[(b, g)]
+            if b == 1 and h == 0 and len(host) > 3:
+                drop = np.zeros(len(host), dtype=bool); drop[1::3] = True
+                host = host[~drop]
+            tokens = np.concatenate([host, np.arange(w.tok_begin[b], w.tok_end[b])]).astype(np.int64)
+            Kr, Vr = np.ascontiguousarray(K[b, :, g]), np.ascontiguousarray(V[b, :, g])
+            ref_out[b, h], ref_lse[b, h] = O.full(q[b, h], Kr, Vr, dtype, idx=tokens)
+            if keep == 1.0 and not (b == 1 and h == 0):
+                lo, ll = O.literal(q[b, h], Kr, Vr, dtype, np.sort(host), np.arange(w.tok_begin[b], w.tok_end[b]))
+                assert np.abs(lo - ref_out[b, h]).max() < 1e-12 and abs(ll - ref_lse[b, h]) < 1e-12
+    assert np.abs(out - ref_out).max() <= OUT_MAX_ABS
+    assert np.linalg.norm(out - ref_out) / np.linalg.norm(ref_out) <= OUT_REL_L2
+    assert np.abs(lse - ref_lse).max() <= LSE_ABS
+
+
+def test_handoff_rejects_bad_descriptions():
+    from paper_2604_18529_b200 import binding as hg
+    t = torch.zeros(8, device=DEV)
+    ti = torch.zeros(8, dtype=torch.int32, device=DEV)
+    for bad in (dict(chunk_tokens=48), dict(chunk_tokens=2048), dict(num_chunks=1, max_selected=4096), dict(head_dim=96)):
+        kw = dict(batch=1, num_q_heads=2, num_kv_heads=1, head_dim=128, dtype="f16", max_selected=64, chunk_tokens=64)
+        kw.update(bad)
+        with pytest.raises(hg.HgError):
+            pkg.hg_attn_partial_from_logits(t, t.half(), ti, t, t, t, pkg.logits_desc(**kw))

@@ -159,6 +159,37 @@ def test_empty_sets():
     assert lse == -math.inf and not out.any()
 
 
+def test_partial_from_logits_is_the_hand_off_form_of_partial():
+    """Host logits + gathered V rows give the partial of those tokens: against brute force, against PARTIAL
+    over an index list, and merged with the device's partial against monolithic attention (the paper's
+    workflow: CPU logits for its tokens, GPU logits for its own, one softmax over both)."""
+    n, D = 90, 16
+    q, K, V = rand_case(n, D, "f16", sigma=1.5)
+    out, lse = O.full(q, K, V, "f16")
+    host = np.sort(RNG.permutation(n)[:37]); dev = np.setdiff1d(np.arange(n), host)
+    s = O.logits(q, K, "f16", idx=host)                                   # what the host's logits calculator sends
+    m, l, o = O.partial_from_logits(s, V[host], "f16")
+    sd = np_decode(V[host], "f16").astype(np.float64)
+    w = np.exp(s - s.max())
+    assert m == s.max() and abs(l - w.sum()) < 1e-13
+    np.testing.assert_allclose(o, (w[:, None] * sd).sum(axis=0), rtol=0, atol=1e-12)
+    pm, pl, po = O.partial(q, K, V, "f16", idx=host)
+    assert (m, l) == (pm, pl) and np.array_equal(o, po)
+    dm, dl, do = O.partial(q, K, V, "f16", idx=dev)
+    mo, ml = O.merge([m, dm], [l, dl], [o, do])
+    np.testing.assert_allclose(mo, out, rtol=1e-12, atol=1e-14)
+    assert abs(ml - lse) < 1e-12
+    lo, ll = O.literal(q, K, V, "f16", host, dev)
+    np.testing.assert_allclose(mo, lo, rtol=1e-12, atol=1e-14)
+    # unselected slots carry -inf; nothing selected is the empty partial
+    s2 = s.copy(); s2[::2] = -np.inf
+    m2, l2, o2 = O.partial_from_logits(s2, V[host], "f16")
+    m3, l3, o3 = O.partial_from_logits(s[1::2], V[host][1::2], "f16")
+    assert (m2, l2) == (m3, l3) and np.array_equal(o2, o3)
+    me, le, oe = O.partial_from_logits(np.full(5, -np.inf), V[:5], "f16")
+    assert me == -math.inf and le == 0 and not oe.any()
+
+
 # ---- invariants -------------------------------------------------------------------------------
 
 def test_partial_invariants_and_convex_hull():
