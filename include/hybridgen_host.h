@@ -1,0 +1,97 @@
+/*
+ * hybridgen_host.h - host-side (CPU) companions of the device library: the pieces of HybridGen's
+ * CPU stage that feed hg_attn_partial_from_logits.  Plain C ABI, host pointers only, no CUDA calls;
+ * they work on a machine without a GPU.
+ *
+ *   hg_host_logits            the Logits Calculator (Section 4.2, CPU-side support): scaled logits
+ *                             q.k / sqrt(D) of host-resident keys
+ *   hg_host_select_topk       Post-QK^T selection (Section 4.3 / 4.5): the K largest scores per row
+ *   hg_host_select_positions  a Pre-QK^T, position-based selection (Section 4.5): the first `sinks` and the
+ *                             last `window` tokens
+ *   hg_host_gather_rows       gathers the selected tokens' V rows into a staging buffer for the transfer
+ *   hg_sched_init / _update   the Feedback Scheduler policy (Algorithm 1)
+ */
+#ifndef HYBRIDGEN_HOST_H_
+#define HYBRIDGEN_HOST_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#include "hybridgen_attn.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Layout of the host-resident K (or V) rows: element (b, t, g, d) at
+ * b * seq_stride + t * tok_stride + g * head_stride + d, in 16-bit elements. */
+typedef struct hg_host_desc {
+    uint32_t struct_size;
+    int32_t batch;          /* B */
+    int32_t num_q_heads;    /* Hq */
+    int32_t num_kv_heads;   /* Hkv */
+    int32_t head_dim;       /* D, a multiple of 8 */
+    int32_t dtype;          /* hg_dtype */
+    int32_t max_selected;   /* K: slots per row in idx / logits */
+    int32_t reserved;
+    int64_t seq_stride;
+    int64_t tok_stride;
+    int64_t head_stride;
+    float scale;            /* 0 means 1/sqrt(D) */
+    int32_t threads;        /* worker threads; 0 means one per available core */
+} hg_host_desc;
+
+/*
+ * logits[b][h][i] = scale * <q[b][h], K[b][tok_i][h / G]> for slot i < n_sel[b], where tok_i = idx[b][h / G][i]
+ * (idx: host int32 [B][Hkv][K]) or tok_i = i when idx is NULL; slots i >= n_sel[b] receive -inf.
+ * q: host [B][Hq][D] 16-bit.  Products are exact, accumulation is fp32.
+ * Returns HG_ERR_INVALID_ARG for null pointers or a malformed description.
+ */
+hg_status hg_host_logits(const void* q, const void* k_rows, const int32_t* idx, const int32_t* n_sel, float* logits,
+                         const hg_host_desc* desc);
+
+/*
+ * For each of `rows` score rows of length `stride` (the first n[r] entries valid): the indices of the
+ * min(k, n[r]) largest scores, in ascending index order; ties go to the lower index; NaN scores are
+ * never selected.  idx_out: int32 [rows][k], unused slots -1; n_out[r] = number selected.
+ */
+hg_status hg_host_select_topk(const float* scores, int64_t rows, int64_t stride, const int32_t* n, int32_t k,
+                              int32_t* idx_out, int32_t* n_out);
+
+/*
+ * Position-based selection among n_tokens tokens: the first `sinks` and the last `window` of them, at most k
+ * (sinks first), ascending.  Returns the number written to idx_out (capacity k).
+ */
+int32_t hg_host_select_positions(int32_t n_tokens, int32_t sinks, int32_t window, int32_t k, int32_t* idx_out);
+
+/*
+ * dst[b][g][i][:] = rows[b][idx[b][g][i]][g][:] for i < n_sel[b] (layout of `rows` as in desc); slots beyond
+ * n_sel[b] are zero-filled.  dst: host 16-bit [B][Hkv][K][D].
+ */
+hg_status hg_host_gather_rows(const void* rows, const int32_t* idx, const int32_t* n_sel, void* dst,
+                              const hg_host_desc* desc);
+
+/* Feedback Scheduler (Algorithm 1). */
+typedef enum hg_sched_strategy { HG_SCHED_POST_QK = 0, HG_SCHED_PRE_QK = 1 } hg_sched_strategy;
+
+typedef struct hg_sched_state {
+    int32_t k;         /* tokens the CPU stage processes */
+    int32_t strategy;  /* hg_sched_strategy */
+} hg_sched_state;
+
+/* K <- K_min, strategy <- Post-QK^T. */
+void hg_sched_init(hg_sched_state* st, int32_t k_min);
+
+/*
+ * One step of the policy on the measured stage latencies (any common unit).  If the CPU stage plus the
+ * transfer hides behind the GPU stage (t_cpu + t_tx <= t_gpu) K grows by `step` (up to k_max) - coming
+ * from Pre-QK^T the strategy first returns to Post-QK^T; otherwise K shrinks by `step` down to k_min, and at
+ * k_min the strategy becomes Pre-QK^T.
+ */
+void hg_sched_update(hg_sched_state* st, double t_gpu, double t_cpu, double t_tx, int32_t k_min, int32_t k_max,
+                     int32_t step);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HYBRIDGEN_HOST_H_ */

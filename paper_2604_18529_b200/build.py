@@ -9,9 +9,9 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libhybridgen_attn.so")
-SOURCES = [os.path.join(CSRC, "hg_attn.cu")]
+SOURCES = [os.path.join(CSRC, "hg_attn.cu"), os.path.join(CSRC, "hg_host.cpp")]
 DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("hg_device.cuh", "hg_partial.cuh", "hg_merge.cuh", "hg_logits.cuh")] + [
-    os.path.join(ROOT, "include", "hybridgen_attn.h")]
+    os.path.join(ROOT, "include", "hybridgen_attn.h"), os.path.join(ROOT, "include", "hybridgen_host.h")]
 
 
 def nvcc_path() -> str:

@@ -1,0 +1,109 @@
+"""ctypes binding of the host-side companions in ``include/hybridgen_host.h`` (argument marshalling only).
+
+Arrays are host torch tensors (16-bit K/V/q as float16 or bfloat16, indices int32, logits float32)."""
+from __future__ import annotations
+
+import ctypes as C
+from typing import Optional
+
+import torch
+
+from .binding import HG_OK, HgError, _DTYPES, _host, lib
+
+HG_SCHED_POST_QK, HG_SCHED_PRE_QK = 0, 1
+
+
+class HgHostDesc(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("batch", C.c_int32), ("num_q_heads", C.c_int32), ("num_kv_heads", C.c_int32),
+        ("head_dim", C.c_int32), ("dtype", C.c_int32), ("max_selected", C.c_int32), ("reserved", C.c_int32),
+        ("seq_stride", C.c_int64), ("tok_stride", C.c_int64), ("head_stride", C.c_int64), ("scale", C.c_float),
+        ("threads", C.c_int32),
+    ]
+
+
+class HgSchedState(C.Structure):
+    _fields_ = [("k", C.c_int32), ("strategy", C.c_int32)]
+
+
+_ready = False
+
+
+def _lib():
+    global _ready
+    L = lib()
+    if not _ready:
+        vp = C.c_void_p
+        L.hg_host_logits.argtypes = [vp, vp, vp, vp, vp, C.POINTER(HgHostDesc)]
+        L.hg_host_logits.restype = C.c_int
+        L.hg_host_select_topk.argtypes = [vp, C.c_int64, C.c_int64, vp, C.c_int32, vp, vp]
+        L.hg_host_select_topk.restype = C.c_int
+        L.hg_host_select_positions.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, vp]
+        L.hg_host_select_positions.restype = C.c_int32
+        L.hg_host_gather_rows.argtypes = [vp, vp, vp, vp, C.POINTER(HgHostDesc)]
+        L.hg_host_gather_rows.restype = C.c_int
+        L.hg_sched_init.argtypes = [C.POINTER(HgSchedState), C.c_int32]
+        L.hg_sched_init.restype = None
+        L.hg_sched_update.argtypes = [C.POINTER(HgSchedState), C.c_double, C.c_double, C.c_double, C.c_int32, C.c_int32, C.c_int32]
+        L.hg_sched_update.restype = None
+        _ready = True
+    return L
+
+
+def host_desc(rows: torch.Tensor, num_q_heads: int, max_selected: int, scale: float = 0.0, threads: int = 0) -> HgHostDesc:
+    """Describe host rows laid out [B][T][Hkv][D] (any strides with D contiguous)."""
+    B, _, Hkv, D = rows.shape
+    assert rows.stride(3) == 1
+    d = HgHostDesc()
+    d.struct_size = C.sizeof(HgHostDesc)
+    d.batch, d.num_q_heads, d.num_kv_heads, d.head_dim = B, num_q_heads, Hkv, D
+    d.dtype = _DTYPES[rows.dtype]
+    d.max_selected = max_selected
+    d.seq_stride, d.tok_stride, d.head_stride = rows.stride(0), rows.stride(1), rows.stride(2)
+    d.scale, d.threads = scale, threads
+    return d
+
+
+def _check(st, where):
+    if st != HG_OK:
+        raise HgError(st, where)
+
+
+def hg_host_logits(q: torch.Tensor, k_rows: torch.Tensor, idx: Optional[torch.Tensor], n_sel: torch.Tensor,
+                   logits: torch.Tensor, desc: HgHostDesc) -> None:
+    _check(_lib().hg_host_logits(_host(q, "q"), k_rows.data_ptr(), _host(idx, "idx", torch.int32),
+                                 _host(n_sel, "n_sel", torch.int32), _host(logits, "logits", torch.float32), C.byref(desc)),
+           "hg_host_logits")
+
+
+def hg_host_select_topk(scores: torch.Tensor, n: torch.Tensor, k: int):
+    rows, stride = scores.shape
+    idx = torch.empty(rows, k, dtype=torch.int32)
+    n_out = torch.empty(rows, dtype=torch.int32)
+    _check(_lib().hg_host_select_topk(_host(scores, "scores", torch.float32), rows, stride, _host(n, "n", torch.int32), k,
+                                      idx.data_ptr(), n_out.data_ptr()), "hg_host_select_topk")
+    return idx, n_out
+
+
+def hg_host_select_positions(n_tokens: int, sinks: int, window: int, k: int) -> torch.Tensor:
+    idx = torch.empty(max(k, 1), dtype=torch.int32)
+    n = _lib().hg_host_select_positions(n_tokens, sinks, window, k, idx.data_ptr())
+    return idx[:n]
+
+
+def hg_host_gather_rows(rows: torch.Tensor, idx: torch.Tensor, n_sel: torch.Tensor, dst: torch.Tensor, desc: HgHostDesc) -> None:
+    _check(_lib().hg_host_gather_rows(rows.data_ptr(), _host(idx, "idx", torch.int32), _host(n_sel, "n_sel", torch.int32),
+                                      _host(dst, "dst"), C.byref(desc)), "hg_host_gather_rows")
+
+
+class FeedbackScheduler:
+    """Algorithm 1 as a small controller: feed it the measured stage latencies, read K and the strategy."""
+
+    def __init__(self, k_min: int, k_max: int, step: int):
+        self.k_min, self.k_max, self.step = k_min, k_max, step
+        self.state = HgSchedState()
+        _lib().hg_sched_init(C.byref(self.state), k_min)
+
+    def update(self, t_gpu: float, t_cpu: float, t_tx: float):
+        _lib().hg_sched_update(C.byref(self.state), t_gpu, t_cpu, t_tx, self.k_min, self.k_max, self.step)
+        return self.state.k, self.state.strategy

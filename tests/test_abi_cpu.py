@@ -11,7 +11,7 @@ from paper_2604_18529_b200 import binding as hg
 from paper_2604_18529_b200 import build as hgbuild
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-HEADER = os.path.join(ROOT, "include", "hybridgen_attn.h")
+HEADERS = [os.path.join(ROOT, "include", "hybridgen_attn.h"), os.path.join(ROOT, "include", "hybridgen_host.h")]
 
 
 @pytest.fixture(scope="module")
@@ -21,15 +21,19 @@ def lib():
 
 
 def declared_functions():
-    src = open(HEADER).read()
-    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
-    return sorted(set(re.findall(r"\b(hg_[a-z_0-9]+)\s*\(", src)))
+    names = set()
+    for header in HEADERS:
+        src = re.sub(r"/\*.*?\*/", "", open(header).read(), flags=re.S)
+        names |= set(re.findall(r"\b(hg_[a-z_0-9]+)\s*\(", src))
+    return sorted(names)
 
 
 def test_header_functions_are_exported(lib):
     names = declared_functions()
     assert {"hg_attn_partial", "hg_attn_merge", "hg_attn_decode", "hg_attn_decode_host",
-            "hg_attn_workspace_bytes", "hg_kv_read_probe", "hg_status_string", "hg_version"} <= set(names)
+            "hg_attn_workspace_bytes", "hg_kv_read_probe", "hg_status_string", "hg_version", "hg_attn_decode_static",
+            "hg_attn_partial_from_logits", "hg_host_logits", "hg_host_select_topk", "hg_host_select_positions",
+            "hg_host_gather_rows", "hg_sched_init", "hg_sched_update"} <= set(names)
     for n in names:
         assert hasattr(lib, n), n
 

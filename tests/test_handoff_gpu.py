@@ -111,3 +111,64 @@ def test_handoff_rejects_bad_descriptions():
         kw.update(bad)
         with pytest.raises(hg.HgError):
             pkg.hg_attn_partial_from_logits(t, t.half(), ti, t, t, t, pkg.logits_desc(**kw))
+
+
+# ---- the whole CPU stage with the library's own host functions ---------------------------------------------------
+
+@pytest.mark.parametrize("strategy", ["post_qk", "pre_qk"])
+@pytest.mark.parametrize("G", [1, 4])
+def test_cpu_stage_feeds_the_gpu_stage(strategy, G):
+    """Post-QK^T: host logits for every offloaded token, top-K per KV head (score = best head of the group),
+    Pre-QK^T: sinks + recent window chosen before any logit is computed; then logits of the chosen tokens and
+    their V rows cross to the GPU, which merges them with its own slice.  Equal to monolithic attention over
+    exactly those tokens."""
+    from paper_2604_18529_b200 import host as H
+    w = W.AttnWorkload("stage", 2, 2 * G, 2, 128, "f16", [1500, 700], [1100, 420], [1500, 700], page_size=16,
+                       chunk_tokens=128, seed=60 + G, outlier_frac=0.02)
+    q_t, K_t, V_t = w.q(), w.kv_logical("k"), w.kv_logical("v")
+    n_host = torch.tensor(w.tok_begin, dtype=torch.int32)
+    Ksel = 96
+    if strategy == "post_qk":
+        all_logits = torch.empty(w.B, w.Hq, int(n_host.max()))
+        H.hg_host_logits(q_t, K_t, None, n_host, all_logits, H.host_desc(K_t, w.Hq, int(n_host.max())))
+        score = all_logits.view(w.B, w.Hkv, G, -1).max(dim=2).values.reshape(w.B * w.Hkv, -1).contiguous()
+        idx, n_out = H.hg_host_select_topk(score, n_host.repeat_interleave(w.Hkv), Ksel)
+        idx = idx.view(w.B, w.Hkv, Ksel)
+        n_sel = n_out.view(w.B, w.Hkv)[:, 0].contiguous()
+    else:
+        idx = torch.full((w.B, w.Hkv, Ksel), -1, dtype=torch.int32)
+        n_sel = torch.zeros(w.B, dtype=torch.int32)
+        for b in range(w.B):
+            sel = H.hg_host_select_positions(int(n_host[b]), 4, 64, Ksel)
+            idx[b, :, : len(sel)] = sel
+            n_sel[b] = len(sel)
+    desc = H.host_desc(K_t, w.Hq, Ksel)
+    logits = torch.empty(w.B, w.Hq, Ksel)
+    H.hg_host_logits(q_t, K_t, idx, n_sel, logits, desc)
+    vsel = torch.empty(w.B, w.Hkv, Ksel, w.D, dtype=torch.float16)
+    H.hg_host_gather_rows(V_t, idx, n_sel, vsel, desc)
+
+    ld = pkg.logits_desc(batch=w.B, num_q_heads=w.Hq, num_kv_heads=w.Hkv, head_dim=w.D, dtype=w.dtype, max_selected=Ksel,
+                         chunk_tokens=32)
+    NCs = ld.num_chunks
+    ho = torch.empty(w.B, w.Hq, NCs, w.D, device=DEV); hm = torch.empty(w.B, w.Hq, NCs, device=DEV); hl = torch.empty_like(hm)
+    pkg.hg_attn_partial_from_logits(logits.to(DEV), vsel.to(DEV), n_sel.to(DEV), ho, hm, hl, ld)
+    prob = DeviceProblem(w, DEV)
+    prob.partial()
+    prob.merge([(ho, hm, hl)])
+    torch.cuda.synchronize()
+
+    q, K, V = bits(q_t), bits(K_t), bits(V_t)
+    out, lse = prob.out.double().cpu().numpy(), prob.lse.double().cpu().numpy()
+    ref_out = np.zeros_like(out); ref_lse = np.zeros_like(lse)
+    for b in range(w.B):
+        for h in range(w.Hq):
+            g = h // G
+            host = idx[b, g, : int(n_sel[b])].numpy().astype(np.int64)
+            assert len(set(host.tolist())) == len(host) and (host < w.tok_begin[b]).all()
+            tokens = np.concatenate([host, np.arange(w.tok_begin[b], w.tok_end[b])])
+            ref_out[b, h], ref_lse[b, h] = O.full(q[b, h], np.ascontiguousarray(K[b, :, g]), np.ascontiguousarray(V[b, :, g]),
+                                                  w.dtype, idx=tokens)
+    assert np.abs(out - ref_out).max() <= OUT_MAX_ABS
+    assert np.linalg.norm(out - ref_out) / np.linalg.norm(ref_out) <= OUT_REL_L2
+    assert np.abs(lse - ref_lse).max() <= LSE_ABS

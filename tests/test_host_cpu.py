@@ -1,0 +1,113 @@
+"""Host-side companions (logits calculator, selection, gather, feedback scheduler) against the oracle and the
+plain statements in oracle/hg_policy.py.  CPU only."""
+import itertools
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import hg_oracle as O
+from oracle import hg_policy as P
+from paper_2604_18529_b200 import build as hgbuild
+from paper_2604_18529_b200 import host as H
+from paper_2604_18529_b200 import workload as W
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    hgbuild.build()
+
+
+def bits(t):
+    return t.contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+@pytest.mark.parametrize("dtype,D,G", [("f16", 128, 1), ("bf16", 64, 4), ("f16", 64, 3)])
+def test_host_logits_match_the_oracle(dtype, D, G):
+    w = W.AttnWorkload("h", 2, 2 * G, 2, D, dtype, [300, 170], [200, 170], [300, 170], seed=3, sigma_kv=1.5)
+    q, K = w.q(), w.kv_logical("k")                         # [B][Hq][D], [B][Lmax][Hkv][D]
+    n_host = torch.tensor(w.tok_begin, dtype=torch.int32)   # the host holds [0, tok_begin)
+    Ksel = int(n_host.max())
+    desc = H.host_desc(K, w.Hq, Ksel, threads=3)
+    logits = torch.empty(w.B, w.Hq, Ksel)
+    H.hg_host_logits(q, K, None, n_host, logits, desc)
+    qb, Kb = bits(q), bits(K)
+    for b in range(w.B):
+        for h in range(w.Hq):
+            want = O.logits(qb[b, h], np.ascontiguousarray(Kb[b, :, h // G]), dtype, t0=0, n=int(n_host[b]))
+            got = logits[b, h, : int(n_host[b])].double().numpy()
+            assert np.abs(got - want).max() <= 2e-5 * max(1.0, np.abs(want).max())
+            assert torch.isinf(logits[b, h, int(n_host[b]):]).all()
+    # through an index list, with an explicit scale
+    idx = torch.stack([torch.stack([torch.randperm(Ksel, generator=torch.Generator().manual_seed(b * 7 + g))[:50]
+                                    for g in range(w.Hkv)]) for b in range(w.B)]).to(torch.int32)
+    idx[1] = idx[1] % max(int(n_host[1]), 1)
+    n_sel = torch.tensor([50, 37], dtype=torch.int32)
+    desc2 = H.host_desc(K, w.Hq, 50, scale=0.25)
+    lg2 = torch.empty(w.B, w.Hq, 50)
+    H.hg_host_logits(q, K, idx, n_sel, lg2, desc2)
+    for b in range(w.B):
+        for h in range(w.Hq):
+            n = int(n_sel[b])
+            want = O.logits(qb[b, h], np.ascontiguousarray(Kb[b, :, h // G]), dtype, scale=0.25, idx=idx[b, h // G, :n].numpy())
+            assert np.abs(lg2[b, h, :n].double().numpy() - want).max() <= 2e-5 * max(1.0, np.abs(want).max())
+
+
+def test_topk_selection_matches_the_sort_definition():
+    rng = np.random.default_rng(5)
+    scores = rng.standard_normal((6, 200)).astype(np.float32)
+    scores[0, 10:20] = scores[0, 5]                       # ties
+    scores[1, 3] = np.nan
+    scores[2, :] = -np.inf
+    n = np.array([200, 200, 200, 0, 7, 150], dtype=np.int32)
+    for k in (1, 5, 64, 300):
+        idx, n_out = H.hg_host_select_topk(torch.from_numpy(scores), torch.from_numpy(n), k)
+        for r in range(6):
+            want = P.topk(list(scores[r, : n[r]]), k)
+            assert int(n_out[r]) == len(want)
+            assert idx[r, : len(want)].tolist() == want and (idx[r, len(want):] == -1).all()
+
+
+def test_position_selection():
+    for n_tokens, sinks, window, k in itertools.product([0, 1, 5, 100, 2000], [0, 4], [0, 3, 1024], [1, 6, 5000]):
+        got = H.hg_host_select_positions(n_tokens, sinks, window, k).tolist()
+        assert got == P.positions(n_tokens, sinks, window, k) if n_tokens > 0 else got == []
+    assert H.hg_host_select_positions(2000, 4, 1024, 1028).tolist() == list(range(4)) + list(range(976, 2000))
+
+
+def test_gather_rows():
+    w = W.AttnWorkload("g", 2, 4, 2, 64, "bf16", [90, 60], [0, 0], [90, 60], seed=9)
+    V = w.kv_logical("v")
+    K = 11
+    idx = torch.tensor([[[5, 0, 89, 3, 3, 7, 1, 2, 4, 6, 8], [1] * 11], [[59, 58, 0, 1, 2, 3, 4, 5, 6, 7, 8], [9] * 11]], dtype=torch.int32)
+    n_sel = torch.tensor([11, 4], dtype=torch.int32)
+    dst = torch.full((2, 2, K, 64), 1.0, dtype=torch.bfloat16)
+    H.hg_host_gather_rows(V, idx, n_sel, dst, H.host_desc(V, 4, K))
+    for b in range(2):
+        for g in range(2):
+            n = int(n_sel[b])
+            assert torch.equal(dst[b, g, :n], V[b, idx[b, g, :n].long(), g])
+            assert (dst[b, g, n:] == 0).all()
+
+
+def test_feedback_scheduler_follows_algorithm_1():
+    rng = np.random.default_rng(11)
+    k_min, k_max, step = 128, 1024, 96
+    s = H.FeedbackScheduler(k_min, k_max, step)
+    k, strat = P.feedback_scheduler_init(k_min)
+    assert (s.state.k, s.state.strategy) == (k, strat) == (128, P.POST_QK)
+    for _ in range(400):
+        t_gpu, t_cpu, t_tx = rng.uniform(0.5, 2.0), rng.uniform(0.1, 2.0), rng.uniform(0.0, 0.5)
+        k, strat = P.feedback_scheduler_step(k, strat, t_gpu, t_cpu, t_tx, k_min, k_max, step)
+        assert s.update(t_gpu, t_cpu, t_tx) == (k, strat)
+        assert k_min <= k <= k_max
+    # the listing's cases, one by one
+    s = H.FeedbackScheduler(128, 1024, 100)
+    assert s.update(1.0, 0.5, 0.2) == (228, H.HG_SCHED_POST_QK)          # hidden: K grows
+    assert s.update(1.0, 0.9, 0.2) == (128, H.HG_SCHED_POST_QK)          # not hidden, K > K_min: shrink, clamped
+    assert s.update(1.0, 0.9, 0.2) == (128, H.HG_SCHED_PRE_QK)           # at K_min: switch strategy
+    assert s.update(1.0, 0.5, 0.5) == (128, H.HG_SCHED_POST_QK)          # boundary t_cpu + t_tx == t_gpu counts as hidden
+    for _ in range(20):
+        s.update(1.0, 0.1, 0.1)
+    assert s.state.k == 1024
