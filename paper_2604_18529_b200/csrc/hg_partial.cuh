@@ -148,8 +148,13 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int Y = p.Hkv * p.head_blocks;
 
-    // a wait already timed out in this call (or the caller left the word set): do not queue behind it
-    if (p.status && *reinterpret_cast<volatile int32_t*>(p.status) == HG_DEV_WAIT_TIMEOUT) return;
+    // Loads whose answers are needed a little later are issued first, so that their round trips overlap the
+    // set-up: the status word (a wait that timed out earlier in this call, or a word the caller left set,
+    // means: do not queue behind it), and this CTA's second work item (its first is its own block index).
+    const int32_t status_at_entry = p.status ? *reinterpret_cast<volatile int32_t*>(p.status) : HG_DEV_OK;
+    int early_request = 0;
+    if (p.persistent && p.sched && tid == CONSUMER_THREADS && !p.test_stall)
+        early_request = (int)gridDim.x + atomicAdd(p.sched, 1);
 
     // ---- set-up: barriers, and for the persistent schedule the item counts per sequence ---------------
     if (tid == 0) {
@@ -162,6 +167,7 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
         fence_barrier_init();
     }
     int n_items = 1, item_step = 1, item_first = 0;
+    if (status_at_entry == HG_DEV_WAIT_TIMEOUT) return;
     if (p.persistent) {
         // cum[b+1] = sum_{b' <= b} nc_b' * Y : one warp, each lane a contiguous block of sequences
         if (warp == 0) {
@@ -191,31 +197,8 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
         item_step = rounds > 0 ? (n_items + rounds - 1) / rounds : 1;
         item_first = blockIdx.x;
 
-        // empty chunk slots (c >= nc_b): neutral elements, spread over all CTAs
-        for (int s = blockIdx.x; s < p.B * Y; s += gridDim.x) {
-            const int b = s / Y, y = s - b * Y;
-            int tb, te;
-            const int nc = seq_chunks(p, b, tb, te);
-            const int ne = p.NC - nc;                 // empty slots per head
-            if (ne <= 0) continue;
-            if constexpr (MODE == MODE_PROBE) {
-                for (int i = tid; i < ne; i += THREADS) p.sink[((size_t)b * p.Hkv + y) * p.NC + nc + i] = 0u;
-            } else {
-                const int hb = y % p.head_blocks, g = y / p.head_blocks;
-                const int nh = (MODE == MODE_GQA) ? min(8, p.G - hb * 8) : 1;
-                const int hq0 = (MODE == MODE_GQA) ? g * p.G + hb * 8 : g;
-                for (int i = tid; i < nh * ne * D; i += THREADS) {
-                    const int sl = i / D, hh = sl / ne, cc = nc + sl % ne;
-                    p.o_part[(((size_t)b * p.Hq + hq0 + hh) * p.NC + cc) * D + i % D] = 0.f;
-                }
-                for (int i = tid; i < nh * ne; i += THREADS) {
-                    const int hh = i / ne, cc = nc + i % ne;
-                    p.m_part[((size_t)b * p.Hq + hq0 + hh) * p.NC + cc] = NEG_INF;
-                    p.l_part[((size_t)b * p.Hq + hq0 + hh) * p.NC + cc] = 0.f;
-                }
-            }
-        }
-        if (n_items == 0 || (!p.sched && (int)blockIdx.x >= item_step)) return;
+        // (CTAs beyond the round-robin width, or any CTA when there is no item at all, still help with the empty
+        // chunk slots below before they leave)
     } else {
         __syncthreads();
     }
@@ -297,17 +280,19 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
         };
         // Index of the k-th item this CTA takes.  With the dynamic schedule lane 0 holds the counter's answer
         // in `raw` until it is needed, so that the atomic's round trip overlaps the current item's loads.
+        // (dynamic schedule: every CTA starts with the item of its own block index, the counter hands out
+        // the items from gridDim.x on)
         auto request = [&](int k) -> int {
             if (!p.persistent) return k == 0 ? 0 : n_items;
-            if (dynamic) return lane == 0 ? atomicAdd(p.sched, 1) : 0;
-            return (int)blockIdx.x + k * item_step;
+            if (dynamic) return k == 0 ? (int)blockIdx.x : (k == 1 ? early_request : (lane == 0 ? (int)gridDim.x + atomicAdd(p.sched, 1) : 0));
+            return (int)blockIdx.x < item_step ? (int)blockIdx.x + k * item_step : n_items;   // round-robin over item_step CTAs
         };
         auto settle = [&](int raw) -> int { return dynamic ? __shfl_sync(0xffffffffu, raw, 0) : raw; };
 
         int s = 0, issued = 0, k = 0;                // ring position, stages armed so far, items taken so far
         uint32_t ph = 0;
         bool alive = true;
-        int i_cur = p.test_stall ? n_items : settle(request(0));
+        int i_cur = p.test_stall ? n_items : request(0);
         int raw_nxt = request(1);
         Item cur;
         if (i_cur < n_items) {                       // page ids of the first item
@@ -319,24 +304,29 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
         while (i_cur < n_items && alive) {
             const int page0 = first_page(cur);
             const int* const pages = &ctl.pages[(k & 1) * (MAX_CHUNK_PAGES / 2)];
-            // the next item: its index was requested one item ago; request the one after it, and start fetching
-            // the next item's page ids (parked in shared memory after this item's loads have been issued)
-            const int i_nxt = settle(raw_nxt);
-            raw_nxt = request(k + 2);
-            const bool has_next = i_nxt < n_items;
+            // the next item (its index was requested one item ago) is looked at right after this item's first
+            // stage has been issued: the request for the item after it goes out, and the next item's page ids
+            // start loading (they are parked in shared memory once this item's loads have all been issued)
+            int i_nxt = n_items;
+            bool has_next = false;
             Item nxt = cur;
             int nxt_ids[PER_LANE];
             int nxt_npages = 0;
-            if (has_next) {
-                nxt = get_item(i_nxt);
-                const int np0 = first_page(nxt);
-                nxt_npages = min(num_pages_of(nxt), PERSIST_CHUNK_PAGES);
+            auto look_ahead = [&]() {
+                i_nxt = settle(raw_nxt);
+                raw_nxt = request(k + 2);
+                has_next = i_nxt < n_items;
+                if (has_next) {
+                    nxt = get_item(i_nxt);
+                    const int np0 = first_page(nxt);
+                    nxt_npages = min(num_pages_of(nxt), PERSIST_CHUNK_PAGES);
 #pragma unroll
-                for (int u = 0; u < PER_LANE; ++u) {
-                    const int idx = u * 32 + lane;
-                    nxt_ids[u] = idx < nxt_npages ? lookup(nxt, np0 + idx) : -2;
+                    for (int u = 0; u < PER_LANE; ++u) {
+                        const int idx = u * 32 + lane;
+                        nxt_ids[u] = idx < nxt_npages ? lookup(nxt, np0 + idx) : -2;
+                    }
                 }
-            }
+            };
             const int g = cur.y / p.head_blocks;
             const int q_heads = (MODE == MODE_GQA) ? min(8, p.G - (cur.y % p.head_blocks) * 8) : 1;
             const int q_head0 = (MODE == MODE_GQA) ? g * p.G + (cur.y % p.head_blocks) * 8 : g;
@@ -364,7 +354,10 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 }
                 ++issued;
                 if (++s == p.stages) { s = 0; ph ^= 1u; }
+                if (it == 0) look_ahead();
             }
+            if (!alive) break;
+            if (cur.ntiles == 0) look_ahead();
             if (!has_next) break;
             int* const dstp = &ctl.pages[((k + 1) & 1) * (MAX_CHUNK_PAGES / 2)];
 #pragma unroll
@@ -396,6 +389,33 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
         }
     } else {
         // =============================== consumer warps ===============================
+        if (p.persistent) {
+            // empty chunk slots (c >= nc_b): neutral elements, spread over all CTAs; the consumer warps write them
+            // while the first stage is on its way
+            for (int sl = blockIdx.x; sl < p.B * Y; sl += gridDim.x) {
+                const int b = sl / Y, y = sl - b * Y;
+                const int tb = ctl.tb[b], te = ctl.te[b];
+                const int nc = te > tb ? min((te + p.C - 1) / p.C - tb / p.C, p.NC) : 0;
+                const int ne = p.NC - nc;                 // empty slots per head
+                if (ne <= 0) continue;
+                if constexpr (MODE == MODE_PROBE) {
+                    for (int i = tid; i < ne; i += CONSUMER_THREADS) p.sink[((size_t)b * p.Hkv + y) * p.NC + nc + i] = 0u;
+                } else {
+                    const int hb = y % p.head_blocks, g = y / p.head_blocks;
+                    const int nh = (MODE == MODE_GQA) ? min(8, p.G - hb * 8) : 1;
+                    const int hq0 = (MODE == MODE_GQA) ? g * p.G + hb * 8 : g;
+                    for (int i = tid; i < nh * ne * D; i += CONSUMER_THREADS) {
+                        const int e = i / D, hh = e / ne, cc = nc + e % ne;
+                        p.o_part[(((size_t)b * p.Hq + hq0 + hh) * p.NC + cc) * D + i % D] = 0.f;
+                    }
+                    for (int i = tid; i < nh * ne; i += CONSUMER_THREADS) {
+                        const int hh = i / ne, cc = nc + i % ne;
+                        p.m_part[((size_t)b * p.Hq + hq0 + hh) * p.NC + cc] = NEG_INF;
+                        p.l_part[((size_t)b * p.Hq + hq0 + hh) * p.NC + cc] = 0.f;
+                    }
+                }
+            }
+        }
         int cs = 0;                // ring position and phase of the next stage to consume
         uint32_t cph = 0;
         // Barrier among the four consumer warps with a bounded wait (false: give up, the CTA is unwinding).
@@ -695,30 +715,46 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                     ctl.red_m[par][warp * 8 + 2 * tq] = m_run[0]; ctl.red_m[par][warp * 8 + 2 * tq + 1] = m_run[1];
                     ctl.red_l[par][warp * 8 + 2 * tq] = l_run[0]; ctl.red_l[par][warp * 8 + 2 * tq + 1] = l_run[1];
                 }
+                {   // this warp's [8 heads][D] into its own rows; heads 2tq and 2tq+1 sit in the same 2 KB part
+                    float* const lane_base = warp_scratch(s, warp, (2 * tq) * D + quad);
 #pragma unroll
-                for (int mt = 0; mt < KSTEPS; ++mt) {               // this warp's [8 heads][D] into its own rows
-                    const int d0 = mt * 16 + quad;
-                    *warp_scratch(s, warp, (2 * tq) * D + d0) = oacc[mt][0];
-                    *warp_scratch(s, warp, (2 * tq + 1) * D + d0) = oacc[mt][1];
-                    *warp_scratch(s, warp, (2 * tq) * D + d0 + 8) = oacc[mt][2];
-                    *warp_scratch(s, warp, (2 * tq + 1) * D + d0 + 8) = oacc[mt][3];
+                    for (int mt = 0; mt < KSTEPS; ++mt) {
+                        lane_base[mt * 16] = oacc[mt][0];
+                        lane_base[D + mt * 16] = oacc[mt][1];
+                        lane_base[mt * 16 + 8] = oacc[mt][2];
+                        lane_base[D + mt * 16 + 8] = oacc[mt][3];
+                    }
                 }
                 if (!consumer_sync()) break;
-                for (int u = tid; u < nheads * D; u += CONSUMER_THREADS) {
-                    const int hh = u / D, dd = u % D;
-                    float M = NEG_INF;
+                {   // thread -> (head, D/16 consecutive components): the four warp states of one head, weighted
+                    constexpr int PER = D / 16;
+                    const int hh = tid >> 4, dbase = (tid & 15) * PER;
+                    if (hh < nheads) {
+                        float mw[CONSUMER_WARPS], M = NEG_INF, lsum = 0.f;
 #pragma unroll
-                    for (int w2 = 0; w2 < CONSUMER_WARPS; ++w2) M = fmaxf(M, ctl.red_m[par][w2 * 8 + hh]);
-                    float accv = 0.f, lsum = 0.f;
+                        for (int w2 = 0; w2 < CONSUMER_WARPS; ++w2) { mw[w2] = ctl.red_m[par][w2 * 8 + hh]; M = fmaxf(M, mw[w2]); }
+                        float accv[PER];
 #pragma unroll
-                    for (int w2 = 0; w2 < CONSUMER_WARPS; ++w2) {
-                        const float w = fast_exp2(ctl.red_m[par][w2 * 8 + hh] - M);     // M is finite: the item has tokens
-                        accv = fmaf(w, *warp_scratch(s, w2, u), accv);
-                        lsum = fmaf(w, ctl.red_l[par][w2 * 8 + hh], lsum);
+                        for (int v = 0; v < PER; ++v) accv[v] = 0.f;
+#pragma unroll
+                        for (int w2 = 0; w2 < CONSUMER_WARPS; ++w2) {
+                            const float w = fast_exp2(mw[w2] - M);                 // M is finite: the item has tokens
+                            lsum = fmaf(w, ctl.red_l[par][w2 * 8 + hh], lsum);
+                            const float4* src = reinterpret_cast<const float4*>(warp_scratch(s, w2, hh * D + dbase));
+#pragma unroll
+                            for (int v4 = 0; v4 < PER / 4; ++v4) {
+                                const float4 x = src[v4];
+                                accv[v4 * 4 + 0] = fmaf(w, x.x, accv[v4 * 4 + 0]); accv[v4 * 4 + 1] = fmaf(w, x.y, accv[v4 * 4 + 1]);
+                                accv[v4 * 4 + 2] = fmaf(w, x.z, accv[v4 * 4 + 2]); accv[v4 * 4 + 3] = fmaf(w, x.w, accv[v4 * 4 + 3]);
+                            }
+                        }
+                        const size_t oslot = ((size_t)cur.b * p.Hq + h0 + hh) * p.NC + cur.c;
+                        float4* dst = reinterpret_cast<float4*>(p.o_part + oslot * D + dbase);
+#pragma unroll
+                        for (int v4 = 0; v4 < PER / 4; ++v4)
+                            dst[v4] = make_float4(accv[v4 * 4 + 0], accv[v4 * 4 + 1], accv[v4 * 4 + 2], accv[v4 * 4 + 3]);
+                        if ((tid & 15) == 0) { p.m_part[oslot] = M * LN2; p.l_part[oslot] = lsum; }
                     }
-                    const size_t oslot = ((size_t)cur.b * p.Hq + h0 + hh) * p.NC + cur.c;
-                    p.o_part[oslot * D + dd] = accv;
-                    if (dd == 0) { p.m_part[oslot] = M * LN2; p.l_part[oslot] = lsum; }
                 }
                 release(s, true);
             }
