@@ -255,6 +255,37 @@ hg_status hg_attn_partial_from_logits(const float* logits, const void* v_rows, c
                                       float* m_part, float* l_part, void* stream, const hg_logits_desc* desc);
 
 /*
+ * Appends the current decode step's K and V rows to the cache (Section 2.1: the new token's K, V are
+ * appended before its attention is computed).
+ *
+ *   k_new, v_new  dev 16-bit [B][Hkv][D], 16-byte aligned
+ *   k_cache, v_cache  dev pools (written)
+ *   seq_lens      dev int32 [B]: row b goes to position seq_lens[b], then seq_lens[b] += 1
+ *   tok_end       dev int32 [B] or NULL: where it equals the old length it grows too (the slice keeps reaching the
+ *                 newest token)
+ * The page that holds the new position must already be mapped in the block table (page allocation is the
+ * caller's); otherwise the row is dropped and *desc->status = HG_DEV_BAD_PAGE.  chunk fields of desc are unused.
+ */
+hg_status hg_kv_append(const void* k_new, const void* v_new, void* k_cache, void* v_cache, int32_t* seq_lens,
+                       int32_t* tok_end, void* stream, const hg_attn_desc* desc);
+
+/*
+ * Device half of the Eviction Engine and Token Mapper (Section 4.2, device-side support): moves the oldest
+ * tokens of the GPU slice out, least recently generated first.
+ *
+ * For every sequence the first ne = min(n_evict[b], max_evict, tok_end[b] - tok_begin[b]) tokens of the slice
+ * are copied, in token order, to k_out / v_out (dev 16-bit [B][max_evict][Hkv][D] - the token-major layout
+ * hg_host_logits reads), ready for one device-to-host copy by the caller.  Then tok_begin[b] += ne, every page
+ * that lies wholly below the new beginning is un-mapped (block-table entry -1) and its physical id listed in
+ * freed_pages (dev int32 [B][max_freed], -1 padded; n_freed dev int32 [B]; both may be NULL).  The pools are
+ * not modified.  desc->block_table is updated in place (it must be writable); with identity paging (NULL)
+ * only tok_begin moves.
+ */
+hg_status hg_kv_evict(const void* k_cache, const void* v_cache, int32_t* tok_begin, const int32_t* tok_end,
+                      const int32_t* n_evict, int32_t max_evict, void* k_out, void* v_out, int32_t* freed_pages,
+                      int32_t* n_freed, int32_t max_freed, void* stream, const hg_attn_desc* desc);
+
+/*
  * Evidence kernel, not part of the attention path: streams the same K and V tiles through the
  * same TMA pipeline as hg_attn_partial and folds them into one 32-bit checksum per work item
  * (sink: dev uint32 [B][Hkv][NC]).  Used to measure the read ceiling of the paged access pattern.

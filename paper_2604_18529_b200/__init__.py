@@ -21,5 +21,7 @@ from .binding import (  # noqa: F401
     hg_attn_workspace_bytes,
     hg_status_string,
     hg_kv_read_probe,
+    hg_kv_append,
+    hg_kv_evict,
     hg_version,
 )

@@ -101,6 +101,10 @@ def lib():
         L.hg_attn_decode_static.restype = C.c_int
         L.hg_attn_partial_from_logits.argtypes = [vp] * 7 + [C.POINTER(HgLogitsDesc)]
         L.hg_attn_partial_from_logits.restype = C.c_int
+        L.hg_kv_append.argtypes = [vp] * 7 + [C.POINTER(HgAttnDesc)]
+        L.hg_kv_append.restype = C.c_int
+        L.hg_kv_evict.argtypes = [vp] * 5 + [i32, vp, vp, vp, vp, i32, vp, C.POINTER(HgAttnDesc)]
+        L.hg_kv_evict.restype = C.c_int
         L.hg_kv_read_probe.argtypes = [vp] * 7 + [C.POINTER(HgAttnDesc)]
         L.hg_kv_read_probe.restype = C.c_int
         L.hg_status_string.argtypes = [C.c_int]
@@ -280,6 +284,26 @@ def hg_attn_decode_host(q_host, k_cache, v_cache, seq_lens_host, tok_begin_host,
                                    _dev(workspace, "workspace"), workspace.numel() * workspace.element_size(),
                                    _stream(stream), C.byref(desc))
     _check(st, "hg_attn_decode_host")
+
+
+def hg_kv_append(k_new, v_new, k_cache, v_cache, seq_lens, tok_end, desc: HgAttnDesc, stream=None) -> None:
+    """Write this step's K/V rows [B][Hkv][D] at position seq_lens[b] and advance seq_lens (and tok_end)."""
+    st = lib().hg_kv_append(_dev(k_new, "k_new"), _dev(v_new, "v_new"), _dev(k_cache, "k_cache"), _dev(v_cache, "v_cache"),
+                            _dev(seq_lens, "seq_lens", torch.int32), _dev(tok_end, "tok_end", torch.int32),
+                            _stream(stream), C.byref(desc))
+    _check(st, "hg_kv_append")
+
+
+def hg_kv_evict(k_cache, v_cache, tok_begin, tok_end, n_evict, k_out, v_out, freed_pages, n_freed, desc: HgAttnDesc,
+                stream=None) -> None:
+    """Copy the oldest n_evict[b] tokens of every slice to k_out / v_out [B][max_evict][Hkv][D], advance tok_begin
+    and un-map the pages that became empty (their ids go to freed_pages [B][max_freed])."""
+    st = lib().hg_kv_evict(_dev(k_cache, "k_cache"), _dev(v_cache, "v_cache"), _dev(tok_begin, "tok_begin", torch.int32),
+                           _dev(tok_end, "tok_end", torch.int32), _dev(n_evict, "n_evict", torch.int32), k_out.shape[1],
+                           _dev(k_out, "k_out"), _dev(v_out, "v_out"), _dev(freed_pages, "freed_pages", torch.int32),
+                           _dev(n_freed, "n_freed", torch.int32), 0 if freed_pages is None else freed_pages.shape[1],
+                           _stream(stream), C.byref(desc))
+    _check(st, "hg_kv_evict")
 
 
 def hg_kv_read_probe(k_cache, v_cache, seq_lens, tok_begin, tok_end, sink, desc: HgAttnDesc, stream=None) -> None:

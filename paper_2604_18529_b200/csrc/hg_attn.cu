@@ -13,6 +13,7 @@
 
 #include <atomic>
 
+#include "hg_kvcache.cuh"
 #include "hg_logits.cuh"
 #include "hg_merge.cuh"
 #include "hg_partial.cuh"
@@ -402,6 +403,62 @@ hg_status hg_attn_decode_host(const void* q_host, const void* k_cache, const voi
     if (lse_host) ok &= cudaMemcpyAsync(lse_host, lse_dev, rows * sizeof(float), cudaMemcpyDeviceToHost, cs) == cudaSuccess;
     if (!ok) { cudaGetLastError(); return HG_ERR_CUDA; }
     return HG_OK;
+}
+
+static KvPoolView pool_view(const hg_attn_desc* d, const void* k, const void* v) {
+    KvPoolView pv;
+    pv.k = static_cast<uint16_t*>(const_cast<void*>(k));
+    pv.v = static_cast<uint16_t*>(const_cast<void*>(v));
+    pv.block_table = d->block_table;
+    pv.page_stride = d->page_stride; pv.head_stride = d->head_stride; pv.tok_stride = d->tok_stride;
+    pv.B = d->batch; pv.Hkv = d->num_kv_heads; pv.D = d->head_dim; pv.page_size = d->page_size;
+    pv.page_shift = ilog2_exact(d->page_size); pv.max_pages = d->max_pages; pv.num_pages = d->num_pages;
+    return pv;
+}
+
+// The KV addressing fields only (chunking is irrelevant to residency operations).
+static hg_status check_pool(const hg_attn_desc* d) {
+    if (!d || d->struct_size < offsetof(hg_attn_desc, sched_counter)) return HG_ERR_INVALID_ARG;
+    hg_attn_desc t;
+    memset(&t, 0, sizeof t);
+    memcpy(&t, d, d->struct_size < sizeof t ? d->struct_size : sizeof t);
+    t.chunk_tokens = t.page_size > TILE_T ? t.page_size : TILE_T;
+    t.num_chunks = 1;
+    t.sched_counter = nullptr;
+    t.struct_size = sizeof t;
+    return check_desc(&t, true);
+}
+
+hg_status hg_kv_append(const void* k_new, const void* v_new, void* k_cache, void* v_cache, int32_t* seq_lens,
+                       int32_t* tok_end, void* stream, const hg_attn_desc* desc) {
+    hg_status st = check_pool(desc);
+    if (st != HG_OK) return st;
+    if (!k_new || !v_new || !k_cache || !v_cache || !seq_lens) return HG_ERR_INVALID_ARG;
+    if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_cache) || !aligned16(v_cache)) return HG_ERR_INVALID_ARG;
+    kv_append_kernel<<<desc->batch, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        pool_view(desc, k_cache, v_cache), static_cast<const uint16_t*>(k_new), static_cast<const uint16_t*>(v_new),
+        seq_lens, tok_end, desc->status);
+    return cudaGetLastError() == cudaSuccess ? HG_OK : HG_ERR_CUDA;
+}
+
+hg_status hg_kv_evict(const void* k_cache, const void* v_cache, int32_t* tok_begin, const int32_t* tok_end,
+                      const int32_t* n_evict, int32_t max_evict, void* k_out, void* v_out, int32_t* freed_pages,
+                      int32_t* n_freed, int32_t max_freed, void* stream, const hg_attn_desc* desc) {
+    hg_status st = check_pool(desc);
+    if (st != HG_OK) return st;
+    if (!k_cache || !v_cache || !tok_begin || !tok_end || !n_evict || !k_out || !v_out) return HG_ERR_INVALID_ARG;
+    if (max_evict < 1 || max_freed < 0 || (freed_pages && max_freed < 1)) return HG_ERR_INVALID_ARG;
+    if (!aligned16(k_cache) || !aligned16(v_cache) || !aligned16(k_out) || !aligned16(v_out)) return HG_ERR_INVALID_ARG;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const KvPoolView pv = pool_view(desc, k_cache, v_cache);
+    dim3 grid((unsigned)((max_evict + 31) / 32), (unsigned)desc->batch);
+    kv_evict_copy_kernel<<<grid, 256, 0, cs>>>(pv, tok_begin, tok_end, n_evict, static_cast<uint16_t*>(k_out),
+                                                static_cast<uint16_t*>(v_out), max_evict, desc->status);
+    if (cudaGetLastError() != cudaSuccess) return HG_ERR_CUDA;
+    kv_evict_commit_kernel<<<(desc->batch + 127) / 128, 128, 0, cs>>>(
+        desc->batch, pv.page_shift, desc->max_pages, tok_begin, tok_end, n_evict, max_evict,
+        const_cast<int32_t*>(desc->block_table), freed_pages, n_freed, max_freed);
+    return cudaGetLastError() == cudaSuccess ? HG_OK : HG_ERR_CUDA;
 }
 
 const char* hg_status_string(hg_status s) {

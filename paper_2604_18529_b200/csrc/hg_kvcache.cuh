@@ -1,0 +1,110 @@
+// KV residency operations on the paged pool (sm_100a): appending the current step's K/V rows and
+// moving the oldest tokens of the GPU slice out (the eviction engine's device half).  Pure data
+// movement: 16-byte vector copies, no arithmetic.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace hg {
+
+struct KvPoolView {
+    uint16_t* k;
+    uint16_t* v;
+    const int32_t* block_table;   // may be NULL: identity paging
+    int64_t page_stride, head_stride, tok_stride;
+    int B, Hkv, D, page_size, page_shift, max_pages, num_pages;
+};
+
+// Physical page of token t of sequence b, or -1 if it is not resident / out of range.
+__device__ __forceinline__ int kv_page_of(const KvPoolView& pv, int b, int t) {
+    const int pg = t >> pv.page_shift;
+    if (t < 0 || pg >= pv.max_pages) return -1;
+    const int phys = pv.block_table ? pv.block_table[(size_t)b * pv.max_pages + pg] : b * pv.max_pages + pg;
+    return (phys < 0 || phys >= pv.num_pages) ? -1 : phys;
+}
+
+// One CTA per sequence: rows k_new / v_new [B][Hkv][D] go to position seq_lens[b]; then seq_lens[b]
+// (and tok_end[b], if given and equal to the old length) grow by one.
+__global__ void kv_append_kernel(KvPoolView pv, const uint16_t* __restrict__ k_new, const uint16_t* __restrict__ v_new,
+                                 int32_t* seq_lens, int32_t* tok_end, int32_t* status) {
+    const int b = blockIdx.x;
+    const int t = seq_lens[b];
+    const int old_end = tok_end ? tok_end[b] : 0;
+    const int phys = kv_page_of(pv, b, t);
+    __syncthreads();                                   // everybody has read the old length
+    if (phys < 0) {
+        if (threadIdx.x == 0 && status) atomicMax(status, HG_DEV_BAD_PAGE);
+        return;
+    }
+    const int vec_per_row = pv.D / 8;                  // 16-byte vectors
+    const int64_t base = (int64_t)phys * pv.page_stride + (int64_t)(t & (pv.page_size - 1)) * pv.tok_stride;
+    for (int i = threadIdx.x; i < pv.Hkv * vec_per_row; i += blockDim.x) {
+        const int g = i / vec_per_row, c = i - g * vec_per_row;
+        const int64_t dst = base + (int64_t)g * pv.head_stride + c * 8;
+        const int64_t src = ((int64_t)b * pv.Hkv + g) * pv.D + c * 8;
+        *reinterpret_cast<uint4*>(pv.k + dst) = *reinterpret_cast<const uint4*>(k_new + src);
+        *reinterpret_cast<uint4*>(pv.v + dst) = *reinterpret_cast<const uint4*>(v_new + src);
+    }
+    if (threadIdx.x == 0) {
+        seq_lens[b] = t + 1;
+        if (tok_end && old_end == t) tok_end[b] = t + 1;
+    }
+}
+
+// Copies the first n_evict[b] tokens of the slice [tok_begin, tok_end) of every sequence into
+// k_out / v_out [B][max_evict][Hkv][D] (token-major rows, the layout the host keeps its part in).
+// Grid (token blocks, B); reads only.
+__global__ void kv_evict_copy_kernel(KvPoolView pv, const int32_t* __restrict__ tok_begin, const int32_t* __restrict__ tok_end,
+                                     const int32_t* __restrict__ n_evict, uint16_t* k_out, uint16_t* v_out, int max_evict,
+                                     int32_t* status) {
+    const int b = blockIdx.y;
+    const int tb = tok_begin[b];
+    const int ne = max(0, min(min(n_evict[b], max_evict), tok_end[b] - tb));
+    const int vec_per_row = pv.D / 8, vec_per_tok = pv.Hkv * vec_per_row;
+    const int tok_per_cta = 32;
+    const int i0 = blockIdx.x * tok_per_cta, i1 = min(ne, i0 + tok_per_cta);
+    for (int idx = threadIdx.x + i0 * vec_per_tok; idx < i1 * vec_per_tok; idx += blockDim.x) {
+        const int i = idx / vec_per_tok, r = idx - i * vec_per_tok;
+        const int g = r / vec_per_row, c = r - g * vec_per_row;
+        const int t = tb + i;
+        const int phys = kv_page_of(pv, b, t);
+        if (phys < 0) { if (status) atomicMax(status, HG_DEV_BAD_PAGE); continue; }
+        const int64_t src = (int64_t)phys * pv.page_stride + (int64_t)(t & (pv.page_size - 1)) * pv.tok_stride +
+                            (int64_t)g * pv.head_stride + c * 8;
+        const int64_t dst = (((int64_t)b * max_evict + i) * pv.Hkv + g) * pv.D + c * 8;
+        *reinterpret_cast<uint4*>(k_out + dst) = *reinterpret_cast<const uint4*>(pv.k + src);
+        *reinterpret_cast<uint4*>(v_out + dst) = *reinterpret_cast<const uint4*>(pv.v + src);
+    }
+}
+
+// After the copy: advances tok_begin, un-maps the pages that no longer hold a token of the slice and lists
+// their physical ids in freed [B][max_freed] (-1 padded), n_freed [B].  One thread per sequence.
+__global__ void kv_evict_commit_kernel(int B, int page_shift, int max_pages, int32_t* tok_begin, const int32_t* tok_end,
+                                       const int32_t* n_evict, int max_evict, int32_t* block_table, int32_t* freed,
+                                       int32_t* n_freed, int max_freed) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const int tb = tok_begin[b], te = tok_end[b];
+    const int ne = max(0, min(min(n_evict[b], max_evict), te - tb));
+    const int nb = tb + ne;
+    // pages wholly below the new beginning leave; a partly used page stays mapped (it may still take appended rows)
+    const int first_pg = tb >> page_shift;
+    const int last_pg = nb >> page_shift;
+    int cnt = 0;
+    for (int pg = first_pg; pg < last_pg && pg < max_pages; ++pg) {
+        if (block_table) {
+            const int phys = block_table[(size_t)b * max_pages + pg];
+            if (phys >= 0) {
+                if (freed && cnt < max_freed) freed[(size_t)b * max_freed + cnt] = phys;
+                ++cnt;
+                block_table[(size_t)b * max_pages + pg] = -1;
+            }
+        }
+    }
+    if (freed) for (int i = cnt; i < max_freed; ++i) freed[(size_t)b * max_freed + i] = -1;
+    if (n_freed) n_freed[b] = cnt;
+    tok_begin[b] = nb;
+}
+
+}  // namespace hg
