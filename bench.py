@@ -73,7 +73,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "25"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -172,6 +172,81 @@ def time_oracle(w, device, target_core_seconds=20.0):
                       f"chunked PARTIAL + MERGE in fp64, {dt:.2f} s"}, items, tokens
 
 
+def time_extras(w, prob, dev, steps):
+    """The widened entry points on the same shapes: the CPU -> GPU hand-off (K_sel selected host tokens per
+    sequence), the host logits calculator feeding it, and the residency operations."""
+    import statistics as st
+    import torch
+    import paper_2604_18529_b200 as pkg
+    from paper_2604_18529_b200 import host as H
+
+    def dev_us(fn, n):
+        for _ in range(3):
+            fn()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        for a, b in ev:
+            a.record(); fn(); b.record()
+        torch.cuda.synchronize()
+        return st.mean(a.elapsed_time(b) for a, b in ev) * 1e3
+
+    out = {}
+    dt = {"f16": torch.float16, "bf16": torch.bfloat16}[w.dtype]
+    gen = torch.Generator(device=dev).manual_seed(7)
+    # ---- hand-off: logits [B][Hq][K] + V rows [B][Hkv][K][D] -> partials
+    K_sel, chunk = 1024, 256
+    logits = torch.randn(w.B, w.Hq, K_sel, device=dev, generator=gen)
+    vrows = torch.randn(w.B, w.Hkv, K_sel, w.D, device=dev, generator=gen).to(dt)
+    n_sel = torch.full((w.B,), K_sel, dtype=torch.int32, device=dev)
+    ld = pkg.logits_desc(batch=w.B, num_q_heads=w.Hq, num_kv_heads=w.Hkv, head_dim=w.D, dtype=w.dtype, max_selected=K_sel,
+                         chunk_tokens=chunk)
+    ho = torch.empty(w.B, w.Hq, ld.num_chunks, w.D, device=dev); hm = torch.empty(w.B, w.Hq, ld.num_chunks, device=dev)
+    hl = torch.empty_like(hm)
+    us = dev_us(lambda: pkg.hg_attn_partial_from_logits(logits, vrows, n_sel, ho, hm, hl, ld), steps)
+    nbytes = logits.numel() * 4 + vrows.numel() * 2
+    out["handoff"] = {"selected_per_seq": K_sel, "us": us, "gbs": nbytes / us / 1e3}
+    # ---- host logits calculator: every host-held token of the first sequence(s), all heads
+    n_host = min(w.tok_begin[0], 16384)
+    if n_host > 0:
+        Bh = min(w.B, 2)
+        k_host = torch.randn(Bh, n_host, w.Hkv, w.D).to(dt)
+        q_host = torch.randn(Bh, w.Hq, w.D).to(dt)
+        lg = torch.empty(Bh, w.Hq, n_host)
+        nh = torch.full((Bh,), n_host, dtype=torch.int32)
+        d = H.host_desc(k_host, w.Hq, n_host)
+        H.hg_host_logits(q_host, k_host, None, nh, lg, d)
+        t0 = time.perf_counter()
+        reps = 3
+        for _ in range(reps):
+            H.hg_host_logits(q_host, k_host, None, nh, lg, d)
+        sec = (time.perf_counter() - t0) / reps
+        out["host_logits"] = {"tokens": Bh * n_host, "q_heads": w.Hq, "ms": sec * 1e3,
+                              "gflops": 2.0 * Bh * n_host * w.Hq * w.D / sec / 1e9,
+                              "k_gbs": Bh * n_host * w.Hkv * w.D * 2 / sec / 1e9, "cores": len(os.sched_getaffinity(0))}
+    # ---- residency: evict 1024 oldest tokens per sequence into staging (state is restored between runs)
+    max_evict = 1024
+    k_out = torch.empty(w.B, max_evict, w.Hkv, w.D, dtype=dt, device=dev); v_out = torch.empty_like(k_out)
+    ne = torch.full((w.B,), max_evict, dtype=torch.int32, device=dev)
+    tb0 = prob.tok_begin.clone()
+    table0 = None if prob.kv["block_table"] is None else prob.kv["block_table"].clone()
+
+    def evict():
+        prob.tok_begin.copy_(tb0)
+        if table0 is not None:
+            prob.kv["block_table"].copy_(table0)
+        pkg.hg_kv_evict(prob.kv["k"], prob.kv["v"], prob.tok_begin, prob.tok_end, ne, k_out, v_out, None, None, prob.desc)
+
+    def restore_only():
+        prob.tok_begin.copy_(tb0)
+        if table0 is not None:
+            prob.kv["block_table"].copy_(table0)
+
+    us = dev_us(evict, steps) - dev_us(restore_only, steps)
+    restore_only()
+    moved = 2 * 2 * w.B * max_evict * w.Hkv * w.D * 2                 # K and V, read + written
+    out["kv_evict"] = {"tokens_per_seq": max_evict, "us": us, "gbs": moved / us / 1e3}
+    return out
+
+
 def run_reference(args, rank, world):
     """--impl reference: the fp64 oracle on the host cores, each step a bounded sample of the workload."""
     if rank != 0:
@@ -210,6 +285,8 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="keep only the first BATCH sequences (small profiling captures)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--probe", action="store_true", help="also time the read-probe kernel")
+    ap.add_argument("--extras", action="store_true",
+                    help="also time the hand-off kernel, the host logits calculator and the residency operations")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -322,6 +399,7 @@ def main():
         torch.cuda.synchronize()
         probe_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in pe)
 
+    extras = time_extras(w, prob, dev, args.steps) if args.extras and rank == 0 else None
     ms_total, e2e_ms = max_over_ranks([ms_total, e2e_ms], dev)
 
     if rank == 0:
@@ -346,7 +424,7 @@ def main():
                        "step_frac_of_8000": prob.alg_bytes() / (ms_step * 1e-3) / 1e9 / 8000.0,
                        "partial_us": part_avg * 1e3, "merge_us": statistics.mean(merge_ms) * 1e3,
                        "roofline_timing": "second pass of K steps with CUDA events around each kernel",
-                       "probe_us": None if probe_ms is None else probe_ms * 1e3},
+                       "probe_us": None if probe_ms is None else probe_ms * 1e3, "extras": extras},
             "roofline": {"bound": "hbm", "kernel": "partial_kernel", "achieved": achieved, "peak": peak,
                          "peak_kind": f"{peak_kind} copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
                          "frac_of_8000": achieved / 8000.0, "alg_bytes_per_launch": part_alg,
