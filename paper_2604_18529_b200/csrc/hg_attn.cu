@@ -20,6 +20,8 @@
 
 namespace hg {
 
+constexpr int kMaxDevices = 64;
+
 // ---- validation ------------------------------------------------------------------------------------
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -115,27 +117,41 @@ static int env_int(const char* name, int dflt, int lo, int hi) {
     return v < lo ? lo : (v > hi ? hi : v);
 }
 
+// Per kernel instantiation and device: the shared-memory opt-in that is in force and the occupancy it gives.
+// Looked up once per (device, size); racing threads would store the same values.
+struct LaunchCache {
+    std::atomic<int> smem[kMaxDevices];
+    std::atomic<int> per_sm[kMaxDevices];
+    std::atomic<int> sms[kMaxDevices];
+};
+
 template <int D, bool BF16, int MODE>
 static hg_status launch_partial_t(const CUtensorMap& tk, const CUtensorMap& tv, PartialParams p, cudaStream_t st) {
+    static LaunchCache cache;                     // zero-initialised
     const size_t smem = (size_t)p.stages * (2 * TILE_T * D * 2 + 8 * D * 2) + 1024;     // per stage: K tile, V tile, q rows
     auto kern = partial_kernel<D, BF16, MODE>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
-        cudaGetLastError();
-        return HG_ERR_CUDA;
-    }
-    const int Y = p.Hkv * p.head_blocks;
-    dim3 grid((unsigned)p.NC, (unsigned)Y, (unsigned)p.B);
-    if (p.persistent) {
-        // one wave of resident CTAs; each takes items round-robin
-        int dev = 0, sms = 0, per_sm = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return HG_ERR_CUDA; }
+    if (cache.smem[dev].load(std::memory_order_acquire) != (int)smem) {
+        int sms = 0, per_sm = 0;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
             cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, THREADS, smem) != cudaSuccess || per_sm < 1) {
             cudaGetLastError();
             return HG_ERR_CUDA;
         }
+        cache.sms[dev].store(sms, std::memory_order_relaxed);
+        cache.per_sm[dev].store(per_sm, std::memory_order_relaxed);
+        cache.smem[dev].store((int)smem, std::memory_order_release);
+    }
+    const int Y = p.Hkv * p.head_blocks;
+    dim3 grid((unsigned)p.NC, (unsigned)Y, (unsigned)p.B);
+    if (p.persistent) {
+        // one wave of resident CTAs; each takes items from the schedule
+        int per_sm = cache.per_sm[dev].load(std::memory_order_relaxed);
         per_sm = env_int("HG_ATTN_CTAS_PER_SM", per_sm, 1, per_sm);
         const long long slots = (long long)p.NC * Y * p.B;
-        const long long resident = (long long)sms * per_sm;
+        const long long resident = (long long)cache.sms[dev].load(std::memory_order_relaxed) * per_sm;
         grid = dim3((unsigned)(slots < resident ? slots : resident), 1, 1);
     }
     kern<<<grid, THREADS, smem, st>>>(tk, tv, p);
@@ -482,13 +498,12 @@ uint32_t hg_version(void) { return HG_VERSION; }
 // device address: the address is obtained once per device with cudaGetSymbolAddress.
 static __device__ __align__(256) unsigned char hg_static_scratch[HG_STATIC_SCRATCH_BYTES];
 
-constexpr int kMaxDevices = 64;
-static std::atomic<void*> g_static_scratch_addr[kMaxDevices];
+static std::atomic<void*> g_static_scratch_addr[hg::kMaxDevices];
 
 // Device address of the scratch array on the current device (looked up on the first call per device).
 static void* static_scratch_ptr() {
     int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return nullptr; }
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= hg::kMaxDevices) { cudaGetLastError(); return nullptr; }
     void* p = g_static_scratch_addr[dev].load(std::memory_order_acquire);
     if (p) return p;
     void* addr = nullptr;

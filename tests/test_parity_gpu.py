@@ -328,3 +328,39 @@ def test_stalled_loader_times_out_with_a_status_and_the_context_stays_usable(G):
     torch.cuda.synchronize()
     assert int(prob.status.item()) == hg.HG_DEV_OK
     check_output(prob.out, prob.lse, ref.out, ref.lse)
+
+
+# ---- the decode call sequence can be captured in a CUDA graph and replayed ------------------------------------------
+
+@pytest.mark.parametrize("G", [1, 4])
+def test_decode_replays_from_a_cuda_graph(G):
+    w = wl(Hq=2 * G, Hkv=2)
+    ref = OracleRef(w)
+    prob = DeviceProblem(w, DEV)
+    host = ref.host_partials_device(DEV)
+    ws = torch.empty(pkg.hg_attn_workspace_bytes(prob.desc, 2), dtype=torch.uint8, device=DEV)
+    out = torch.empty_like(prob.out); lse = torch.empty_like(prob.lse)
+    call = lambda: pkg.hg_attn_decode(prob.q, prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end,
+                                      host, out, lse, ws, prob.desc)
+    call()                                            # warm up outside the capture (first-use set-up of the kernels)
+    torch.cuda.synchronize()
+    want_out, want_lse = out.clone(), lse.clone()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            call()
+    for _ in range(3):
+        out.fill_(float("nan")); lse.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, want_out) and torch.equal(lse, want_lse)
+    # device-resident ranges: the same graph follows a changed slice without re-capture
+    prob.tok_begin += 64
+    ref2 = OracleRef(dataclasses.replace(w, tok_begin=[t + 64 for t in w.tok_begin]))
+    for dst, src in zip(host, ref2.host_partials_device(DEV)):
+        for a, b in zip(dst, src):
+            a.copy_(b)
+    graph.replay()
+    torch.cuda.synchronize()
+    check_output(out, lse, ref2.out, ref2.lse, "replayed on a moved slice")
