@@ -227,22 +227,42 @@ static hg_status run_merge(const hg_partial_src* src, int32_t n_src, float* out,
     }
     p.n_src = n_src; p.out = out; p.lse = lse;
 
+    // long rows and few of them: a cluster of 2, 4 or 8 CTAs splits each row's partials, as long as the grid
+    // stays within a few CTAs per SM
+    const int rows = d->batch * d->num_q_heads;
+    int cluster = 1;
+    if (p.total > 64 && env_int("HG_ATTN_MERGE_CLUSTER", 1, 0, 1)) cluster = rows <= 64 ? 8 : (rows <= 128 ? 4 : (rows <= 256 ? 2 : 1));
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
-    cfg.gridDim = dim3((unsigned)(d->batch * d->num_q_heads));
-    const bool wide = p.total > 64;                              // long rows: 32 warps per row
-    cfg.blockDim = dim3(wide ? 1024 : 256);
+    cfg.gridDim = dim3((unsigned)(rows * cluster));
+    const bool big_cta = cluster == 1 && p.total > 64;             // many long rows: 32 warps per row instead
+    cfg.blockDim = dim3(big_cta ? 1024 : 256);
     cfg.stream = static_cast<cudaStream_t>(stream);
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;     // start while the producer of the partials drains
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    if (env_int("HG_ATTN_PDL", 1, 0, 1)) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;     // start while the producer of the partials drains
+        ++na;
+    }
+    if (cluster > 1) {
+        attr[na].id = cudaLaunchAttributeClusterDimension;
+        attr[na].val.clusterDim.x = (unsigned)cluster; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;
+        ++na;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = env_int("HG_ATTN_PDL", 1, 0, 1);
+    cfg.numAttrs = na;
+    auto launch = [&](auto k128, auto k64) { return d->head_dim == 128 ? cudaLaunchKernelEx(&cfg, k128, p) : cudaLaunchKernelEx(&cfg, k64, p); };
     cudaError_t e;
-    if (d->head_dim == 128)
-        e = wide ? cudaLaunchKernelEx(&cfg, merge_kernel<128, 1024>, p) : cudaLaunchKernelEx(&cfg, merge_kernel<128, 256>, p);
-    else
-        e = wide ? cudaLaunchKernelEx(&cfg, merge_kernel<64, 1024>, p) : cudaLaunchKernelEx(&cfg, merge_kernel<64, 256>, p);
+    switch (cluster) {
+        case 8: e = launch(merge_kernel<128, 256, 8>, merge_kernel<64, 256, 8>); break;
+        case 4: e = launch(merge_kernel<128, 256, 4>, merge_kernel<64, 256, 4>); break;
+        case 2: e = launch(merge_kernel<128, 256, 2>, merge_kernel<64, 256, 2>); break;
+        default:
+            e = big_cta ? launch(merge_kernel<128, 1024, 1>, merge_kernel<64, 1024, 1>)
+                        : launch(merge_kernel<128, 256, 1>, merge_kernel<64, 256, 1>);
+            break;
+    }
     if (e != cudaSuccess) { cudaGetLastError(); return HG_ERR_CUDA; }
     return HG_OK;
 }

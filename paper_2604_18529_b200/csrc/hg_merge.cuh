@@ -1,12 +1,15 @@
 // Log-sum-exp merge of softmax partials and final normalisation (sm_100a).
 //
-// One CTA per (sequence, query head), 8 or 32 warps depending on how many partials a row has.  Pass 1
-// finds M = max_i m_i over every partial of every source; pass 2 accumulates w_i * o_i and w_i * l_i
-// with w_i = e^{m_i - M}, each warp taking every W-th partial (four loads in flight) and each lane D/32
-// contiguous output components; a fixed-order cross-warp sum and one division finish
-// out = sum w o / sum w l and lse = M + ln sum w l.  No atomics: bit-reproducible.
+// One CTA of 8 warps per (sequence, query head) - or, when a row has many partials, a thread-block
+// cluster of CLUSTER such CTAs that split the row's partials and combine through distributed shared
+// memory.  Pass 1 finds M = max_i m_i over every partial of every source; pass 2 accumulates
+// w_i * o_i and w_i * l_i with w_i = e^{m_i - M}, each warp taking every W-th partial (four loads in
+// flight) and each lane D/32 contiguous output components; fixed-order sums across warps and across
+// the cluster's CTAs and one division finish out = sum w o / sum w l and lse = M + ln sum w l.
+// No atomics: bit-reproducible for a given launch shape.
 #pragma once
 
+#include <cooperative_groups.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -25,15 +28,20 @@ struct MergeParams {
     float* lse;
 };
 
-template <int D, int THREADS_>
+template <int D, int THREADS_, int CLUSTER>
 __global__ void __launch_bounds__(THREADS_) merge_kernel(const MergeParams p) {
+    namespace cg = cooperative_groups;
     constexpr int VEC = D / 32;
     constexpr int WARPS = THREADS_ / 32;
     __shared__ float s_max[WARPS];
     __shared__ float s_l[WARPS];
     __shared__ float s_o[WARPS][D];
+    __shared__ float s_cta_max;                 // this CTA's share, read by its cluster peers
+    __shared__ float s_cta_l;
+    __shared__ float s_cta_o[D];
     const float NEG_INF = __int_as_float(0xff800000);
-    const int row = blockIdx.x;                 // b * Hq + h
+    const int row = blockIdx.x / CLUSTER;       // b * Hq + h
+    const int rank = blockIdx.x % CLUSTER;      // position in the cluster
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
 #if __CUDA_ARCH__ >= 900
@@ -44,7 +52,7 @@ __global__ void __launch_bounds__(THREADS_) merge_kernel(const MergeParams p) {
     float mx = NEG_INF;
     for (int s = 0; s < p.n_src; ++s) {
         const float* ms = p.m[s] + (size_t)row * p.nc[s];
-        for (int i = tid; i < p.nc[s]; i += THREADS_) mx = fmaxf(mx, ms[i]);
+        for (int i = rank * THREADS_ + tid; i < p.nc[s]; i += CLUSTER * THREADS_) mx = fmaxf(mx, ms[i]);
     }
 #pragma unroll
     for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
@@ -53,6 +61,13 @@ __global__ void __launch_bounds__(THREADS_) merge_kernel(const MergeParams p) {
     float M = s_max[0];
 #pragma unroll
     for (int w = 1; w < WARPS; ++w) M = fmaxf(M, s_max[w]);
+    if constexpr (CLUSTER > 1) {
+        cg::cluster_group cluster = cg::this_cluster();
+        if (tid == 0) s_cta_max = M;
+        cluster.sync();
+#pragma unroll
+        for (int r = 0; r < CLUSTER; ++r) M = fmaxf(M, *cluster.map_shared_rank(&s_cta_max, r));
+    }
 
     // ---- pass 2: weighted sums ----------------------------------------------------------------------
     float acc[VEC];
@@ -65,11 +80,11 @@ __global__ void __launch_bounds__(THREADS_) merge_kernel(const MergeParams p) {
             const float* ms = p.m[s] + (size_t)row * nc;
             const float* ls = p.l[s] + (size_t)row * nc;
             const float* os = p.o[s] + (size_t)row * nc * D;
-            for (int i0 = warp; i0 < nc; i0 += 4 * WARPS) {
+            for (int i0 = rank * WARPS + warp; i0 < nc; i0 += 4 * CLUSTER * WARPS) {
                 float mi[4], li[4], ov[4][VEC];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {                  // four independent partials in flight
-                    const int i = i0 + u * WARPS;
+                    const int i = i0 + u * CLUSTER * WARPS;
                     const bool in = i < nc;
                     mi[u] = in ? ms[i] : NEG_INF;
                     li[u] = in ? ls[i] : 0.f;
@@ -98,10 +113,28 @@ __global__ void __launch_bounds__(THREADS_) merge_kernel(const MergeParams p) {
     for (int v = 0; v < VEC; ++v) s_o[warp][lane * VEC + v] = acc[v];
     __syncthreads();
 
+    float Lsum = 0.f, o = 0.f;
     if (tid < D) {
-        float Lsum = 0.f, o = 0.f;
 #pragma unroll
         for (int w = 0; w < WARPS; ++w) { Lsum += s_l[w]; o += s_o[w][tid]; }
+    }
+    if constexpr (CLUSTER > 1) {
+        cg::cluster_group cluster = cg::this_cluster();
+        if (tid < D) s_cta_o[tid] = o;
+        if (tid == 0) s_cta_l = Lsum;
+        cluster.sync();
+        if (rank == 0 && tid < D) {
+            Lsum = 0.f; o = 0.f;
+#pragma unroll
+            for (int r = 0; r < CLUSTER; ++r) {
+                Lsum += *cluster.map_shared_rank(&s_cta_l, r);
+                o += cluster.map_shared_rank(&s_cta_o[0], r)[tid];
+            }
+        }
+        cluster.sync();                         // peers keep their shared memory alive until rank 0 has read it
+        if (rank != 0) return;
+    }
+    if (tid < D) {
         const bool empty = (M == NEG_INF);
         p.out[(size_t)row * D + tid] = empty ? 0.f : o / Lsum;
         if (tid == 0 && p.lse) p.lse[row] = empty ? NEG_INF : M + logf(Lsum);

@@ -364,3 +364,33 @@ def test_decode_replays_from_a_cuda_graph(G):
     graph.replay()
     torch.cuda.synchronize()
     check_output(out, lse, ref2.out, ref2.lse, "replayed on a moved slice")
+
+
+# ---- seeded random sweep over everything at once ---------------------------------------------------------------------
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_shapes(seed):
+    rng = np.random.default_rng(1000 + seed)
+    B = int(rng.integers(1, 6))
+    Hkv = int(rng.choice([1, 2, 3]))
+    G = int(rng.choice([1, 1, 2, 4, 5, 8, 9, 16]))
+    D = int(rng.choice([64, 128]))
+    page = int(rng.choice([16, 32, 64, 128]))
+    layout, paged = [("HND", True), ("NHD", True), ("NHD", False)][int(rng.integers(0, 3))]
+    chunk = int(rng.choice([64, 128, 256, 512]))
+    chunk = max(chunk, page)
+    lens = [int(rng.integers(1, 1400)) for _ in range(B)]
+    tb, te = [], []
+    for L in lens:
+        kind = rng.integers(0, 5)
+        if kind == 0:
+            a = e = int(rng.integers(0, L + 1))                   # empty slice
+        elif kind == 1:
+            a, e = 0, L                                           # whole sequence on the GPU
+        else:
+            a = int(rng.integers(0, L)); e = int(rng.integers(a, L + 1))
+        tb.append(a); te.append(e)
+    w = W.AttnWorkload(f"rand{seed}", B, Hkv * G, Hkv, D, str(rng.choice(["f16", "bf16"])), lens, tb, te, page_size=page,
+                       layout=layout, paged=paged, chunk_tokens=chunk, seed=2000 + seed,
+                       sigma_kv=float(rng.choice([0.5, 1.0, 2.0])), outlier_frac=float(rng.choice([0.0, 0.02])))
+    run_and_check(w, poison_tail=bool(rng.integers(0, 2)), what=repr(w))
