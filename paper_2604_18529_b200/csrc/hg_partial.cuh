@@ -153,8 +153,11 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
     // means: do not queue behind it), and this CTA's second work item (its first is its own block index).
     const int32_t status_at_entry = p.status ? *reinterpret_cast<volatile int32_t*>(p.status) : HG_DEV_OK;
     int early_request = 0;
-    if (p.persistent && p.sched && tid == CONSUMER_THREADS && !p.test_stall)
-        early_request = (int)gridDim.x + atomicAdd(p.sched, 1);
+    if (tid == CONSUMER_THREADS) {
+        prefetch_tensormap(&tmK);                    // the descriptors are on their way long before the first load
+        prefetch_tensormap(&tmV);
+        if (p.persistent && p.sched && !p.test_stall) early_request = (int)gridDim.x + atomicAdd(p.sched, 1);
+    }
 
     // ---- set-up: barriers, and for the persistent schedule the item counts per sequence ---------------
     if (tid == 0) {
@@ -250,8 +253,6 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
 
     if (warp == CONSUMER_WARPS) {
         // =============================== producer warp ===============================
-        prefetch_tensormap(&tmK);
-        prefetch_tensormap(&tmV);
         const uint64_t policy = l2_evict_first_policy();
         const int nbox = TILE_T >> rshift;           // boxes per tile: 4, 2 or 1
         const int j = lane & (nbox - 1);             // this lane's box
