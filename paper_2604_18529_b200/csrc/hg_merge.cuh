@@ -2,11 +2,12 @@
 //
 // One CTA of 8 warps per (sequence, query head) - or, when a row has many partials, a thread-block
 // cluster of CLUSTER such CTAs that split the row's partials and combine through distributed shared
-// memory.  Pass 1 finds M = max_i m_i over every partial of every source; pass 2 accumulates
-// w_i * o_i and w_i * l_i with w_i = e^{m_i - M}, each warp taking every W-th partial (four loads in
-// flight) and each lane D/32 contiguous output components; fixed-order sums across warps and across
-// the cluster's CTAs and one division finish out = sum w o / sum w l and lse = M + ln sum w l.
-// No atomics: bit-reproducible for a given launch shape.
+// memory.  One sweep: each warp takes every W-th partial (four loads in flight), keeps a running
+// maximum M_w and the sums of w_i * o_i and w_i * l_i with w_i = e^{m_i - M_w}, rescaling them when
+// M_w grows; each lane holds D/32 contiguous output components.  The warps' triples, then the
+// cluster's CTAs' triples, are combined the same way in fixed order, and one division finishes
+// out = sum w o / sum w l and lse = M + ln sum w l.  No atomics: bit-reproducible for a given launch
+// shape.
 #pragma once
 
 #include <cooperative_groups.h>
@@ -33,10 +34,10 @@ __global__ void __launch_bounds__(THREADS_) merge_kernel(const MergeParams p) {
     namespace cg = cooperative_groups;
     constexpr int VEC = D / 32;
     constexpr int WARPS = THREADS_ / 32;
-    __shared__ float s_max[WARPS];
+    __shared__ float s_m[WARPS];
     __shared__ float s_l[WARPS];
     __shared__ float s_o[WARPS][D];
-    __shared__ float s_cta_max;                 // this CTA's share, read by its cluster peers
+    __shared__ float s_cta_m;                   // this CTA's share, read by its cluster peers
     __shared__ float s_cta_l;
     __shared__ float s_cta_o[D];
     const float NEG_INF = __int_as_float(0xff800000);
@@ -48,87 +49,89 @@ __global__ void __launch_bounds__(THREADS_) merge_kernel(const MergeParams p) {
     cudaGridDependencySynchronize();            // partials may come from the kernel launched just before
 #endif
 
-    // ---- pass 1: global maximum -------------------------------------------------------------------
-    float mx = NEG_INF;
-    for (int s = 0; s < p.n_src; ++s) {
-        const float* ms = p.m[s] + (size_t)row * p.nc[s];
-        for (int i = rank * THREADS_ + tid; i < p.nc[s]; i += CLUSTER * THREADS_) mx = fmaxf(mx, ms[i]);
-    }
-#pragma unroll
-    for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    if (lane == 0) s_max[warp] = mx;
-    __syncthreads();
-    float M = s_max[0];
-#pragma unroll
-    for (int w = 1; w < WARPS; ++w) M = fmaxf(M, s_max[w]);
-    if constexpr (CLUSTER > 1) {
-        cg::cluster_group cluster = cg::this_cluster();
-        if (tid == 0) s_cta_max = M;
-        cluster.sync();
-#pragma unroll
-        for (int r = 0; r < CLUSTER; ++r) M = fmaxf(M, *cluster.map_shared_rank(&s_cta_max, r));
-    }
-
-    // ---- pass 2: weighted sums ----------------------------------------------------------------------
+    // ---- one sweep: every warp keeps a running maximum and rescales its sums when it grows ----------
     float acc[VEC];
 #pragma unroll
     for (int v = 0; v < VEC; ++v) acc[v] = 0.f;
-    float lsum = 0.f;
-    if (M != NEG_INF) {
-        for (int s = 0; s < p.n_src; ++s) {
-            const int nc = p.nc[s];
-            const float* ms = p.m[s] + (size_t)row * nc;
-            const float* ls = p.l[s] + (size_t)row * nc;
-            const float* os = p.o[s] + (size_t)row * nc * D;
-            for (int i0 = rank * WARPS + warp; i0 < nc; i0 += 4 * CLUSTER * WARPS) {
-                float mi[4], li[4], ov[4][VEC];
+    float lsum = 0.f, Mw = NEG_INF;
+    for (int s = 0; s < p.n_src; ++s) {
+        const int nc = p.nc[s];
+        const float* ms = p.m[s] + (size_t)row * nc;
+        const float* ls = p.l[s] + (size_t)row * nc;
+        const float* os = p.o[s] + (size_t)row * nc * D;
+        for (int i0 = rank * WARPS + warp; i0 < nc; i0 += 4 * CLUSTER * WARPS) {
+            float mi[4], li[4], ov[4][VEC];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {                  // four independent partials in flight
-                    const int i = i0 + u * CLUSTER * WARPS;
-                    const bool in = i < nc;
-                    mi[u] = in ? ms[i] : NEG_INF;
-                    li[u] = in ? ls[i] : 0.f;
-                    const bool live = in && mi[u] != NEG_INF;  // an empty partial's o is not read
-                    const float* orow = os + (size_t)(in ? i : 0) * D + lane * VEC;
-                    if constexpr (VEC == 4) {
-                        const float4 v = live ? *reinterpret_cast<const float4*>(orow) : make_float4(0.f, 0.f, 0.f, 0.f);
-                        ov[u][0] = v.x; ov[u][1] = v.y; ov[u][2] = v.z; ov[u][3] = v.w;
-                    } else {
-                        const float2 v = live ? *reinterpret_cast<const float2*>(orow) : make_float2(0.f, 0.f);
-                        ov[u][0] = v.x; ov[u][1] = v.y;
-                    }
+            for (int u = 0; u < 4; ++u) {                      // four independent partials in flight
+                const int i = i0 + u * CLUSTER * WARPS;
+                const bool in = i < nc;
+                mi[u] = in ? ms[i] : NEG_INF;
+                li[u] = in ? ls[i] : 0.f;
+                const bool live = in && mi[u] != NEG_INF;      // an empty partial's o is not read
+                const float* orow = os + (size_t)(in ? i : 0) * D + lane * VEC;
+                if constexpr (VEC == 4) {
+                    const float4 v = live ? *reinterpret_cast<const float4*>(orow) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    ov[u][0] = v.x; ov[u][1] = v.y; ov[u][2] = v.z; ov[u][3] = v.w;
+                } else {
+                    const float2 v = live ? *reinterpret_cast<const float2*>(orow) : make_float2(0.f, 0.f);
+                    ov[u][0] = v.x; ov[u][1] = v.y;
                 }
+            }
+            const float m4 = fmaxf(fmaxf(mi[0], mi[1]), fmaxf(mi[2], mi[3]));
+            if (m4 == NEG_INF) continue;                        // four empty partials (warp-uniform)
+            if (m4 > Mw) {
+                const float r = __expf(Mw - m4);                // 0 while Mw is still -inf
+                lsum *= r;
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const float w = mi[u] == NEG_INF ? 0.f : __expf(mi[u] - M);
-                    lsum = fmaf(w, li[u], lsum);
+                for (int v = 0; v < VEC; ++v) acc[v] *= r;
+                Mw = m4;
+            }
 #pragma unroll
-                    for (int v = 0; v < VEC; ++v) acc[v] = fmaf(w, ov[u][v], acc[v]);
-                }
+            for (int u = 0; u < 4; ++u) {
+                const float w = mi[u] == NEG_INF ? 0.f : __expf(mi[u] - Mw);
+                lsum = fmaf(w, li[u], lsum);
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) acc[v] = fmaf(w, ov[u][v], acc[v]);
             }
         }
     }
-    if (lane == 0) s_l[warp] = lsum;
+    if (lane == 0) { s_m[warp] = Mw; s_l[warp] = lsum; }
 #pragma unroll
     for (int v = 0; v < VEC; ++v) s_o[warp][lane * VEC + v] = acc[v];
     __syncthreads();
 
+    // ---- warps of the CTA, in fixed order ---------------------------------------------------------------
+    float M = s_m[0];
+#pragma unroll
+    for (int w = 1; w < WARPS; ++w) M = fmaxf(M, s_m[w]);
     float Lsum = 0.f, o = 0.f;
     if (tid < D) {
 #pragma unroll
-        for (int w = 0; w < WARPS; ++w) { Lsum += s_l[w]; o += s_o[w][tid]; }
+        for (int w = 0; w < WARPS; ++w) {
+            const float r = s_m[w] == NEG_INF ? 0.f : __expf(s_m[w] - M);
+            Lsum = fmaf(r, s_l[w], Lsum);
+            o = fmaf(r, s_o[w][tid], o);
+        }
     }
+    // ---- CTAs of the cluster, in fixed order -------------------------------------------------------------
     if constexpr (CLUSTER > 1) {
         cg::cluster_group cluster = cg::this_cluster();
         if (tid < D) s_cta_o[tid] = o;
-        if (tid == 0) s_cta_l = Lsum;
+        if (tid == 0) { s_cta_l = Lsum; s_cta_m = M; }
         cluster.sync();
         if (rank == 0 && tid < D) {
+            float mr[CLUSTER];
+#pragma unroll
+            for (int r = 0; r < CLUSTER; ++r) mr[r] = *cluster.map_shared_rank(&s_cta_m, r);
+            M = mr[0];
+#pragma unroll
+            for (int r = 1; r < CLUSTER; ++r) M = fmaxf(M, mr[r]);
             Lsum = 0.f; o = 0.f;
 #pragma unroll
             for (int r = 0; r < CLUSTER; ++r) {
-                Lsum += *cluster.map_shared_rank(&s_cta_l, r);
-                o += cluster.map_shared_rank(&s_cta_o[0], r)[tid];
+                const float w = mr[r] == NEG_INF ? 0.f : __expf(mr[r] - M);
+                Lsum = fmaf(w, *cluster.map_shared_rank(&s_cta_l, r), Lsum);
+                o = fmaf(w, cluster.map_shared_rank(&s_cta_o[0], r)[tid], o);
             }
         }
         cluster.sync();                         // peers keep their shared memory alive until rank 0 has read it
