@@ -394,3 +394,34 @@ def test_random_shapes(seed):
                        layout=layout, paged=paged, chunk_tokens=chunk, seed=2000 + seed,
                        sigma_kv=float(rng.choice([0.5, 1.0, 2.0])), outlier_frac=float(rng.choice([0.0, 0.02])))
     run_and_check(w, poison_tail=bool(rng.integers(0, 2)), what=repr(w))
+
+
+# ---- a token set made of several ranges (Section 4.3's position-based choice: sinks + recent window) ----
+
+@pytest.mark.parametrize("G", [1, 4])
+def test_sinks_plus_recent_window_as_two_ranges(G):
+    """Two calls over disjoint ranges of the same pool, merged as two sources, give attention over
+    exactly the union of the ranges."""
+    from oracle import hg_oracle as O
+    L, sinks, window = [1500, 777], 4, [600, 130]
+    w = wl(Hq=2 * G, Hkv=2, seq_lens=L, tok_begin=[0, 0], tok_end=L, chunk_tokens=256, seed=77)
+    prob = DeviceProblem(w, DEV)
+    parts = []
+    for lo, hi in (([0, 0], [sinks, sinks]), ([l - n for l, n in zip(L, window)], L)):
+        o, m, l = torch.empty_like(prob.o_part), torch.empty_like(prob.m_part), torch.empty_like(prob.l_part)
+        hg.hg_attn_partial(prob.q, prob.kv["k"], prob.kv["v"], prob.seq_lens,
+                           torch.tensor(lo, dtype=torch.int32, device=DEV), torch.tensor(hi, dtype=torch.int32, device=DEV),
+                           o, m, l, prob.desc)
+        parts.append((o, m, l))
+    hg.hg_attn_merge(parts, prob.out, prob.lse, prob.desc)
+    torch.cuda.synchronize()
+    assert int(prob.status.item()) == hg.HG_DEV_OK
+    q, K, V = bits(w.q()), bits(w.kv_logical("k")), bits(w.kv_logical("v"))
+    ref_out = np.empty((w.B, w.Hq, w.D)); ref_lse = np.empty((w.B, w.Hq))
+    for b in range(w.B):
+        idx = np.concatenate([np.arange(sinks), np.arange(L[b] - window[b], L[b])]).astype(np.int64)
+        for h in range(w.Hq):
+            g = h // G
+            ref_out[b, h], ref_lse[b, h] = O.full(q[b, h], np.ascontiguousarray(K[b, :, g]), np.ascontiguousarray(V[b, :, g]),
+                                                   w.dtype, idx=idx)
+    check_output(prob.out, prob.lse, ref_out, ref_lse, "sinks + window")
