@@ -177,10 +177,15 @@ hg_status hg_attn_decode(const void* q, const void* k_cache, const void* v_cache
 /*
  * The same pass for a caller whose per-step data lives in HOST memory: q, the three range arrays,
  * the host-slice partials (hg_partial_src with HOST pointers here) and the results out / lse are
- * host buffers (pinned memory makes the copies asynchronous); they are staged through the device
- * workspace with cudaMemcpyAsync on the stream.  The KV pools and the block table stay device
- * resident - they are the GPU's slice of the cache, not per-step input.  Returns after enqueuing;
- * out / lse are valid once the stream has been synchronised.
+ * host buffers.  When every one of them is pinned (or registered) host memory that the device can
+ * address, no copy is enqueued at all: one small kernel stages q and the ranges into the
+ * workspace, the merge reads the host partials and writes out / lse in place over the bus (the
+ * host partial's o must then be 16-byte aligned).  Otherwise - pageable memory, or any buffer the
+ * device cannot address - everything is staged through the device workspace with
+ * cudaMemcpyAsync on the stream.  Either way the buffers are read and written when the stream
+ * reaches the work, not at call time: leave them alone until the stream has been synchronised,
+ * after which out / lse are valid.  The KV pools and the block table stay device resident - they
+ * are the GPU's slice of the cache, not per-step input.  Returns after enqueuing.
  */
 hg_status hg_attn_decode_host(const void* q_host, const void* k_cache, const void* v_cache,
                               const int32_t* seq_lens_host, const int32_t* tok_begin_host,

@@ -17,6 +17,7 @@
 #include "hg_logits.cuh"
 #include "hg_merge.cuh"
 #include "hg_partial.cuh"
+#include "hg_stage.cuh"
 
 namespace hg {
 
@@ -269,6 +270,14 @@ static hg_status run_merge(const hg_partial_src* src, int32_t n_src, float* out,
 
 // ---- workspace layout for the fused entry points ---------------------------------------------------------
 
+// The address at which the current device can read or write a host buffer directly (pinned or registered
+// host memory under unified addressing), or NULL when it cannot (pageable memory, device memory).
+static void* device_alias(const void* host_ptr) {
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, host_ptr) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    return a.type == cudaMemoryTypeHost ? a.devicePointer : nullptr;
+}
+
 static size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct Workspace {
@@ -410,6 +419,42 @@ hg_status hg_attn_decode_host(const void* q_host, const void* k_cache, const voi
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     const size_t rows = (size_t)desc->batch * desc->num_q_heads;
     const int D = desc->head_dim;
+    // Fast path when the device can address every host buffer: one kernel stages q and the ranges, the merge
+    // reads the host partials and writes the results in place - no copy-engine transfers at all.
+    if (env_int("HG_ATTN_HOST_DIRECT", 1, 0, 1) && rows * D * 2 < (1ull << 32)) {
+        StageParams sp;
+        memset(&sp, 0, sizeof sp);
+        const void* in[4] = {q_host, seq_lens_host, tok_begin_host, tok_end_host};
+        const size_t at[4] = {w.q, w.seq_lens, w.tok_begin, w.tok_end};
+        const size_t nb[4] = {rows * D * 2, (size_t)desc->batch * 4, (size_t)desc->batch * 4, (size_t)desc->batch * 4};
+        bool direct = true;
+        for (int i = 0; i < 4 && direct; ++i) {
+            sp.src[i] = device_alias(in[i]); sp.dst[i] = ws + at[i]; sp.bytes[i] = (uint32_t)nb[i];
+            direct = sp.src[i] != nullptr;
+        }
+        sp.n = 4;
+        hg_partial_src alias[HG_MAX_MERGE_SRC];
+        for (int i = 0; i < n_host_src && direct; ++i) {
+            const hg_partial_src& s = host_partials_host[i];
+            alias[i].nc = s.nc; alias[i].reserved = 0;
+            alias[i].o = static_cast<const float*>(device_alias(s.o));
+            alias[i].m = static_cast<const float*>(device_alias(s.m));
+            alias[i].l = static_cast<const float*>(device_alias(s.l));
+            direct = alias[i].o && alias[i].m && alias[i].l && aligned16(alias[i].o);
+        }
+        float* out_alias = direct ? static_cast<float*>(device_alias(out_host)) : nullptr;
+        float* lse_alias = direct && lse_host ? static_cast<float*>(device_alias(lse_host)) : nullptr;
+        direct = direct && out_alias && (!lse_host || lse_alias);
+        if (direct) {
+            const unsigned blocks = (unsigned)((rows * D * 2 / 16 + STAGE_THREADS - 1) / STAGE_THREADS);
+            stage_kernel<<<blocks < 1 ? 1 : (blocks > 64 ? 64 : blocks), STAGE_THREADS, 0, cs>>>(sp);
+            if (cudaGetLastError() != cudaSuccess) return HG_ERR_CUDA;
+            return hg_attn_decode(ws + w.q, k_cache, v_cache, reinterpret_cast<const int32_t*>(ws + w.seq_lens),
+                                  reinterpret_cast<const int32_t*>(ws + w.tok_begin),
+                                  reinterpret_cast<const int32_t*>(ws + w.tok_end), alias, n_host_src, out_alias, lse_alias,
+                                  workspace, workspace_bytes, stream, desc);
+        }
+    }
     bool ok = true;
     ok &= cudaMemcpyAsync(ws + w.q, q_host, rows * D * 2, cudaMemcpyHostToDevice, cs) == cudaSuccess;
     ok &= cudaMemcpyAsync(ws + w.seq_lens, seq_lens_host, (size_t)desc->batch * 4, cudaMemcpyHostToDevice, cs) == cudaSuccess;

@@ -212,6 +212,41 @@ def test_decode_and_decode_host_match_partial_plus_merge(G):
     check_output(out_h, lse_h, ref.out, ref.lse)
 
 
+@pytest.mark.parametrize("how", ["pinned", "pageable", "pinned_copies", "mixed", "unaligned"])
+def test_decode_host_paths_agree(how, monkeypatch):
+    """Pinned host buffers are read and written by the kernels in place; pageable ones (or a mix, or a
+    host partial the merge cannot read with 16-byte loads) go through staged copies.  Same bits either way."""
+    w = wl(Hq=8, Hkv=2, seq_lens=[900, 411], tok_begin=[77, 0], tok_end=[900, 300])
+    ref = OracleRef(w)
+    prob = DeviceProblem(w, DEV)
+    host_dev = ref.host_partials_device(DEV)
+    prob.step(host_dev)
+    torch.cuda.synchronize()
+    if how == "pinned_copies":
+        monkeypatch.setenv("HG_ATTN_HOST_DIRECT", "0")
+    pin = (lambda t: t.cpu()) if how == "pageable" else (lambda t: t.cpu().pin_memory())
+    host_h = [tuple(pin(x) for x in src) for src in host_dev]
+    if how == "mixed":
+        host_h[1] = tuple(x.cpu() for x in host_dev[1])          # one pageable buffer sends the whole call to copies
+    if how == "unaligned":
+        o, m, l = host_h[0]
+        shifted = torch.empty(o.numel() + 1, dtype=torch.float32).pin_memory()
+        shifted[1:].copy_(o.reshape(-1))
+        host_h[0] = (shifted[1:].view(o.shape), m, l)
+        assert host_h[0][0].data_ptr() % 16 == 4
+    out_h = torch.full(prob.out.shape, float("nan"), dtype=torch.float32)
+    lse_h = torch.full(prob.lse.shape, float("nan"), dtype=torch.float32)
+    if how != "pageable":
+        out_h, lse_h = out_h.pin_memory(), lse_h.pin_memory()
+    ws = torch.empty(pkg.hg_attn_workspace_bytes(prob.desc, 2), dtype=torch.uint8, device=DEV)
+    q_h, sl_h, tb_h, te_h = pin(prob.q), pin(prob.seq_lens), pin(prob.tok_begin), pin(prob.tok_end)
+    for _ in range(2):
+        pkg.hg_attn_decode_host(q_h, prob.kv["k"], prob.kv["v"], sl_h, tb_h, te_h, host_h, out_h, lse_h, ws, prob.desc)
+        torch.cuda.synchronize()
+    assert torch.equal(out_h, prob.out.cpu()) and torch.equal(lse_h, prob.lse.cpu())
+    check_output(out_h, lse_h, ref.out, ref.lse, how)
+
+
 # ---- the read probe moves exactly the slice's bytes -------------------------------------------------------------
 
 @pytest.mark.parametrize("layout", ["HND", "NHD"])
