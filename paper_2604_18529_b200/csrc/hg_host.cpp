@@ -41,45 +41,131 @@ inline float bf16_bits_to_float(uint16_t h) {
     return f;
 }
 
-float dot_scalar(const uint16_t* a, const uint16_t* b, int D, bool bf16) {
-    float acc = 0.f;
-    if (bf16) for (int d = 0; d < D; ++d) acc = fmaf(bf16_bits_to_float(a[d]), bf16_bits_to_float(b[d]), acc);
-    else for (int d = 0; d < D; ++d) acc = fmaf(half_bits_to_float(a[d]), half_bits_to_float(b[d]), acc);
-    return acc;
-}
-
 #if defined(__x86_64__)
-__attribute__((target("avx2,fma,f16c"))) float dot_avx2(const uint16_t* a, const uint16_t* b, int D, bool bf16) {
-    __m256 acc = _mm256_setzero_ps();
-    for (int d = 0; d < D; d += 8) {
-        const __m128i ra = _mm_loadu_si128(reinterpret_cast<const __m128i*>(a + d));
-        const __m128i rb = _mm_loadu_si128(reinterpret_cast<const __m128i*>(b + d));
-        __m256 fa, fb;
-        if (bf16) {
-            fa = _mm256_castsi256_ps(_mm256_slli_epi32(_mm256_cvtepu16_epi32(ra), 16));
-            fb = _mm256_castsi256_ps(_mm256_slli_epi32(_mm256_cvtepu16_epi32(rb), 16));
-        } else {
-            fa = _mm256_cvtph_ps(ra);
-            fb = _mm256_cvtph_ps(rb);
-        }
-        acc = _mm256_fmadd_ps(fa, fb, acc);
-    }
-    __m128 s = _mm_add_ps(_mm256_castps256_ps128(acc), _mm256_extractf128_ps(acc, 1));
-    s = _mm_add_ps(s, _mm_movehl_ps(s, s));
-    s = _mm_add_ss(s, _mm_shuffle_ps(s, s, 1));
-    return _mm_cvtss_f32(s);
-}
 bool have_avx2() {
     static const bool ok = __builtin_cpu_supports("avx2") && __builtin_cpu_supports("fma") && __builtin_cpu_supports("f16c");
     return ok;
 }
 #endif
 
-inline float dot16(const uint16_t* a, const uint16_t* b, int D, bool bf16) {
+// ---- tiled logits: TILE_T token rows of one KV head against the G query heads that share it ------------
+//
+// The rows are converted to fp32 once into a small buffer; every head of the group then takes its dot
+// products from that buffer with one accumulator per token, and the TILE_T accumulators are summed across
+// lanes together (a transposing add tree) so that a head's logits for the tile leave as one vector.
+
+constexpr int TILE_T = 16;
+constexpr int MAX_D = 256;
+
+struct TileArgs {
+    const uint16_t* rows[TILE_T];   // K rows of the tile (rows past `valid` repeat the last valid one)
+    const uint16_t* next[TILE_T];   // the rows the following tile will read: prefetched while this one is converted
+    int valid;                      // tokens of the tile that exist
+    int D, G;
+    bool bf16;
+    float scale;
+    const float* qf;                // [G][D] fp32 query rows of the group
+    float* out;                     // logits of the group's first head at the tile's first token
+    int64_t out_stride;             // floats between consecutive heads
+};
+
+void tile_scalar(const TileArgs& a) {
+    for (int h = 0; h < a.G; ++h)
+        for (int t = 0; t < a.valid; ++t) {
+            float acc = 0.f;
+            const float* q = a.qf + (int64_t)h * a.D;
+            for (int d = 0; d < a.D; ++d)
+                acc = fmaf(a.bf16 ? bf16_bits_to_float(a.rows[t][d]) : half_bits_to_float(a.rows[t][d]), q[d], acc);
+            a.out[h * a.out_stride + t] = a.scale * acc;
+        }
+}
+
 #if defined(__x86_64__)
-    if (have_avx2()) return dot_avx2(a, b, D, bf16);
+// eight accumulators -> one vector holding their eight horizontal sums
+__attribute__((target("avx2,fma,f16c"))) inline __m256 hsum8(const __m256* v) {
+    const __m256 h01 = _mm256_hadd_ps(v[0], v[1]), h23 = _mm256_hadd_ps(v[2], v[3]);
+    const __m256 h45 = _mm256_hadd_ps(v[4], v[5]), h67 = _mm256_hadd_ps(v[6], v[7]);
+    const __m256 a = _mm256_hadd_ps(h01, h23), b = _mm256_hadd_ps(h45, h67);
+    return _mm256_add_ps(_mm256_permute2f128_ps(a, b, 0x20), _mm256_permute2f128_ps(a, b, 0x31));
+}
+
+__attribute__((target("avx2,fma,f16c"))) void tile_avx2(const TileArgs& a) {
+    alignas(32) float buf[TILE_T * MAX_D];
+    const int D = a.D;
+    for (int t = 0; t < TILE_T; ++t) {
+        for (int d = 0; d < D; d += 32) _mm_prefetch(reinterpret_cast<const char*>(a.next[t] + d), _MM_HINT_T0);
+        for (int d = 0; d < D; d += 8) {
+            const __m128i r = _mm_loadu_si128(reinterpret_cast<const __m128i*>(a.rows[t] + d));
+            const __m256 f = a.bf16 ? _mm256_castsi256_ps(_mm256_slli_epi32(_mm256_cvtepu16_epi32(r), 16)) : _mm256_cvtph_ps(r);
+            _mm256_store_ps(buf + t * D + d, f);
+        }
+    }
+    const __m256 sc = _mm256_set1_ps(a.scale);
+    for (int h = 0; h < a.G; ++h) {
+        const float* q = a.qf + (int64_t)h * D;
+        alignas(32) float res[TILE_T];
+        for (int half = 0; half < 2; ++half) {
+            __m256 acc[8];
+            for (int t = 0; t < 8; ++t) acc[t] = _mm256_setzero_ps();
+            const float* b0 = buf + half * 8 * D;
+            for (int d = 0; d < D; d += 8) {
+                const __m256 qv = _mm256_loadu_ps(q + d);
+                for (int t = 0; t < 8; ++t) acc[t] = _mm256_fmadd_ps(_mm256_load_ps(b0 + t * D + d), qv, acc[t]);
+            }
+            _mm256_store_ps(res + half * 8, _mm256_mul_ps(hsum8(acc), sc));
+        }
+        float* o = a.out + h * a.out_stride;
+        if (a.valid == TILE_T) { _mm256_storeu_ps(o, _mm256_load_ps(res)); _mm256_storeu_ps(o + 8, _mm256_load_ps(res + 8)); }
+        else memcpy(o, res, sizeof(float) * a.valid);
+    }
+}
+
+__attribute__((target("avx512f,avx2,fma,f16c"))) void tile_avx512(const TileArgs& a) {
+    alignas(64) float buf[TILE_T * MAX_D];
+    const int D = a.D;                                   // a multiple of 16 here
+    for (int t = 0; t < TILE_T; ++t) {
+        for (int d = 0; d < D; d += 32) _mm_prefetch(reinterpret_cast<const char*>(a.next[t] + d), _MM_HINT_T0);
+        for (int d = 0; d < D; d += 16) {
+            const __m256i r = _mm256_loadu_si256(reinterpret_cast<const __m256i*>(a.rows[t] + d));
+            const __m512 f = a.bf16 ? _mm512_castsi512_ps(_mm512_slli_epi32(_mm512_cvtepu16_epi32(r), 16)) : _mm512_cvtph_ps(r);
+            _mm512_store_ps(buf + t * D + d, f);
+        }
+    }
+    const __m256 sc = _mm256_set1_ps(a.scale);
+    for (int h = 0; h < a.G; ++h) {
+        const float* q = a.qf + (int64_t)h * D;
+        __m512 acc[TILE_T];
+        for (int t = 0; t < TILE_T; ++t) acc[t] = _mm512_setzero_ps();
+        for (int d = 0; d < D; d += 16) {
+            const __m512 qv = _mm512_loadu_ps(q + d);
+            for (int t = 0; t < TILE_T; ++t) acc[t] = _mm512_fmadd_ps(_mm512_load_ps(buf + t * D + d), qv, acc[t]);
+        }
+        __m256 half[TILE_T];
+        for (int t = 0; t < TILE_T; ++t)
+            half[t] = _mm256_add_ps(_mm512_castps512_ps256(acc[t]),
+                                    _mm256_castpd_ps(_mm512_extractf64x4_pd(_mm512_castps_pd(acc[t]), 1)));
+        alignas(32) float res[TILE_T];
+        _mm256_store_ps(res, _mm256_mul_ps(hsum8(half), sc));
+        _mm256_store_ps(res + 8, _mm256_mul_ps(hsum8(half + 8), sc));
+        float* o = a.out + h * a.out_stride;
+        if (a.valid == TILE_T) { _mm256_storeu_ps(o, _mm256_load_ps(res)); _mm256_storeu_ps(o + 8, _mm256_load_ps(res + 8)); }
+        else memcpy(o, res, sizeof(float) * a.valid);
+    }
+}
+bool have_avx512() {
+    static const bool ok = have_avx2() && __builtin_cpu_supports("avx512f");
+    return ok;
+}
 #endif
-    return dot_scalar(a, b, D, bf16);
+
+using TileFn = void (*)(const TileArgs&);
+
+TileFn pick_tile_fn(int D) {
+#if defined(__x86_64__)
+    if (D <= MAX_D && D % 16 == 0 && have_avx512()) return tile_avx512;
+    if (D <= MAX_D && have_avx2()) return tile_avx2;
+#endif
+    return tile_scalar;
 }
 
 bool desc_ok(const hg_host_desc* d) {
@@ -116,18 +202,48 @@ hg_status hg_host_logits(const void* q, const void* k_rows, const int32_t* idx, 
     const float scale = d->scale > 0.f ? d->scale : 1.0f / sqrtf((float)D);
     const uint16_t* qp = static_cast<const uint16_t*>(q);
     const uint16_t* kp = static_cast<const uint16_t*>(k_rows);
-    parallel_for((int64_t)d->batch * d->num_q_heads, d->threads, [&](int64_t row) {
-        const int b = (int)(row / d->num_q_heads), h = (int)(row % d->num_q_heads), g = h / G;
+    const int Hq = d->num_q_heads, Hkv = d->num_kv_heads;
+    // query rows once as fp32
+    std::vector<float> qf((size_t)d->batch * Hq * D);
+    for (size_t i = 0; i < qf.size(); ++i) qf[i] = bf16 ? bf16_bits_to_float(qp[i]) : half_bits_to_float(qp[i]);
+    const TileFn tile = pick_tile_fn(D);
+
+    // Work items: (sequence, block of tokens, KV heads).  When a token's heads lie next to each other in memory
+    // (token-major rows) one item sweeps all heads of its tokens, so that memory is read front to back; with
+    // head-major rows every KV head is an item of its own stream.
+    constexpr int BLOCK = 256;
+    const bool token_major = d->head_stride < d->tok_stride;
+    const int g_per_item = token_major ? Hkv : 1;
+    const int g_items = Hkv / g_per_item;
+    const int blocks = (K + BLOCK - 1) / BLOCK;
+    parallel_for((int64_t)d->batch * blocks * g_items, d->threads, [&](int64_t item) {
+        const int gi = (int)(item % g_items);
+        const int blk = (int)((item / g_items) % blocks);
+        const int b = (int)(item / ((int64_t)g_items * blocks));
         const int n = std::max(0, std::min(n_sel[b], K));
-        const uint16_t* qrow = qp + row * D;
-        const uint16_t* kb = kp + (int64_t)b * d->seq_stride + (int64_t)g * d->head_stride;
-        const int32_t* ix = idx ? idx + ((int64_t)b * d->num_kv_heads + g) * K : nullptr;
-        float* out = logits + row * K;
-        for (int i = 0; i < n; ++i) {
-            const int64_t t = ix ? ix[i] : i;
-            out[i] = scale * dot16(qrow, kb + t * d->tok_stride, D, bf16);
+        const int t0 = blk * BLOCK, t1 = std::min(K, t0 + BLOCK);
+        const float ninf = -std::numeric_limits<float>::infinity();
+        for (int g = gi * g_per_item; g < (gi + 1) * g_per_item; ++g) {
+            const uint16_t* kb = kp + (int64_t)b * d->seq_stride + (int64_t)g * d->head_stride;
+            const int32_t* ix = idx ? idx + ((int64_t)b * Hkv + g) * K : nullptr;
+            float* out = logits + ((int64_t)b * Hq + (int64_t)g * G) * K;
+            TileArgs a;
+            a.D = D; a.G = G; a.bf16 = bf16; a.scale = scale; a.out_stride = K;
+            a.qf = qf.data() + ((size_t)b * Hq + (size_t)g * G) * D;
+            for (int t = t0; t < std::min(t1, n); t += TILE_T) {
+                a.valid = std::min(TILE_T, n - t);
+                for (int i = 0; i < TILE_T; ++i) {
+                    const int tt = t + std::min(i, a.valid - 1);
+                    const int tn = std::min(tt + TILE_T, n - 1);
+                    a.rows[i] = kb + (int64_t)(ix ? ix[tt] : tt) * d->tok_stride;
+                    a.next[i] = kb + (int64_t)(ix ? ix[tn] : tn) * d->tok_stride;
+                }
+                a.out = out + t;
+                tile(a);
+            }
+            for (int h = 0; h < G; ++h)
+                for (int t = std::max(t0, n); t < t1; ++t) out[(int64_t)h * K + t] = ninf;
         }
-        for (int i = n; i < K; ++i) out[i] = -std::numeric_limits<float>::infinity();
     });
     return HG_OK;
 }

@@ -23,7 +23,8 @@ def bits(t):
     return t.contiguous().view(torch.int16).numpy().view(np.uint16)
 
 
-@pytest.mark.parametrize("dtype,D,G", [("f16", 128, 1), ("bf16", 64, 4), ("f16", 64, 3)])
+@pytest.mark.parametrize("dtype,D,G", [("f16", 128, 1), ("bf16", 64, 4), ("f16", 64, 3), ("f16", 128, 8), ("bf16", 40, 2),
+                                       ("f16", 320, 1)])
 def test_host_logits_match_the_oracle(dtype, D, G):
     w = W.AttnWorkload("h", 2, 2 * G, 2, D, dtype, [300, 170], [200, 170], [300, 170], seed=3, sigma_kv=1.5)
     q, K = w.q(), w.kv_logical("k")                         # [B][Hq][D], [B][Lmax][Hkv][D]
@@ -52,6 +53,22 @@ def test_host_logits_match_the_oracle(dtype, D, G):
             n = int(n_sel[b])
             want = O.logits(qb[b, h], np.ascontiguousarray(Kb[b, :, h // G]), dtype, scale=0.25, idx=idx[b, h // G, :n].numpy())
             assert np.abs(lg2[b, h, :n].double().numpy() - want).max() <= 2e-5 * max(1.0, np.abs(want).max())
+
+
+def test_host_logits_head_major_rows_give_the_same_bits():
+    """Rows stored [B][Hkv][T][D] (each KV head a stream of its own) take the other split of the work; the
+    arithmetic per (token, head) is the same, so the logits are bit-identical to the token-major call."""
+    w = W.AttnWorkload("h", 2, 8, 2, 128, "f16", [700, 333], [650, 301], [700, 333], seed=8)
+    q, K = w.q(), w.kv_logical("k")
+    n_host = torch.tensor(w.tok_begin, dtype=torch.int32)
+    Ksel = int(n_host.max())
+    a = torch.empty(w.B, w.Hq, Ksel)
+    H.hg_host_logits(q, K, None, n_host, a, H.host_desc(K, w.Hq, Ksel, threads=2))
+    K_hm = K.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)        # same shape, head-major storage
+    assert K_hm.stride(2) > K_hm.stride(1)
+    b = torch.empty(w.B, w.Hq, Ksel)
+    H.hg_host_logits(q, K_hm, None, n_host, b, H.host_desc(K_hm, w.Hq, Ksel, threads=5))
+    assert torch.equal(a, b)
 
 
 def test_topk_selection_matches_the_sort_definition():
