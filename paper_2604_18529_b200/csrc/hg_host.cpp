@@ -5,8 +5,13 @@
 #include <math.h>
 #include <string.h>
 
+#include <pthread.h>
+
 #include <algorithm>
 #include <atomic>
+#include <condition_variable>
+#include <functional>
+#include <mutex>
 #include <limits>
 #include <thread>
 #include <vector>
@@ -175,19 +180,82 @@ bool desc_ok(const hg_host_desc* d) {
            d->threads >= 0;
 }
 
-// Runs fn(i) for i in [0, n) on `threads` workers (0: one per core).
+// Worker threads that outlive a call: starting a thread costs tens of microseconds, a logits call for a
+// thousand selected tokens has a few hundred microseconds of work.  The pool grows on demand, is never torn
+// down (its threads end with the process) and is forgotten by a forked child, which starts its own.
+class Pool {
+public:
+    // Runs work() on `extra` pool threads and on the caller; returns when all have finished.  A second caller
+    // arriving meanwhile is told to fend for itself.
+    bool run(int extra, const std::function<void()>& work) {
+        std::unique_lock<std::mutex> busy(busy_, std::try_to_lock);
+        if (!busy.owns_lock()) return false;
+        {
+            std::lock_guard<std::mutex> g(mu_);
+            while ((int)threads_.size() < extra) threads_.emplace_back([this, id = (int)threads_.size()] { loop(id); });
+            work_ = &work; wanted_ = extra; pending_ = extra; ++generation_;
+        }
+        wake_.notify_all();
+        work();
+        std::unique_lock<std::mutex> g(mu_);
+        done_.wait(g, [this] { return pending_ == 0; });
+        work_ = nullptr;
+        return true;
+    }
+
+private:
+    void loop(int id) {
+        uint64_t seen = 0;
+        for (;;) {
+            const std::function<void()>* w;
+            {
+                std::unique_lock<std::mutex> g(mu_);
+                wake_.wait(g, [&] { return generation_ != seen; });
+                seen = generation_;
+                if (id >= wanted_) continue;
+                w = work_;
+            }
+            (*w)();
+            std::lock_guard<std::mutex> g(mu_);
+            if (--pending_ == 0) done_.notify_one();
+        }
+    }
+    std::mutex busy_, mu_;
+    std::condition_variable wake_, done_;
+    std::vector<std::thread> threads_;
+    const std::function<void()>* work_ = nullptr;
+    int wanted_ = 0, pending_ = 0;
+    uint64_t generation_ = 0;
+};
+
+std::atomic<Pool*> g_pool{nullptr};
+
+Pool* pool() {
+    Pool* p = g_pool.load(std::memory_order_acquire);
+    if (p) return p;
+    static std::once_flag fork_hook;
+    std::call_once(fork_hook, [] { pthread_atfork(nullptr, nullptr, [] { g_pool.store(nullptr); }); });
+    Pool* fresh = new Pool;
+    if (g_pool.compare_exchange_strong(p, fresh, std::memory_order_acq_rel)) return fresh;
+    delete fresh;                                   // another thread was first; no thread had been started in ours
+    return p;
+}
+
+// Runs fn(i) for i in [0, n) on `threads` workers (0: one per core), the caller being one of them.
 template <class F>
 void parallel_for(int64_t n, int threads, F fn) {
     int nt = threads > 0 ? threads : (int)std::thread::hardware_concurrency();
     if (nt < 1) nt = 1;
+    if (nt > 256) nt = 256;
     if ((int64_t)nt > n) nt = (int)n;
     if (nt <= 1) { for (int64_t i = 0; i < n; ++i) fn(i); return; }
     std::atomic<int64_t> next{0};
-    std::vector<std::thread> pool;
-    auto work = [&] { for (int64_t i; (i = next.fetch_add(1)) < n;) fn(i); };
-    for (int t = 1; t < nt; ++t) pool.emplace_back(work);
+    const std::function<void()> work = [&] { for (int64_t i; (i = next.fetch_add(1)) < n;) fn(i); };
+    if (pool()->run(nt - 1, work)) return;
+    std::vector<std::thread> own;                   // the pool is serving another caller
+    for (int t = 1; t < nt; ++t) own.emplace_back(work);
     work();
-    for (auto& t : pool) t.join();
+    for (auto& t : own) t.join();
 }
 
 }  // namespace
@@ -216,7 +284,12 @@ hg_status hg_host_logits(const void* q, const void* k_rows, const int32_t* idx, 
     const int g_per_item = token_major ? Hkv : 1;
     const int g_items = Hkv / g_per_item;
     const int blocks = (K + BLOCK - 1) / BLOCK;
-    parallel_for((int64_t)d->batch * blocks * g_items, d->threads, [&](int64_t item) {
+    // a worker thread costs tens of microseconds to start: give each at least 256 KB of keys to read
+    int64_t key_bytes = 0;
+    for (int b = 0; b < d->batch; ++b) key_bytes += (int64_t)std::max(0, std::min(n_sel[b], K)) * Hkv * D * 2;
+    int workers = d->threads > 0 ? d->threads : (int)std::thread::hardware_concurrency();
+    workers = (int)std::max<int64_t>(1, std::min<int64_t>(workers, key_bytes >> 18));
+    parallel_for((int64_t)d->batch * blocks * g_items, workers, [&](int64_t item) {
         const int gi = (int)(item % g_items);
         const int blk = (int)((item / g_items) % blocks);
         const int b = (int)(item / ((int64_t)g_items * blocks));

@@ -71,6 +71,30 @@ def test_host_logits_head_major_rows_give_the_same_bits():
     assert torch.equal(a, b)
 
 
+def test_host_logits_from_two_caller_threads_at_once():
+    """The worker pool serves one call at a time; a call that finds it busy runs on threads of its own.
+    Either way the result is the same."""
+    import threading
+    w = W.AttnWorkload("h", 4, 8, 4, 128, "bf16", [3000] * 4, [2900] * 4, [3000] * 4, seed=12)
+    q, K = w.q(), w.kv_logical("k")
+    n_host = torch.tensor(w.tok_begin, dtype=torch.int32)
+    want = torch.empty(w.B, w.Hq, 2900)
+    H.hg_host_logits(q, K, None, n_host, want, H.host_desc(K, w.Hq, 2900, threads=1))
+    outs = [torch.empty(w.B, w.Hq, 2900) for _ in range(4)]
+
+    def call(o):
+        for _ in range(5):
+            H.hg_host_logits(q, K, None, n_host, o, H.host_desc(K, w.Hq, 2900, threads=4))
+
+    ts = [threading.Thread(target=call, args=(o,)) for o in outs]
+    for t in ts:
+        t.start()
+    for t in ts:
+        t.join()
+    for o in outs:
+        assert torch.equal(o, want)
+
+
 def test_topk_selection_matches_the_sort_definition():
     rng = np.random.default_rng(5)
     scores = rng.standard_normal((6, 200)).astype(np.float32)
