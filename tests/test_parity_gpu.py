@@ -460,3 +460,30 @@ def test_sinks_plus_recent_window_as_two_ranges(G):
             ref_out[b, h], ref_lse[b, h] = O.full(q[b, h], np.ascontiguousarray(K[b, :, g]), np.ascontiguousarray(V[b, :, g]),
                                                    w.dtype, idx=idx)
     check_output(prob.out, prob.lse, ref_out, ref_lse, "sinks + window")
+
+
+@pytest.mark.parametrize("G", [1, 4])
+def test_a_slice_longer_than_num_chunks_is_cut_to_its_first_chunks(G):
+    """num_chunks bounds the work: tokens past the last chunk slot are not attended, and what is produced equals attention over the kept range."""
+    C, keep = 128, 3
+    w = wl(Hq=2 * G, Hkv=2, seq_lens=[900, 500], tok_begin=[70, 0], tok_end=[900, 200], chunk_tokens=C, seed=31)
+    prob = DeviceProblem(w, DEV)
+    assert prob.NC > keep
+    prob.NC = keep
+    prob.desc = prob.make_desc(C, keep)
+    prob.o_part = torch.empty(w.B, w.Hq, keep, w.D, device=DEV)
+    prob.m_part = torch.empty(w.B, w.Hq, keep, device=DEV)
+    prob.l_part = torch.empty(w.B, w.Hq, keep, device=DEV)
+    prob.step([])
+    torch.cuda.synchronize()
+    assert int(prob.status.item()) == hg.HG_DEV_OK
+    kept_end = [min(te, (tb // C + keep) * C) for tb, te in zip(w.tok_begin, w.tok_end)]
+    assert kept_end == [384, 200]
+    w_cut = dataclasses.replace(w, tok_end=kept_end)
+    ref = OracleRef(w_cut)
+    rm, rl, ro = ref.chunk_partials(C, keep)
+    check_partials(prob.o_part.reshape(-1, w.D), prob.m_part.reshape(-1), prob.l_part.reshape(-1),
+                   rm.reshape(-1), rl.reshape(-1), ro.reshape(-1, w.D), "cut")
+    from oracle import hg_oracle as O
+    ref_out, ref_lse = O.full_batch(ref.q, ref.K, ref.V, w.dtype, w.tok_begin, kept_end)
+    check_output(prob.out, prob.lse, ref_out, ref_lse, "cut")
