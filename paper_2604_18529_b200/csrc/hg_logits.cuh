@@ -77,25 +77,38 @@ __global__ void __launch_bounds__(LG_THREADS) logits_partial_kernel(const Logits
         for (int hh = 0; hh < 8; ++hh)
 #pragma unroll
             for (int v = 0; v < VEC; ++v) acc[hh][v] = 0.f;
-        for (int t = warp; t < nt; t += LG_WARPS) {
-            const uint16_t* vrow = vbase + (size_t)(t0 + t) * D + lane * VEC;
-            float vv[VEC];
-            if constexpr (VEC == 4) {
-                const uint2 raw = *reinterpret_cast<const uint2*>(vrow);
-                const float2 a = unpack2<BF16>(raw.x), bb = unpack2<BF16>(raw.y);
-                vv[0] = a.x; vv[1] = a.y; vv[2] = bb.x; vv[3] = bb.y;
-            } else {
-                const uint32_t raw = *reinterpret_cast<const uint32_t*>(vrow);
-                const float2 a = unpack2<BF16>(raw);
-                vv[0] = a.x; vv[1] = a.y;
+        constexpr int UNROLL = 4;                                  // V rows in flight per warp
+        for (int tt = warp; tt < nt; tt += UNROLL * LG_WARPS) {
+            uint2 raw[UNROLL];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const int t = tt + u * LG_WARPS;
+                raw[u] = make_uint2(0u, 0u);
+                if (t < nt) {
+                    const uint16_t* vrow = vbase + (size_t)(t0 + t) * D + lane * VEC;
+                    if constexpr (VEC == 4) raw[u] = *reinterpret_cast<const uint2*>(vrow);
+                    else raw[u].x = *reinterpret_cast<const uint32_t*>(vrow);
+                }
             }
 #pragma unroll
-            for (int hh = 0; hh < 8; ++hh) {
-                if (hh < nh) {
-                    const float pv = s_p[hh * p.chunk + t];       // broadcast read
-                    if (pv != 0.f) {                              // unselected slots (and their V rows) never enter the sum
+            for (int u = 0; u < UNROLL; ++u) {
+                const int t = tt + u * LG_WARPS;
+                if (t >= nt) break;
+                float vv[VEC];
+                const float2 a = unpack2<BF16>(raw[u].x);
+                vv[0] = a.x; vv[1] = a.y;
+                if constexpr (VEC == 4) {
+                    const float2 bb = unpack2<BF16>(raw[u].y);
+                    vv[2] = bb.x; vv[3] = bb.y;
+                }
 #pragma unroll
-                        for (int v = 0; v < VEC; ++v) acc[hh][v] = fmaf(pv, vv[v], acc[hh][v]);
+                for (int hh = 0; hh < 8; ++hh) {
+                    if (hh < nh) {
+                        const float pv = s_p[hh * p.chunk + t];       // broadcast read
+                        if (pv != 0.f) {                              // unselected slots (and their V rows) never enter the sum
+#pragma unroll
+                            for (int v = 0; v < VEC; ++v) acc[hh][v] = fmaf(pv, vv[v], acc[hh][v]);
+                        }
                     }
                 }
             }
