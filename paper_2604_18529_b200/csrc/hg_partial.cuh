@@ -170,7 +170,6 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
         fence_barrier_init();
     }
     int n_items = 1, item_step = 1, item_first = 0;
-    if (status_at_entry == HG_DEV_WAIT_TIMEOUT) return;
     if (p.persistent) {
         // cum[b+1] = sum_{b' <= b} nc_b' * Y : one warp, each lane a contiguous block of sequences
         if (warp == 0) {
@@ -205,6 +204,7 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
     } else {
         __syncthreads();
     }
+    if (status_at_entry == HG_DEV_WAIT_TIMEOUT) return;   // checked only now: its load overlapped the scan's loads
 
     volatile int* abort_flag = &ctl.abort_flag;
     auto get_item = [&](int i) -> Item {
