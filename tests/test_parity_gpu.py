@@ -431,6 +431,29 @@ def test_random_shapes(seed):
     run_and_check(w, poison_tail=bool(rng.integers(0, 2)), what=repr(w))
 
 
+@pytest.mark.parametrize("dynamic", ["1", "0"])
+@pytest.mark.parametrize("seed", range(5))
+def test_random_shapes_with_many_items_per_cta(seed, dynamic, monkeypatch):
+    """Several hundred to a couple of thousand work items: every resident CTA takes several, so the ring runs
+    across item boundaries, the look-ahead of item indices and page ids is in play, and (dynamic) the counter."""
+    monkeypatch.setenv("HG_ATTN_DYNAMIC", dynamic)
+    rng = np.random.default_rng(50000 + seed)
+    B = int(rng.integers(4, 9))
+    Hkv = int(rng.choice([4, 8]))
+    G = int(rng.choice([1, 2, 4, 8]))
+    D = int(rng.choice([64, 128]))
+    page = int(rng.choice([16, 64]))
+    chunk = max(int(rng.choice([64, 128])), page)
+    layout, paged = [("HND", True), ("NHD", True), ("NHD", False)][int(rng.integers(0, 3))]
+    lens = [int(rng.integers(4000, 8000)) for _ in range(B)]
+    tb = [int(rng.integers(0, L // 4)) for L in lens]
+    te = [int(rng.integers(3 * L // 4, L + 1)) for L in lens]
+    w = W.AttnWorkload(f"many{seed}", B, Hkv * G, Hkv, D, str(rng.choice(["f16", "bf16"])), lens, tb, te, page_size=page,
+                       layout=layout, paged=paged, chunk_tokens=chunk, seed=7000 + seed)
+    assert sum(w.chunk_grid(b)[1] for b in range(B)) * Hkv > 296
+    run_and_check(w, what=repr(w)[:200])
+
+
 # ---- a token set made of several ranges (Section 4.3's position-based choice: sinks + recent window) ----
 
 @pytest.mark.parametrize("G", [1, 4])
