@@ -17,6 +17,7 @@ from .binding import (  # noqa: F401
     logits_desc,
     hg_attn_decode,
     hg_attn_decode_host,
+    prepare_decode_host,
     hg_attn_decode_static,
     hg_attn_workspace_bytes,
     hg_status_string,

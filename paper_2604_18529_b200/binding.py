@@ -286,6 +286,31 @@ def hg_attn_decode_host(q_host, k_cache, v_cache, seq_lens_host, tok_begin_host,
     _check(st, "hg_attn_decode_host")
 
 
+def prepare_decode_host(q_host, k_cache, v_cache, seq_lens_host, tok_begin_host, tok_end_host, host_partials_host,
+                        out_host, lse_host, workspace, desc: HgAttnDesc, stream=None):
+    """Marshal the arguments of ``hg_attn_decode_host`` once and return a callable that makes the call.
+
+    For a decode loop that reuses the same buffers every step (the usual case): the per-call cost of
+    checking and converting a dozen tensors is paid once.  The returned callable keeps the tensors alive.
+    """
+    arr = _src_array(host_partials_host, host=True)
+    args = (_host(q_host, "q_host"), _dev(k_cache, "k_cache"), _dev(v_cache, "v_cache"),
+            _host(seq_lens_host, "seq_lens_host", torch.int32), _host(tok_begin_host, "tok_begin_host", torch.int32),
+            _host(tok_end_host, "tok_end_host", torch.int32), arr, len(host_partials_host),
+            _host(out_host, "out_host", torch.float32), _host(lse_host, "lse_host", torch.float32),
+            _dev(workspace, "workspace"), workspace.numel() * workspace.element_size(), _stream(stream), C.byref(desc))
+    keep = (q_host, k_cache, v_cache, seq_lens_host, tok_begin_host, tok_end_host, host_partials_host, out_host, lse_host,
+            workspace, desc, arr)
+    fn = lib().hg_attn_decode_host
+
+    def call(_keep=keep) -> None:
+        st = fn(*args)
+        if st != HG_OK:
+            _check(st, "hg_attn_decode_host")
+
+    return call
+
+
 def hg_kv_append(k_new, v_new, k_cache, v_cache, seq_lens, tok_end, desc: HgAttnDesc, stream=None) -> None:
     """Write this step's K/V rows [B][Hkv][D] at position seq_lens[b] and advance seq_lens (and tok_end)."""
     st = lib().hg_kv_append(_dev(k_new, "k_new"), _dev(v_new, "v_new"), _dev(k_cache, "k_cache"), _dev(v_cache, "v_cache"),

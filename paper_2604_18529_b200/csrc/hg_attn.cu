@@ -168,7 +168,7 @@ static hg_status launch_partial_m(int D, bool bf16, const CUtensorMap& tk, const
 
 static hg_status run_partial(int mode, const void* q, const void* k, const void* v, const int32_t* seq_lens,
                              const int32_t* tok_begin, const int32_t* tok_end, float* o_part, float* m_part, float* l_part,
-                             uint32_t* sink, void* stream, const hg_attn_desc* d) {
+                             uint32_t* sink, void* stream, const hg_attn_desc* d, bool counter_is_zero = false) {
     hg_status st = check_desc(d, true);
     if (st != HG_OK) return st;
     if (!k || !v || !seq_lens || !tok_begin || !tok_end) return HG_ERR_INVALID_ARG;
@@ -201,7 +201,7 @@ static hg_status run_partial(int mode, const void* q, const void* k, const void*
     p.test_stall = (d->flags & HG_FLAG_TEST_STALL) ? 1 : 0;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     p.sched = p.persistent && env_int("HG_ATTN_DYNAMIC", 1, 0, 1) ? desc_sched(d) : nullptr;
-    if (p.sched && cudaMemsetAsync(p.sched, 0, sizeof(int32_t), cs) != cudaSuccess) {
+    if (p.sched && !counter_is_zero && cudaMemsetAsync(p.sched, 0, sizeof(int32_t), cs) != cudaSuccess) {
         cudaGetLastError();
         return HG_ERR_CUDA;
     }
@@ -371,10 +371,10 @@ size_t hg_attn_workspace_bytes(const hg_attn_desc* desc, int32_t n_host_partials
     return plan_workspace(desc, n_host_partials, HG_MAX_MERGE_SRC).total;
 }
 
-hg_status hg_attn_decode(const void* q, const void* k_cache, const void* v_cache, const int32_t* seq_lens,
-                         const int32_t* tok_begin, const int32_t* tok_end, const hg_partial_src* host_partials,
-                         int32_t n_host_src, float* out, float* lse, void* workspace, size_t workspace_bytes, void* stream,
-                         const hg_attn_desc* desc) {
+static hg_status decode_impl(const void* q, const void* k_cache, const void* v_cache, const int32_t* seq_lens,
+                             const int32_t* tok_begin, const int32_t* tok_end, const hg_partial_src* host_partials,
+                             int32_t n_host_src, float* out, float* lse, void* workspace, size_t workspace_bytes, void* stream,
+                             const hg_attn_desc* desc, bool counter_is_zero) {
     hg_status st = check_desc(desc, true);
     if (st != HG_OK) return st;
     if (n_host_src < 0 || n_host_src > HG_MAX_MERGE_SRC - 1 || (n_host_src && !host_partials)) return HG_ERR_INVALID_ARG;
@@ -390,12 +390,21 @@ hg_status hg_attn_decode(const void* q, const void* k_cache, const void* v_cache
     memcpy(&dd, desc, desc->struct_size < sizeof dd ? desc->struct_size : sizeof dd);
     dd.struct_size = sizeof dd;
     dd.sched_counter = reinterpret_cast<int32_t*>(ws + w.sched);       // the workspace provides the work counter
-    st = run_partial(MODE_MHA, q, k_cache, v_cache, seq_lens, tok_begin, tok_end, o_part, m_part, l_part, nullptr, stream, &dd);
+    st = run_partial(MODE_MHA, q, k_cache, v_cache, seq_lens, tok_begin, tok_end, o_part, m_part, l_part, nullptr, stream, &dd,
+                     counter_is_zero);
     if (st != HG_OK) return st;
     hg_partial_src src[HG_MAX_MERGE_SRC];
     src[0].o = o_part; src[0].m = m_part; src[0].l = l_part; src[0].nc = desc->num_chunks; src[0].reserved = 0;
     for (int i = 0; i < n_host_src; ++i) src[1 + i] = host_partials[i];
     return run_merge(src, 1 + n_host_src, out, lse, stream, desc);
+}
+
+hg_status hg_attn_decode(const void* q, const void* k_cache, const void* v_cache, const int32_t* seq_lens,
+                         const int32_t* tok_begin, const int32_t* tok_end, const hg_partial_src* host_partials,
+                         int32_t n_host_src, float* out, float* lse, void* workspace, size_t workspace_bytes, void* stream,
+                         const hg_attn_desc* desc) {
+    return decode_impl(q, k_cache, v_cache, seq_lens, tok_begin, tok_end, host_partials, n_host_src, out, lse, workspace,
+                       workspace_bytes, stream, desc, false);
 }
 
 hg_status hg_attn_decode_host(const void* q_host, const void* k_cache, const void* v_cache, const int32_t* seq_lens_host,
@@ -446,13 +455,14 @@ hg_status hg_attn_decode_host(const void* q_host, const void* k_cache, const voi
         float* lse_alias = direct && lse_host ? static_cast<float*>(device_alias(lse_host)) : nullptr;
         direct = direct && out_alias && (!lse_host || lse_alias);
         if (direct) {
+            sp.zero = reinterpret_cast<int32_t*>(ws + w.sched);        // the staging kernel also clears the work counter
             const unsigned blocks = (unsigned)((rows * D * 2 / 16 + STAGE_THREADS - 1) / STAGE_THREADS);
             stage_kernel<<<blocks < 1 ? 1 : (blocks > 64 ? 64 : blocks), STAGE_THREADS, 0, cs>>>(sp);
             if (cudaGetLastError() != cudaSuccess) return HG_ERR_CUDA;
-            return hg_attn_decode(ws + w.q, k_cache, v_cache, reinterpret_cast<const int32_t*>(ws + w.seq_lens),
-                                  reinterpret_cast<const int32_t*>(ws + w.tok_begin),
-                                  reinterpret_cast<const int32_t*>(ws + w.tok_end), alias, n_host_src, out_alias, lse_alias,
-                                  workspace, workspace_bytes, stream, desc);
+            return decode_impl(ws + w.q, k_cache, v_cache, reinterpret_cast<const int32_t*>(ws + w.seq_lens),
+                               reinterpret_cast<const int32_t*>(ws + w.tok_begin),
+                               reinterpret_cast<const int32_t*>(ws + w.tok_end), alias, n_host_src, out_alias, lse_alias,
+                               workspace, workspace_bytes, stream, desc, true);
         }
     }
     bool ok = true;

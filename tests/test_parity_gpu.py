@@ -245,6 +245,12 @@ def test_decode_host_paths_agree(how, monkeypatch):
         torch.cuda.synchronize()
     assert torch.equal(out_h, prob.out.cpu()) and torch.equal(lse_h, prob.lse.cpu())
     check_output(out_h, lse_h, ref.out, ref.lse, how)
+    # the same call with its arguments marshalled once
+    call = pkg.prepare_decode_host(q_h, prob.kv["k"], prob.kv["v"], sl_h, tb_h, te_h, host_h, out_h, lse_h, ws, prob.desc)
+    out_h.fill_(float("nan"))
+    call()
+    torch.cuda.synchronize()
+    assert torch.equal(out_h, prob.out.cpu()) and torch.equal(lse_h, prob.lse.cpu())
 
 
 # ---- the read probe moves exactly the slice's bytes -------------------------------------------------------------
