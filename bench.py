@@ -32,7 +32,11 @@ NCU_TRAFFIC_BYTES = {
     # profiles/partial_kernel_opt13b.md: two sequences captured (805.54 MB read + 4.74 MB written), x 4
     "opt13b": 4 * (805_537_024 + 4_742_400),
     # profiles/partial_kernel_llama70b.md: the full launch captured
-    "llama70b": 1_718_222_000 + 6_867_968,
+    "llama70b": 1_718_226_000 + 7_822_080,
+    # profiles/partial_kernel_opt30b.md: one of the four sequences captured (1879.14 MB read + 3.87 MB written), x 4
+    "opt30b": 4 * (1_879_144_000 + 3_870_464),
+    # profiles/partial_kernel_ragged.md: the full launch captured
+    "ragged": 951_494_144 + 8_356_864,
 }
 
 
@@ -431,7 +435,7 @@ def main():
             "roofline": {"bound": "hbm", "kernel": "partial_kernel", "achieved": achieved, "peak": peak,
                          "peak_kind": f"{peak_kind} copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
                          "frac_of_8000": achieved / 8000.0, "alg_bytes_per_launch": part_alg,
-                         "traffic": NCU_TRAFFIC_BYTES.get(args.workload)},
+                         "traffic": None if args.batch else NCU_TRAFFIC_BYTES.get(args.workload)},
             "e2e": {"value": whole_job_value(tokens, world, e2e_ms / args.steps), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps, "matches_device_path": bool(same),
                     "api": "hg_attn_decode_host via prepare_decode_host (KV pools stay device resident: they are the GPU's slice of the cache)"},
