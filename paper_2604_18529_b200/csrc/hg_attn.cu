@@ -542,7 +542,7 @@ hg_status hg_kv_evict(const void* k_cache, const void* v_cache, int32_t* tok_beg
     if (!aligned16(k_cache) || !aligned16(v_cache) || !aligned16(k_out) || !aligned16(v_out)) return HG_ERR_INVALID_ARG;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     const KvPoolView pv = pool_view(desc, k_cache, v_cache);
-    dim3 grid((unsigned)((max_evict + 31) / 32), (unsigned)desc->batch);
+    dim3 grid((unsigned)((max_evict + EVICT_TOK_PER_CTA - 1) / EVICT_TOK_PER_CTA), (unsigned)desc->batch);
     kv_evict_copy_kernel<<<grid, 256, 0, cs>>>(pv, tok_begin, tok_end, n_evict, static_cast<uint16_t*>(k_out),
                                                 static_cast<uint16_t*>(v_out), max_evict, desc->status);
     if (cudaGetLastError() != cudaSuccess) return HG_ERR_CUDA;

@@ -52,6 +52,8 @@ __global__ void kv_append_kernel(KvPoolView pv, const uint16_t* __restrict__ k_n
     }
 }
 
+constexpr int EVICT_TOK_PER_CTA = 8;
+
 // Copies the first n_evict[b] tokens of the slice [tok_begin, tok_end) of every sequence into
 // k_out / v_out [B][max_evict][Hkv][D] (token-major rows, the layout the host keeps its part in).
 // Grid (token blocks, B); reads only.
@@ -62,19 +64,41 @@ __global__ void kv_evict_copy_kernel(KvPoolView pv, const int32_t* __restrict__ 
     const int tb = tok_begin[b];
     const int ne = max(0, min(min(n_evict[b], max_evict), tok_end[b] - tb));
     const int vec_per_row = pv.D / 8, vec_per_tok = pv.Hkv * vec_per_row;
-    const int tok_per_cta = 32;
-    const int i0 = blockIdx.x * tok_per_cta, i1 = min(ne, i0 + tok_per_cta);
-    for (int idx = threadIdx.x + i0 * vec_per_tok; idx < i1 * vec_per_tok; idx += blockDim.x) {
-        const int i = idx / vec_per_tok, r = idx - i * vec_per_tok;
-        const int g = r / vec_per_row, c = r - g * vec_per_row;
-        const int t = tb + i;
-        const int phys = kv_page_of(pv, b, t);
-        if (phys < 0) { if (status) atomicMax(status, HG_DEV_BAD_PAGE); continue; }
-        const int64_t src = (int64_t)phys * pv.page_stride + (int64_t)(t & (pv.page_size - 1)) * pv.tok_stride +
-                            (int64_t)g * pv.head_stride + c * 8;
-        const int64_t dst = (((int64_t)b * max_evict + i) * pv.Hkv + g) * pv.D + c * 8;
-        *reinterpret_cast<uint4*>(k_out + dst) = *reinterpret_cast<const uint4*>(pv.k + src);
-        *reinterpret_cast<uint4*>(v_out + dst) = *reinterpret_cast<const uint4*>(pv.v + src);
+    const int i0 = blockIdx.x * EVICT_TOK_PER_CTA, i1 = min(ne, i0 + EVICT_TOK_PER_CTA);
+    __shared__ int s_phys[EVICT_TOK_PER_CTA];          // one block-table look-up per token, not per vector
+    if ((int)threadIdx.x < i1 - i0) {
+        const int phys = kv_page_of(pv, b, tb + i0 + threadIdx.x);
+        s_phys[threadIdx.x] = phys;
+        if (phys < 0 && status) atomicMax(status, HG_DEV_BAD_PAGE);
+    }
+    __syncthreads();
+    const int n_vec = (i1 - i0) * vec_per_tok;
+    constexpr int UNROLL = 4;                           // independent 16-byte K and V loads in flight per thread
+    for (int base = threadIdx.x; base < n_vec; base += UNROLL * blockDim.x) {
+        uint4 kk[UNROLL], vv[UNROLL];
+        int64_t dst[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const int idx = base + u * blockDim.x;
+            dst[u] = -1;
+            if (idx >= n_vec) continue;
+            const int i = idx / vec_per_tok, r = idx - i * vec_per_tok;
+            const int g = r / vec_per_row, c = r - g * vec_per_row;
+            const int phys = s_phys[i];
+            if (phys < 0) continue;
+            const int t = tb + i0 + i;
+            const int64_t src = (int64_t)phys * pv.page_stride + (int64_t)(t & (pv.page_size - 1)) * pv.tok_stride +
+                                (int64_t)g * pv.head_stride + c * 8;
+            dst[u] = (((int64_t)b * max_evict + i0 + i) * pv.Hkv + g) * pv.D + c * 8;
+            kk[u] = *reinterpret_cast<const uint4*>(pv.k + src);
+            vv[u] = *reinterpret_cast<const uint4*>(pv.v + src);
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            if (dst[u] < 0) continue;
+            *reinterpret_cast<uint4*>(k_out + dst[u]) = kk[u];
+            *reinterpret_cast<uint4*>(v_out + dst[u]) = vv[u];
+        }
     }
 }
 
