@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(LG_THREADS) logits_partial_kernel(const Logits
         for (int hh = 0; hh < 8; ++hh)
 #pragma unroll
             for (int v = 0; v < VEC; ++v) acc[hh][v] = 0.f;
-        constexpr int UNROLL = 4;                                  // V rows in flight per warp
+        constexpr int UNROLL = 8;                                  // V rows in flight per warp
         for (int tt = warp; tt < nt; tt += UNROLL * LG_WARPS) {
             uint2 raw[UNROLL];
 #pragma unroll
@@ -114,9 +114,12 @@ __global__ void __launch_bounds__(LG_THREADS) logits_partial_kernel(const Logits
             }
         }
 #pragma unroll
-        for (int hh = 0; hh < 8; ++hh)
+        for (int hh = 0; hh < 8; ++hh) {
+            if (hh < nh) {
 #pragma unroll
-            for (int v = 0; v < VEC; ++v) s_red[((size_t)warp * 8 + hh) * D + lane * VEC + v] = acc[hh][v];
+                for (int v = 0; v < VEC; ++v) s_red[((size_t)warp * 8 + hh) * D + lane * VEC + v] = acc[hh][v];
+            }
+        }
         __syncthreads();
         for (int i = tid; i < nh * D; i += LG_THREADS) {
             const int hh = i / D, d = i - hh * D;
