@@ -226,6 +226,23 @@ def time_extras(w, prob, dev, steps):
         out["host_logits"] = {"tokens": Bh * n_host, "q_heads": w.Hq, "ms": sec * 1e3,
                               "gflops": 2.0 * Bh * n_host * w.Hq * w.D / sec / 1e9,
                               "k_gbs": Bh * n_host * w.Hkv * w.D * 2 / sec / 1e9, "cores": len(os.sched_getaffinity(0))}
+    # ---- the whole hybrid step with Algorithm 1 in the loop: GPU slice + up to 8192 host-held tokens per sequence,
+    #      of which the scheduler lets the CPU stage hand K over
+    n_h = min(min(w.tok_begin), 8192)
+    if n_h >= 512:
+        from paper_2604_18529_b200 import hybrid
+        kh = torch.randn(w.B, n_h, w.Hkv, w.D).to(dt); vh = torch.randn(w.B, n_h, w.Hkv, w.D).to(dt)
+        qh = prob.q.cpu()
+        eng = hybrid.HybridAttentionStep(prob.desc, kh, vh, torch.full((w.B,), n_h, dtype=torch.int32), k_min=128, k_max=1024,
+                                         k_step=128, sinks=4, device=dev)
+        with torch.cuda.device(dev):
+            recs = [eng.step(prob.q, qh, prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end,
+                             prob.out, prob.lse) for _ in range(12)]
+        out["hybrid_step"] = {"host_tokens_per_seq": n_h, "k_min": 128, "k_max": 1024, "k_step": 128,
+                              "steps": [{"k": r.k, "strategy": "post_qk" if r.strategy == 0 else "pre_qk",
+                                         "t_gpu_ms": round(r.t_gpu, 3), "t_cpu_ms": round(r.t_cpu, 3),
+                                         "t_tx_ms": round(r.t_tx, 3), "t_step_ms": round(r.t_step, 3)} for r in recs]}
+        del eng, kh, vh
     # ---- residency: evict 1024 oldest tokens per sequence into staging (state is restored between runs)
     max_evict = 1024
     k_out = torch.empty(w.B, max_evict, w.Hkv, w.D, dtype=dt, device=dev); v_out = torch.empty_like(k_out)

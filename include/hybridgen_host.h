@@ -6,6 +6,8 @@
  *   hg_host_logits            the Logits Calculator (Section 4.2, CPU-side support): scaled logits
  *                             q.k / sqrt(D) of host-resident keys
  *   hg_host_select_topk       Post-QK^T selection (Section 4.3 / 4.5): the K largest scores per row
+ *   hg_host_group_scores      a KV head's token scores from its query heads' logits (their maximum)
+ *   hg_host_gather_logits     the selected tokens' logits out of the full rows
  *   hg_host_select_positions  a Pre-QK^T, position-based selection (Section 4.5): the first `sinks` and the
  *                             last `window` tokens
  *   hg_host_gather_rows       gathers the selected tokens' V rows into a staging buffer for the transfer
@@ -57,6 +59,25 @@ hg_status hg_host_logits(const void* q, const void* k_rows, const int32_t* idx, 
  */
 hg_status hg_host_select_topk(const float* scores, int64_t rows, int64_t stride, const int32_t* n, int32_t k,
                               int32_t* idx_out, int32_t* n_out);
+
+/*
+ * Token scores of a KV head for Post-QK^T selection when `group` query heads share it (they share the
+ * selected token set too): scores[r][i] = max over the group's rows of logits[r * group + j][i], for
+ * i < n[r]; entries from n[r] on are -inf.  logits: [rows * group][stride], scores: [rows][stride].
+ * With group = 1 this is a copy.  The paper leaves the sharing rule open; the maximum keeps every token
+ * that matters to any head of the group.
+ */
+hg_status hg_host_group_scores(const float* logits, int64_t rows, int32_t group, int64_t stride, const int32_t* n,
+                               float* scores);
+
+/*
+ * out[b][h][i] = full[b][h][idx[b][h / G][i]] for i < n_sel[b], -inf beyond: the logits of the chosen
+ * tokens, taken from rows that hold the logits of all host tokens (Post-QK^T computes those anyway).
+ * full: [B][Hq][full_stride], idx: int32 [B][Hkv][K], out: [B][Hq][K] with K = desc->max_selected.
+ * An index outside [0, full_stride) gives -inf.
+ */
+hg_status hg_host_gather_logits(const float* full, int64_t full_stride, const int32_t* idx, const int32_t* n_sel,
+                                float* out, const hg_host_desc* desc);
 
 /*
  * Position-based selection among n_tokens tokens: the first `sinks` and the last `window` of them, at most k

@@ -53,6 +53,31 @@ bool have_avx2() {
 }
 #endif
 
+// ---- row copies into the transfer buffer ----------------------------------------------------------------------
+// The staging buffer is written once and then read by the GPU's copy engine, never by a core: streaming stores
+// put the rows in memory without leaving dirty lines in some core's cache for the engine to chase.
+
+#if defined(__x86_64__)
+__attribute__((target("avx2"))) void copy_row_stream(void* dst, const void* src, size_t bytes) {
+    const __m256i* s = static_cast<const __m256i*>(src);
+    __m256i* d = static_cast<__m256i*>(dst);
+    for (size_t i = 0; i < bytes / 32; ++i) _mm256_stream_si256(d + i, _mm256_loadu_si256(s + i));
+}
+#endif
+
+inline void copy_row(void* dst, const void* src, size_t bytes) {
+#if defined(__x86_64__)
+    if (have_avx2() && bytes % 32 == 0 && (reinterpret_cast<uintptr_t>(dst) & 31u) == 0) { copy_row_stream(dst, src, bytes); return; }
+#endif
+    memcpy(dst, src, bytes);
+}
+
+inline void rows_written() {
+#if defined(__x86_64__)
+    _mm_sfence();                                    // streaming stores are ordered before whatever publishes the buffer
+#endif
+}
+
 // ---- tiled logits: TILE_T token rows of one KV head against the G query heads that share it ------------
 //
 // The rows are converted to fp32 once into a small buffer; every head of the group then takes its dot
@@ -279,16 +304,18 @@ hg_status hg_host_logits(const void* q, const void* k_rows, const int32_t* idx, 
     // Work items: (sequence, block of tokens, KV heads).  When a token's heads lie next to each other in memory
     // (token-major rows) one item sweeps all heads of its tokens, so that memory is read front to back; with
     // head-major rows every KV head is an item of its own stream.
-    constexpr int BLOCK = 256;
     const bool token_major = d->head_stride < d->tok_stride;
     const int g_per_item = token_major ? Hkv : 1;
     const int g_items = Hkv / g_per_item;
-    const int blocks = (K + BLOCK - 1) / BLOCK;
-    // a worker thread costs tens of microseconds to start: give each at least 256 KB of keys to read
+    // a worker thread costs tens of microseconds to wake: give each at least 256 KB of keys to read
     int64_t key_bytes = 0;
     for (int b = 0; b < d->batch; ++b) key_bytes += (int64_t)std::max(0, std::min(n_sel[b], K)) * Hkv * D * 2;
     int workers = d->threads > 0 ? d->threads : (int)std::thread::hardware_concurrency();
     workers = (int)std::max<int64_t>(1, std::min<int64_t>(workers, key_bytes >> 18));
+    // token blocks of up to 256, smaller when that is what it takes to give every worker a few items
+    int BLOCK = 256;
+    while (BLOCK > TILE_T && (int64_t)d->batch * ((K + BLOCK - 1) / BLOCK) * g_items < 4 * (int64_t)workers) BLOCK /= 2;
+    const int blocks = (K + BLOCK - 1) / BLOCK;
     parallel_for((int64_t)d->batch * blocks * g_items, workers, [&](int64_t item) {
         const int gi = (int)(item % g_items);
         const int blk = (int)((item / g_items) % blocks);
@@ -296,27 +323,29 @@ hg_status hg_host_logits(const void* q, const void* k_rows, const int32_t* idx, 
         const int n = std::max(0, std::min(n_sel[b], K));
         const int t0 = blk * BLOCK, t1 = std::min(K, t0 + BLOCK);
         const float ninf = -std::numeric_limits<float>::infinity();
-        for (int g = gi * g_per_item; g < (gi + 1) * g_per_item; ++g) {
-            const uint16_t* kb = kp + (int64_t)b * d->seq_stride + (int64_t)g * d->head_stride;
-            const int32_t* ix = idx ? idx + ((int64_t)b * Hkv + g) * K : nullptr;
-            float* out = logits + ((int64_t)b * Hq + (int64_t)g * G) * K;
-            TileArgs a;
-            a.D = D; a.G = G; a.bf16 = bf16; a.scale = scale; a.out_stride = K;
-            a.qf = qf.data() + ((size_t)b * Hq + (size_t)g * G) * D;
-            for (int t = t0; t < std::min(t1, n); t += TILE_T) {
-                a.valid = std::min(TILE_T, n - t);
+        const int g0 = gi * g_per_item, g1 = g0 + g_per_item;
+        TileArgs a;
+        a.D = D; a.G = G; a.bf16 = bf16; a.scale = scale; a.out_stride = K;
+        // tile by tile, and within a tile head by head: with token-major rows that walks each token's row from
+        // its first head to its last
+        for (int t = t0; t < std::min(t1, n); t += TILE_T) {
+            a.valid = std::min(TILE_T, n - t);
+            for (int g = g0; g < g1; ++g) {
+                const uint16_t* kb = kp + (int64_t)b * d->seq_stride + (int64_t)g * d->head_stride;
+                const int32_t* ix = idx ? idx + ((int64_t)b * Hkv + g) * K : nullptr;
                 for (int i = 0; i < TILE_T; ++i) {
                     const int tt = t + std::min(i, a.valid - 1);
                     const int tn = std::min(tt + TILE_T, n - 1);
                     a.rows[i] = kb + (int64_t)(ix ? ix[tt] : tt) * d->tok_stride;
                     a.next[i] = kb + (int64_t)(ix ? ix[tn] : tn) * d->tok_stride;
                 }
-                a.out = out + t;
+                a.qf = qf.data() + ((size_t)b * Hq + (size_t)g * G) * D;
+                a.out = logits + ((int64_t)b * Hq + (int64_t)g * G) * K + t;
                 tile(a);
             }
-            for (int h = 0; h < G; ++h)
-                for (int t = std::max(t0, n); t < t1; ++t) out[(int64_t)h * K + t] = ninf;
         }
+        for (int h = g0 * G; h < g1 * G; ++h)
+            for (int t = std::max(t0, n); t < t1; ++t) logits[((int64_t)b * Hq + h) * K + t] = ninf;
     });
     return HG_OK;
 }
@@ -343,6 +372,41 @@ hg_status hg_host_select_topk(const float* scores, int64_t rows, int64_t stride,
     return HG_OK;
 }
 
+hg_status hg_host_group_scores(const float* logits, int64_t rows, int32_t group, int64_t stride, const int32_t* n,
+                               float* scores) {
+    if (!logits || !n || !scores || rows < 0 || group < 1 || stride < 1) return HG_ERR_INVALID_ARG;
+    const float ninf = -std::numeric_limits<float>::infinity();
+    parallel_for(rows, 0, [&](int64_t r) {
+        const int64_t nv = std::max<int64_t>(0, std::min<int64_t>(n[r], stride));
+        float* out = scores + r * stride;
+        const float* in = logits + r * group * stride;
+        for (int64_t i = 0; i < nv; ++i) out[i] = in[i];
+        for (int j = 1; j < group; ++j) {
+            const float* row = in + (int64_t)j * stride;
+            for (int64_t i = 0; i < nv; ++i) out[i] = row[i] > out[i] || out[i] != out[i] ? row[i] : out[i];
+        }
+        for (int64_t i = nv; i < stride; ++i) out[i] = ninf;
+    });
+    return HG_OK;
+}
+
+hg_status hg_host_gather_logits(const float* full, int64_t full_stride, const int32_t* idx, const int32_t* n_sel,
+                                float* out, const hg_host_desc* d) {
+    if (!desc_ok(d) || !full || !idx || !n_sel || !out || full_stride < 1) return HG_ERR_INVALID_ARG;
+    const int K = d->max_selected, G = d->num_q_heads / d->num_kv_heads;
+    const float ninf = -std::numeric_limits<float>::infinity();
+    parallel_for((int64_t)d->batch * d->num_q_heads, d->threads, [&](int64_t row) {
+        const int b = (int)(row / d->num_q_heads), h = (int)(row % d->num_q_heads);
+        const int nsel = std::max(0, std::min(n_sel[b], K));
+        const int32_t* ix = idx + ((int64_t)b * d->num_kv_heads + h / G) * K;
+        const float* src = full + row * full_stride;
+        float* o = out + row * K;
+        for (int i = 0; i < nsel; ++i) o[i] = (ix[i] >= 0 && ix[i] < full_stride) ? src[ix[i]] : ninf;
+        for (int i = nsel; i < K; ++i) o[i] = ninf;
+    });
+    return HG_OK;
+}
+
 int32_t hg_host_select_positions(int32_t n_tokens, int32_t sinks, int32_t window, int32_t k, int32_t* idx_out) {
     if (!idx_out || n_tokens <= 0 || k <= 0) return 0;
     sinks = std::max(0, std::min(sinks, n_tokens));
@@ -365,8 +429,9 @@ hg_status hg_host_gather_rows(const void* rows, const int32_t* idx, const int32_
         const int32_t* ix = idx + bg * K;
         uint16_t* o = out + bg * (int64_t)K * D;
         const uint16_t* base = src + (int64_t)b * d->seq_stride + (int64_t)g * d->head_stride;
-        for (int i = 0; i < n; ++i) memcpy(o + (int64_t)i * D, base + (int64_t)ix[i] * d->tok_stride, (size_t)D * 2);
+        for (int i = 0; i < n; ++i) copy_row(o + (int64_t)i * D, base + (int64_t)ix[i] * d->tok_stride, (size_t)D * 2);
         if (n < K) memset(o + (int64_t)n * D, 0, (size_t)(K - n) * D * 2);
+        rows_written();
     });
     return HG_OK;
 }

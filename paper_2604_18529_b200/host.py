@@ -38,6 +38,10 @@ def _lib():
         L.hg_host_logits.restype = C.c_int
         L.hg_host_select_topk.argtypes = [vp, C.c_int64, C.c_int64, vp, C.c_int32, vp, vp]
         L.hg_host_select_topk.restype = C.c_int
+        L.hg_host_group_scores.argtypes = [vp, C.c_int64, C.c_int32, C.c_int64, vp, vp]
+        L.hg_host_group_scores.restype = C.c_int
+        L.hg_host_gather_logits.argtypes = [vp, C.c_int64, vp, vp, vp, C.POINTER(HgHostDesc)]
+        L.hg_host_gather_logits.restype = C.c_int
         L.hg_host_select_positions.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, vp]
         L.hg_host_select_positions.restype = C.c_int32
         L.hg_host_gather_rows.argtypes = [vp, vp, vp, vp, C.POINTER(HgHostDesc)]
@@ -83,6 +87,24 @@ def hg_host_select_topk(scores: torch.Tensor, n: torch.Tensor, k: int):
     _check(_lib().hg_host_select_topk(_host(scores, "scores", torch.float32), rows, stride, _host(n, "n", torch.int32), k,
                                       idx.data_ptr(), n_out.data_ptr()), "hg_host_select_topk")
     return idx, n_out
+
+
+def hg_host_group_scores(logits: torch.Tensor, group: int, n: torch.Tensor, scores: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Per-KV-head token scores [rows // group][stride] from per-query-head logits [rows][stride] (group maximum)."""
+    rows, stride = logits.shape
+    assert rows % group == 0
+    if scores is None:
+        scores = torch.empty(rows // group, stride)
+    _check(_lib().hg_host_group_scores(_host(logits, "logits", torch.float32), rows // group, group, stride,
+                                       _host(n, "n", torch.int32), _host(scores, "scores", torch.float32)), "hg_host_group_scores")
+    return scores
+
+
+def hg_host_gather_logits(full: torch.Tensor, idx: torch.Tensor, n_sel: torch.Tensor, out: torch.Tensor, desc: HgHostDesc) -> None:
+    """out[b][h][i] = full[b][h][idx[b][h // G][i]] for i < n_sel[b], -inf beyond."""
+    _check(_lib().hg_host_gather_logits(_host(full, "full", torch.float32), full.shape[-1], _host(idx, "idx", torch.int32),
+                                        _host(n_sel, "n_sel", torch.int32), _host(out, "out", torch.float32), C.byref(desc)),
+           "hg_host_gather_logits")
 
 
 def hg_host_select_positions(n_tokens: int, sinks: int, window: int, k: int) -> torch.Tensor:

@@ -1,0 +1,163 @@
+"""One layer's hybrid attention step as the paper runs it (Section 4.2 workflow, Section 4.3 scheduler).
+
+The GPU attends the tokens it holds (``hg_attn_partial``) while the CPU stage runs beside it: it picks K
+of the host-held tokens per (sequence, KV head) - Post-QK^T: logits of all host tokens, the K best;
+Pre-QK^T: a position-based set, logits only for it - and ships those logits and the matching V rows.
+The GPU turns them into softmax partials (``hg_attn_partial_from_logits``) and merges both sides
+(``hg_attn_merge``).  The three measured latencies of a step (GPU stage, CPU stage, transfer) drive the
+feedback scheduler (Algorithm 1), which sets K and the strategy of the next step.
+
+This module is plumbing: buffers, two streams, events, clocks and calls.  All arithmetic is in the CUDA
+library and the host library.  The CPU's query is an input here (the paper derives it from the previous
+layer's input; that speculation is outside this package).
+"""
+from __future__ import annotations
+
+import time
+from dataclasses import dataclass
+from typing import List, Optional
+
+import torch
+
+from . import binding as hg
+from . import host as H
+
+POST_QK, PRE_QK = 0, 1
+
+
+@dataclass
+class StepRecord:
+    k: int                 # tokens per (sequence, KV head) the CPU stage handled in this step
+    strategy: int          # POST_QK or PRE_QK
+    t_gpu: float           # ms: the GPU's own partial kernel
+    t_cpu: float           # ms: selection + logits + V-row gather on the host
+    t_tx: float            # ms: host -> device copies of logits, V rows and counts
+    t_step: float          # ms: wall clock of the whole step, results on the device
+
+
+class HybridAttentionStep:
+    """Buffers and control for repeated hybrid steps over one KV configuration.
+
+    ``desc`` describes the GPU slice (as for ``hg_attn_partial``); ``k_host`` / ``v_host`` are the host-held
+    rows ``[B][T][Hkv][D]`` (any strides, D contiguous) of which the first ``n_host[b]`` are valid.
+    """
+
+    def __init__(self, desc: hg.HgAttnDesc, k_host: torch.Tensor, v_host: torch.Tensor, n_host: torch.Tensor,
+                 k_min: int, k_max: int, k_step: int, sinks: int = 4, handoff_chunk: int = 256, host_threads: int = 0,
+                 overlap_transfer: bool = True, device="cuda"):
+        self.desc, self.k_host, self.v_host, self.n_host = desc, k_host, v_host, n_host.to(torch.int32).contiguous()
+        self.dev = torch.device(device)
+        self.B, self.Hq, self.Hkv, self.D = desc.batch, desc.num_q_heads, desc.num_kv_heads, desc.head_dim
+        self.G = self.Hq // self.Hkv
+        self.dtype = k_host.dtype
+        self.sinks, self.chunk, self.threads = sinks, handoff_chunk, host_threads
+        # True: the copies start as soon as the CPU stage has its data, beside the partial kernel if that is still
+        # running; False: they wait for it.  Measured on the OPT-13B shape the two differ by under 2 %.
+        self.overlap_transfer = overlap_transfer
+        self.k_max = k_max
+        self.sched = H.FeedbackScheduler(k_min, k_max, k_step)
+        self.k, self.strategy = k_min, POST_QK
+        self.n_host_max = int(self.n_host.max()) if self.n_host.numel() else 0
+        B, Hq, Hkv, D, NC = self.B, self.Hq, self.Hkv, self.D, desc.num_chunks
+        dev = self.dev
+        # GPU side
+        self.o_part = torch.empty(B, Hq, NC, D, dtype=torch.float32, device=dev)
+        self.m_part = torch.empty(B, Hq, NC, dtype=torch.float32, device=dev)
+        self.l_part = torch.empty(B, Hq, NC, dtype=torch.float32, device=dev)
+        ncs = -(-k_max // handoff_chunk)
+        self.h_o = torch.empty(B * Hq * ncs * D, dtype=torch.float32, device=dev)
+        self.h_m = torch.empty(B * Hq * ncs, dtype=torch.float32, device=dev)
+        self.h_l = torch.empty(B * Hq * ncs, dtype=torch.float32, device=dev)
+        self.d_logits = torch.empty(B * Hq * k_max, dtype=torch.float32, device=dev)
+        self.d_vsel = torch.empty(B * Hkv * k_max * D, dtype=self.dtype, device=dev)
+        self.d_nsel = torch.empty(B, dtype=torch.int32, device=dev)
+        # host side (pinned: the copies are asynchronous)
+        self.p_logits = torch.empty(B * Hq * k_max, dtype=torch.float32).pin_memory()
+        self.p_vsel = torch.empty(B * Hkv * k_max * D, dtype=self.dtype).pin_memory()
+        self.p_nsel = torch.empty(B, dtype=torch.int32).pin_memory()
+        self.full_logits = torch.empty(B, Hq, max(self.n_host_max, 1), dtype=torch.float32)
+        self.scores = torch.empty(B * Hkv, max(self.n_host_max, 1), dtype=torch.float32)
+        self.n_rows = self.n_host.repeat_interleave(Hkv).contiguous()
+        self.idx: Optional[torch.Tensor] = None        # [B][Hkv][k] of the last step
+        self.n_sel: Optional[torch.Tensor] = None      # [B]
+        self.copy_stream = torch.cuda.Stream(device=dev)
+        self.ev = {n: torch.cuda.Event(enable_timing=True) for n in ("g0", "g1", "t0", "t1", "h1")}
+        self.history: List[StepRecord] = []
+        self._plan_k, self._plan_pos = -1, None
+
+    def set_operating_point(self, k: int, strategy: int) -> None:
+        """Override what the scheduler decided (tests, warm starts); the scheduler carries on from here."""
+        self.k, self.strategy = k, strategy
+        self.sched.state.k, self.sched.state.strategy = k, strategy
+
+    # ---- CPU stage ------------------------------------------------------------------------------------------
+    def _cpu_stage(self, q_host: torch.Tensor, k: int):
+        B, Hq, Hkv, D = self.B, self.Hq, self.Hkv, self.D
+        logits = self.p_logits[:B * Hq * k].view(B, Hq, k)
+        vsel = self.p_vsel[:B * Hkv * k * D].view(B, Hkv, k, D)
+        n_sel = self.p_nsel
+        if self._plan_k != k:                       # counts and the position-based set depend on k alone: kept between steps
+            torch.minimum(self.n_host, torch.tensor(k, dtype=torch.int32), out=n_sel)
+            pos = torch.full((B, Hkv, k), -1, dtype=torch.int32)
+            for b in range(B):
+                sel = H.hg_host_select_positions(int(self.n_host[b]), self.sinks, max(k - self.sinks, 0), k)
+                pos[b, :, : len(sel)] = sel
+            self._plan_k, self._plan_pos = k, pos
+        sel_desc = H.host_desc(self.k_host, Hq, k, scale=self.desc.scale, threads=self.threads)
+        if self.strategy == POST_QK and self.n_host_max > 0:
+            full_desc = H.host_desc(self.k_host, Hq, self.n_host_max, scale=self.desc.scale, threads=self.threads)
+            H.hg_host_logits(q_host, self.k_host, None, self.n_host, self.full_logits, full_desc)
+            H.hg_host_group_scores(self.full_logits.view(B * Hq, -1), self.G, self.n_rows, self.scores)
+            idx, _ = H.hg_host_select_topk(self.scores, self.n_rows, k)
+            idx = idx.view(B, Hkv, k)
+            H.hg_host_gather_logits(self.full_logits, idx, n_sel, logits, sel_desc)
+        else:
+            idx = self._plan_pos
+            H.hg_host_logits(q_host, self.k_host, idx, n_sel, logits, sel_desc)
+        H.hg_host_gather_rows(self.v_host, idx, n_sel, vsel, sel_desc)
+        self.idx, self.n_sel = idx, n_sel.clone()
+        return logits, vsel, n_sel
+
+    # ---- one step ---------------------------------------------------------------------------------------------
+    def step(self, q_dev, q_host, k_cache, v_cache, seq_lens, tok_begin, tok_end, out, lse) -> StepRecord:
+        B, Hq, Hkv, D = self.B, self.Hq, self.Hkv, self.D
+        k, ev = self.k, self.ev
+        main = torch.cuda.current_stream(self.dev)
+        t_wall = time.perf_counter()
+        # GPU stage: enqueued first, runs while the host works
+        ev["g0"].record(main)
+        hg.hg_attn_partial(q_dev, k_cache, v_cache, seq_lens, tok_begin, tok_end, self.o_part, self.m_part, self.l_part,
+                           self.desc, main)
+        ev["g1"].record(main)
+        # CPU stage
+        t0 = time.perf_counter()
+        logits, vsel, n_sel = self._cpu_stage(q_host, k)
+        t_cpu = (time.perf_counter() - t0) * 1e3
+        # transfer and hand-off partials on the second stream
+        ld = hg.logits_desc(batch=B, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, dtype=self.dtype, max_selected=k,
+                            chunk_tokens=self.chunk)
+        ncs = ld.num_chunks
+        d_logits = self.d_logits[:B * Hq * k].view(B, Hq, k)
+        d_vsel = self.d_vsel[:B * Hkv * k * D].view(B, Hkv, k, D)
+        h_o = self.h_o[:B * Hq * ncs * D].view(B, Hq, ncs, D)
+        h_m = self.h_m[:B * Hq * ncs].view(B, Hq, ncs)
+        h_l = self.h_l[:B * Hq * ncs].view(B, Hq, ncs)
+        cs = self.copy_stream
+        with torch.cuda.stream(cs):
+            if not self.overlap_transfer:
+                cs.wait_event(ev["g1"])
+            ev["t0"].record(cs)
+            d_logits.copy_(logits, non_blocking=True)
+            d_vsel.copy_(vsel, non_blocking=True)
+            self.d_nsel.copy_(n_sel, non_blocking=True)
+            ev["t1"].record(cs)
+            hg.hg_attn_partial_from_logits(d_logits, d_vsel, self.d_nsel, h_o, h_m, h_l, ld, cs)
+            ev["h1"].record(cs)
+        main.wait_event(ev["h1"])
+        hg.hg_attn_merge([(self.o_part, self.m_part, self.l_part), (h_o, h_m, h_l)], out, lse, self.desc, main)
+        main.synchronize()
+        rec = StepRecord(k=k, strategy=self.strategy, t_gpu=ev["g0"].elapsed_time(ev["g1"]), t_cpu=t_cpu,
+                         t_tx=ev["t0"].elapsed_time(ev["t1"]), t_step=(time.perf_counter() - t_wall) * 1e3)
+        self.history.append(rec)
+        self.k, self.strategy = self.sched.update(rec.t_gpu, rec.t_cpu, rec.t_tx)      # Algorithm 1, for the next step
+        return rec

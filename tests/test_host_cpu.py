@@ -110,6 +110,34 @@ def test_topk_selection_matches_the_sort_definition():
             assert idx[r, : len(want)].tolist() == want and (idx[r, len(want):] == -1).all()
 
 
+def test_group_scores_and_logit_gather():
+    rng = np.random.default_rng(9)
+    rows, group, stride = 6, 3, 41
+    lg = rng.standard_normal((rows * group, stride)).astype(np.float32)
+    lg[4, 7] = np.nan                                         # a NaN loses to any number
+    n = np.array([41, 0, 17, 41, 1, 30], dtype=np.int32)
+    got = H.hg_host_group_scores(torch.from_numpy(lg), group, torch.from_numpy(n)).numpy()
+    for r in range(rows):
+        want = np.fmax.reduce(lg[r * group:(r + 1) * group, : n[r]], axis=0) if n[r] else np.empty(0)
+        assert np.array_equal(got[r, : n[r]], want)
+        assert np.isneginf(got[r, n[r]:]).all()
+    # gather: [B][Hq][full] -> [B][Hq][K] through idx [B][Hkv][K]
+    B, Hkv, G, D, full, K = 2, 2, 3, 64, 50, 8
+    fl = torch.from_numpy(rng.standard_normal((B, Hkv * G, full)).astype(np.float32))
+    idx = torch.from_numpy(rng.integers(0, full, (B, Hkv, K)).astype(np.int32))
+    idx[1, 0, 2] = full + 3                                   # out of range: -inf, never read
+    n_sel = torch.tensor([8, 5], dtype=torch.int32)
+    desc = H.host_desc(torch.zeros(B, 1, Hkv, D, dtype=torch.float16), Hkv * G, K)
+    out = torch.empty(B, Hkv * G, K)
+    H.hg_host_gather_logits(fl, idx, n_sel, out, desc)
+    for b in range(B):
+        for h in range(Hkv * G):
+            for i in range(K):
+                j = int(idx[b, h // G, i])
+                want = fl[b, h, j].item() if i < int(n_sel[b]) and 0 <= j < full else -np.inf
+                assert out[b, h, i].item() == want
+
+
 def test_position_selection():
     for n_tokens, sinks, window, k in itertools.product([0, 1, 5, 100, 2000], [0, 4], [0, 3, 1024], [1, 6, 5000]):
         got = H.hg_host_select_positions(n_tokens, sinks, window, k).tolist()

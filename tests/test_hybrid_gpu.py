@@ -1,0 +1,87 @@
+"""The whole hybrid step (GPU slice + CPU-selected host tokens, Algorithm 1 in the loop) against the oracle.
+
+Every step's output must equal monolithic attention over exactly the tokens that took part in it - the GPU
+slice plus the host tokens the CPU stage chose in that step - and the (K, strategy) sequence must be what
+Algorithm 1 gives on the latencies the steps measured.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import hg_oracle as O
+from oracle import hg_policy as P
+from paper_2604_18529_b200 import hybrid
+from paper_2604_18529_b200 import workload as W
+from paper_2604_18529_b200.problem import DeviceProblem
+from parity_util import LSE_ABS, OUT_MAX_ABS, OUT_REL_L2, bits
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def reference(w, q, K, V, idx, n_sel, G):
+    out = np.zeros((w.B, w.Hq, w.D)); lse = np.zeros((w.B, w.Hq))
+    for b in range(w.B):
+        for h in range(w.Hq):
+            g = h // G
+            host = idx[b, g, : int(n_sel[b])].numpy().astype(np.int64)
+            assert len(set(host.tolist())) == len(host) and (host >= 0).all() and (host < w.tok_begin[b]).all()
+            tokens = np.concatenate([host, np.arange(w.tok_begin[b], w.tok_end[b])])
+            out[b, h], lse[b, h] = O.full(q[b, h], np.ascontiguousarray(K[b, :, g]), np.ascontiguousarray(V[b, :, g]),
+                                          w.dtype, idx=tokens)
+    return out, lse
+
+
+@pytest.mark.parametrize("G,dtype", [(1, "f16"), (4, "bf16")])
+def test_hybrid_steps_match_attention_over_the_tokens_they_used(G, dtype):
+    w = W.AttnWorkload("hyb", 2, 2 * G, 2, 128, dtype, [1500, 700], [1100, 420], [1500, 700], page_size=16,
+                       chunk_tokens=128, seed=90 + G, outlier_frac=0.02)
+    q_t, K_t, V_t = w.q(), w.kv_logical("k"), w.kv_logical("v")
+    prob = DeviceProblem(w, DEV)
+    n_host = torch.tensor(w.tok_begin, dtype=torch.int32)                 # the host holds [0, tok_begin)
+    eng = hybrid.HybridAttentionStep(prob.desc, K_t, V_t, n_host, k_min=32, k_max=160, k_step=32, sinks=4,
+                                     handoff_chunk=64, host_threads=2, device=DEV)
+    q, K, V = bits(q_t), bits(K_t), bits(V_t)
+    seen = set()
+    for step in range(8):
+        if step == 4:                                                     # force the other strategy for the rest
+            eng.set_operating_point(eng.k, hybrid.PRE_QK if eng.strategy == hybrid.POST_QK else hybrid.POST_QK)
+        k_used, strat_used = eng.k, eng.strategy
+        with torch.cuda.device(DEV):
+            rec = eng.step(prob.q, q_t, prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end,
+                           prob.out, prob.lse)
+        assert (rec.k, rec.strategy) == (k_used, strat_used)
+        assert rec.t_gpu > 0 and rec.t_cpu > 0 and rec.t_tx > 0 and rec.t_step >= rec.t_cpu
+        assert eng.idx.shape == (w.B, w.Hkv, k_used)
+        assert [int(x) for x in eng.n_sel] == [min(k_used, n) for n in w.tok_begin]
+        if strat_used == hybrid.PRE_QK:                                   # sinks + the most recent host tokens
+            for b in range(w.B):
+                want = P.positions(w.tok_begin[b], 4, max(k_used - 4, 0), k_used)
+                assert eng.idx[b, 0, : len(want)].tolist() == want
+        ref_out, ref_lse = reference(w, q, K, V, eng.idx, eng.n_sel, G)
+        out, lse = prob.out.double().cpu().numpy(), prob.lse.double().cpu().numpy()
+        assert np.abs(out - ref_out).max() <= OUT_MAX_ABS
+        assert np.linalg.norm(out - ref_out) / np.linalg.norm(ref_out) <= OUT_REL_L2
+        assert np.abs(lse - ref_lse).max() <= LSE_ABS
+        # Algorithm 1 on the latencies this step measured gives the next step's K and strategy
+        assert (eng.k, eng.strategy) == P.feedback_scheduler_step(k_used, strat_used, rec.t_gpu, rec.t_cpu, rec.t_tx, 32, 160, 32)
+        seen.add(strat_used)
+    assert seen == {hybrid.POST_QK, hybrid.PRE_QK}
+    assert len(eng.history) == 8
+
+
+def test_post_qk_picks_the_heaviest_host_tokens():
+    """With a few host tokens made to dominate (keys aligned with the query), Post-QK^T selection finds them."""
+    w = W.AttnWorkload("heavy", 1, 2, 2, 128, "f16", [900], [600], [900], page_size=16, chunk_tokens=128, seed=5)
+    q_t, K_t, V_t = w.q(), w.kv_logical("k").clone(), w.kv_logical("v")
+    heavy = [17, 250, 333, 599]
+    for g in range(w.Hkv):
+        for t in heavy:
+            K_t[0, t, g] = (q_t[0, g].float() * 3).half()                   # logit = 3 |q|^2 / sqrt(D): far above the rest
+    prob = DeviceProblem(w, DEV)
+    eng = hybrid.HybridAttentionStep(prob.desc, K_t, V_t, torch.tensor([600], dtype=torch.int32), k_min=8, k_max=8, k_step=8,
+                                     handoff_chunk=32, device=DEV)
+    with torch.cuda.device(DEV):
+        eng.step(prob.q, q_t, prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end, prob.out, prob.lse)
+    for g in range(w.Hkv):
+        assert set(heavy) <= set(eng.idx[0, g].tolist())
