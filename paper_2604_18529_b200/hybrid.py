@@ -57,7 +57,7 @@ class HybridAttentionStep:
         self.k_max = k_max
         self.sched = H.FeedbackScheduler(k_min, k_max, k_step)
         self.k, self.strategy = k_min, POST_QK
-        self.n_host_max = int(self.n_host.max()) if self.n_host.numel() else 0
+        self.capacity = k_host.shape[1]                 # host rows per sequence the buffers are sized for
         B, Hq, Hkv, D, NC = self.B, self.Hq, self.Hkv, self.D, desc.num_chunks
         dev = self.dev
         # GPU side
@@ -75,15 +75,24 @@ class HybridAttentionStep:
         self.p_logits = torch.empty(B * Hq * k_max, dtype=torch.float32).pin_memory()
         self.p_vsel = torch.empty(B * Hkv * k_max * D, dtype=self.dtype).pin_memory()
         self.p_nsel = torch.empty(B, dtype=torch.int32).pin_memory()
-        self.full_logits = torch.empty(B, Hq, max(self.n_host_max, 1), dtype=torch.float32)
-        self.scores = torch.empty(B * Hkv, max(self.n_host_max, 1), dtype=torch.float32)
-        self.n_rows = self.n_host.repeat_interleave(Hkv).contiguous()
+        self.full_logits = torch.empty(B * Hq * max(self.capacity, 1), dtype=torch.float32)
+        self.scores = torch.empty(B * Hkv * max(self.capacity, 1), dtype=torch.float32)
         self.idx: Optional[torch.Tensor] = None        # [B][Hkv][k] of the last step
         self.n_sel: Optional[torch.Tensor] = None      # [B]
         self.copy_stream = torch.cuda.Stream(device=dev)
         self.ev = {n: torch.cuda.Event(enable_timing=True) for n in ("g0", "g1", "t0", "t1", "h1")}
         self.history: List[StepRecord] = []
         self._plan_k, self._plan_pos = -1, None
+        self.set_host_tokens(self.n_host)
+
+    def set_host_tokens(self, n_host: torch.Tensor) -> None:
+        """The host now holds the first ``n_host[b]`` rows of every sequence (after an eviction, say)."""
+        self.n_host = n_host.to(torch.int32).contiguous()
+        self.n_host_max = int(self.n_host.max()) if self.n_host.numel() else 0
+        if self.n_host_max > self.capacity:
+            raise ValueError("more host tokens than the host rows hold")
+        self.n_rows = self.n_host.repeat_interleave(self.Hkv).contiguous()
+        self._plan_k = -1
 
     def set_operating_point(self, k: int, strategy: int) -> None:
         """Override what the scheduler decided (tests, warm starts); the scheduler carries on from here."""
@@ -105,12 +114,15 @@ class HybridAttentionStep:
             self._plan_k, self._plan_pos = k, pos
         sel_desc = H.host_desc(self.k_host, Hq, k, scale=self.desc.scale, threads=self.threads)
         if self.strategy == POST_QK and self.n_host_max > 0:
-            full_desc = H.host_desc(self.k_host, Hq, self.n_host_max, scale=self.desc.scale, threads=self.threads)
-            H.hg_host_logits(q_host, self.k_host, None, self.n_host, self.full_logits, full_desc)
-            H.hg_host_group_scores(self.full_logits.view(B * Hq, -1), self.G, self.n_rows, self.scores)
-            idx, _ = H.hg_host_select_topk(self.scores, self.n_rows, k)
+            n_max = self.n_host_max
+            full = self.full_logits[:B * Hq * n_max].view(B, Hq, n_max)
+            scores = self.scores[:B * Hkv * n_max].view(B * Hkv, n_max)
+            full_desc = H.host_desc(self.k_host, Hq, n_max, scale=self.desc.scale, threads=self.threads)
+            H.hg_host_logits(q_host, self.k_host, None, self.n_host, full, full_desc)
+            H.hg_host_group_scores(full.view(B * Hq, n_max), self.G, self.n_rows, scores)
+            idx, _ = H.hg_host_select_topk(scores, self.n_rows, k)
             idx = idx.view(B, Hkv, k)
-            H.hg_host_gather_logits(self.full_logits, idx, n_sel, logits, sel_desc)
+            H.hg_host_gather_logits(full, idx, n_sel, logits, sel_desc)
         else:
             idx = self._plan_pos
             H.hg_host_logits(q_host, self.k_host, idx, n_sel, logits, sel_desc)
@@ -161,3 +173,37 @@ class HybridAttentionStep:
         self.history.append(rec)
         self.k, self.strategy = self.sched.update(rec.t_gpu, rec.t_cpu, rec.t_tx)      # Algorithm 1, for the next step
         return rec
+
+
+class HostKvStore:
+    """The host tier of the cache: pinned rows ``k``, ``v`` ``[B][capacity][Hkv][D]`` holding, for every sequence,
+    its oldest tokens in original order - row i is absolute token i, ``n[b]`` rows valid - i.e. the prefix
+    ``[0, tok_begin[b])`` that the Eviction Engine (Section 4.2) has moved off the GPU."""
+
+    def __init__(self, batch: int, capacity: int, num_kv_heads: int, head_dim: int, dtype: torch.dtype):
+        self.k = torch.zeros(batch, capacity, num_kv_heads, head_dim, dtype=dtype).pin_memory()
+        self.v = torch.zeros(batch, capacity, num_kv_heads, head_dim, dtype=dtype).pin_memory()
+        self.n = torch.zeros(batch, dtype=torch.int32)
+        self.capacity = capacity
+
+    def evict_from_gpu(self, k_cache, v_cache, tok_begin, tok_end, n_evict: List[int], desc: hg.HgAttnDesc,
+                       freed: Optional[torch.Tensor] = None, n_freed: Optional[torch.Tensor] = None) -> None:
+        """Move the oldest ``n_evict[b]`` tokens of every GPU slice here: ``hg_kv_evict`` into a device staging
+        buffer, one device -> host copy per sequence to the end of that sequence's rows, counts advanced.
+        ``n_evict`` must not exceed the slices (the caller knows its own ranges); returns when the rows are here."""
+        B, dev = len(n_evict), k_cache.device
+        max_evict = max(max(n_evict), 1)
+        if any(int(self.n[b]) + n_evict[b] > self.capacity for b in range(B)):
+            raise ValueError("host rows full")
+        Hkv, D = self.k.shape[2], self.k.shape[3]
+        k_out = torch.empty(B, max_evict, Hkv, D, dtype=self.k.dtype, device=dev)
+        v_out = torch.empty_like(k_out)
+        hg.hg_kv_evict(k_cache, v_cache, tok_begin, tok_end, torch.tensor(n_evict, dtype=torch.int32, device=dev), k_out, v_out,
+                       freed, n_freed, desc)
+        for b in range(B):
+            n0, ne = int(self.n[b]), n_evict[b]
+            if ne:
+                self.k[b, n0:n0 + ne].copy_(k_out[b, :ne], non_blocking=True)
+                self.v[b, n0:n0 + ne].copy_(v_out[b, :ne], non_blocking=True)
+            self.n[b] = n0 + ne
+        torch.cuda.current_stream(dev).synchronize()

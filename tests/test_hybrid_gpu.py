@@ -85,3 +85,53 @@ def test_post_qk_picks_the_heaviest_host_tokens():
         eng.step(prob.q, q_t, prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end, prob.out, prob.lse)
     for g in range(w.Hkv):
         assert set(heavy) <= set(eng.idx[0, g].tolist())
+
+
+def test_decode_loop_with_append_eviction_and_exact_hybrid_attention():
+    """The cache's whole life: every step appends the new token's K/V on the GPU; when a slice outgrows its
+    budget the oldest tokens move to the host store; attention is the hybrid step with K large enough to take
+    every host token, so each step must equal monolithic attention over the whole sequence so far."""
+    import dataclasses
+    import paper_2604_18529_b200 as pkg
+    from test_kv_residency_gpu import poison_future_rows, rows_at
+    G, steps, budget, evict_n = 2, 12, 200, 64
+    final = W.AttnWorkload("loop", 2, 2 * G, 2, 128, "f16", [400, 260], [0, 0], [400, 260], page_size=16, chunk_tokens=128,
+                           seed=123)
+    start = [L - steps for L in final.seq_lens]
+    prob = DeviceProblem(final, DEV)                      # pool and block table sized for the final lengths
+    poison_future_rows(prob, final, start)
+    prob.seq_lens = torch.tensor(start, dtype=torch.int32, device=DEV)
+    prob.tok_end = torch.tensor(start, dtype=torch.int32, device=DEV)
+    store = hybrid.HostKvStore(final.B, 512, final.Hkv, final.D, torch.float16)
+    eng = hybrid.HybridAttentionStep(prob.desc, store.k, store.v, store.n, k_min=512, k_max=512, k_step=64, handoff_chunk=128,
+                                     device=DEV)
+    q_t = final.q()
+    q, K, V = bits(q_t), bits(final.kv_logical("k")), bits(final.kv_logical("v"))
+    tb = [0, 0]
+    evictions = 0
+    with torch.cuda.device(DEV):
+        for s in range(steps):
+            t_new = [a + s for a in start]
+            pkg.hg_kv_append(rows_at(final, "k", t_new), rows_at(final, "v", t_new), prob.kv["k"], prob.kv["v"],
+                             prob.seq_lens, prob.tok_end, prob.desc)
+            lens = [t + 1 for t in t_new]
+            n_evict = [evict_n if lens[b] - tb[b] > budget else 0 for b in range(final.B)]
+            if any(n_evict):
+                store.evict_from_gpu(prob.kv["k"], prob.kv["v"], prob.tok_begin, prob.tok_end, n_evict, prob.desc)
+                tb = [a + n for a, n in zip(tb, n_evict)]
+                eng.set_host_tokens(store.n)
+                evictions += 1
+            assert prob.tok_begin.tolist() == tb == store.n.tolist() and prob.tok_end.tolist() == lens
+            for b in range(final.B):                      # the host rows are the sequence's prefix, bit for bit
+                for g in range(final.Hkv):
+                    assert torch.equal(store.k[b, : tb[b], g], final.kv_rows("k", b, g, 0, tb[b]))
+                    assert torch.equal(store.v[b, : tb[b], g], final.kv_rows("v", b, g, 0, tb[b]))
+            eng.set_operating_point(512, hybrid.POST_QK if s % 2 == 0 else hybrid.PRE_QK)
+            eng.step(prob.q, q_t, prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end, prob.out, prob.lse)
+            assert int(prob.status.item()) == 0
+            ref_out, ref_lse = O.full_batch(q, K, V, final.dtype, [0, 0], lens)
+            out, lse = prob.out.double().cpu().numpy(), prob.lse.double().cpu().numpy()
+            assert np.abs(out - ref_out).max() <= OUT_MAX_ABS, s
+            assert np.linalg.norm(out - ref_out) / np.linalg.norm(ref_out) <= OUT_REL_L2, s
+            assert np.abs(lse - ref_lse).max() <= LSE_ABS, s
+    assert evictions >= 3 and tb[0] > tb[1] >= 0
