@@ -356,17 +356,28 @@ hg_status hg_host_select_topk(const float* scores, int64_t rows, int64_t stride,
     parallel_for(rows, 0, [&](int64_t r) {
         const float* s = scores + r * stride;
         const int nv = (int)std::max<int64_t>(0, std::min<int64_t>(n[r], stride));
-        std::vector<int32_t> cand;
-        cand.reserve(nv);
-        for (int i = 0; i < nv; ++i) if (!(s[i] != s[i])) cand.push_back(i);      // NaN is never selected
-        const int take = std::min<int>(k, (int)cand.size());
-        auto better = [&](int32_t a, int32_t b) { return s[a] > s[b] || (s[a] == s[b] && a < b); };
-        if (take < (int)cand.size()) std::nth_element(cand.begin(), cand.begin() + take, cand.end(), better);
-        cand.resize(take);
-        std::sort(cand.begin(), cand.end());
+        // value of the k-th largest score (NaN left out), then one pass in index order: everything above it, and of
+        // the scores equal to it the lowest indices until k are taken - the same set as sorting by (-score, index)
+        std::vector<float> vals;
+        vals.reserve(nv);
+        for (int i = 0; i < nv; ++i) if (s[i] == s[i]) vals.push_back(s[i]);
+        const int take = std::min<int>(k, (int)vals.size());
         int32_t* out = idx_out + r * k;
-        for (int i = 0; i < take; ++i) out[i] = cand[i];
-        for (int i = take; i < k; ++i) out[i] = -1;
+        int w = 0;
+        if (take == (int)vals.size()) {
+            for (int i = 0; i < nv; ++i) if (s[i] == s[i]) out[w++] = i;
+        } else if (take > 0) {
+            std::nth_element(vals.begin(), vals.begin() + (take - 1), vals.end(), std::greater<float>());
+            const float kth = vals[take - 1];
+            int above = 0;
+            for (int i = 0; i < nv; ++i) above += s[i] > kth;
+            int ties = take - above;                           // how many scores equal to kth still fit
+            for (int i = 0; i < nv && w < take; ++i) {
+                if (s[i] > kth) out[w++] = i;
+                else if (s[i] == kth && ties > 0) { out[w++] = i; --ties; }
+            }
+        }
+        for (int i = w; i < k; ++i) out[i] = -1;
         if (n_out) n_out[r] = take;
     });
     return HG_OK;

@@ -110,6 +110,21 @@ def test_topk_selection_matches_the_sort_definition():
             assert idx[r, : len(want)].tolist() == want and (idx[r, len(want):] == -1).all()
 
 
+def test_topk_with_many_ties_and_nans_matches_the_sort_definition():
+    rng = np.random.default_rng(1)
+    for trial in range(30):
+        rows, stride = 5, int(rng.integers(1, 300))
+        sc = rng.integers(-3, 4, (rows, stride)).astype(np.float32)          # seven distinct values: ties everywhere
+        sc[rng.random((rows, stride)) < 0.05] = np.nan
+        n = rng.integers(0, stride + 1, rows).astype(np.int32)
+        k = int(rng.integers(1, 40))
+        idx, n_out = H.hg_host_select_topk(torch.from_numpy(sc), torch.from_numpy(n), k)
+        for r in range(rows):
+            want = P.topk(list(sc[r, : n[r]]), k)
+            assert [i for i in idx[r].tolist() if i >= 0] == want and int(n_out[r]) == len(want)
+            assert idx[r, len(want):].tolist() == [-1] * (k - len(want))
+
+
 def test_group_scores_and_logit_gather():
     rng = np.random.default_rng(9)
     rows, group, stride = 6, 3, 41
