@@ -18,6 +18,8 @@ from .binding import (  # noqa: F401
     hg_attn_decode,
     hg_attn_decode_host,
     prepare_decode_host,
+    prepare_merge,
+    prepare_partial,
     hg_attn_decode_static,
     hg_attn_workspace_bytes,
     hg_status_string,

@@ -286,6 +286,32 @@ def hg_attn_decode_host(q_host, k_cache, v_cache, seq_lens_host, tok_begin_host,
     _check(st, "hg_attn_decode_host")
 
 
+def _prepared(fn, args, keep, where: str):
+    def call(_keep=keep) -> None:
+        st = fn(*args)
+        if st != HG_OK:
+            _check(st, where)
+    return call
+
+
+def prepare_partial(q, k_cache, v_cache, seq_lens, tok_begin, tok_end, o_part, m_part, l_part, desc: HgAttnDesc, stream=None):
+    """``hg_attn_partial`` with its arguments marshalled once: returns a callable for a decode loop that reuses the
+    same buffers (and stream) every step.  The callable keeps the tensors alive."""
+    args = (_dev(q, "q"), _dev(k_cache, "k_cache"), _dev(v_cache, "v_cache"), _dev(seq_lens, "seq_lens", torch.int32),
+            _dev(tok_begin, "tok_begin", torch.int32), _dev(tok_end, "tok_end", torch.int32),
+            _dev(o_part, "o_part", torch.float32), _dev(m_part, "m_part", torch.float32), _dev(l_part, "l_part", torch.float32),
+            _stream(stream), C.byref(desc))
+    keep = (q, k_cache, v_cache, seq_lens, tok_begin, tok_end, o_part, m_part, l_part, desc)
+    return _prepared(lib().hg_attn_partial, args, keep, "hg_attn_partial")
+
+
+def prepare_merge(partials, out, lse, desc: HgAttnDesc, stream=None):
+    """``hg_attn_merge`` with its arguments marshalled once (see ``prepare_partial``)."""
+    arr = _src_array(partials, host=False)
+    args = (arr, len(partials), _dev(out, "out", torch.float32), _dev(lse, "lse", torch.float32), _stream(stream), C.byref(desc))
+    return _prepared(lib().hg_attn_merge, args, (partials, out, lse, desc, arr), "hg_attn_merge")
+
+
 def prepare_decode_host(q_host, k_cache, v_cache, seq_lens_host, tok_begin_host, tok_end_host, host_partials_host,
                         out_host, lse_host, workspace, desc: HgAttnDesc, stream=None):
     """Marshal the arguments of ``hg_attn_decode_host`` once and return a callable that makes the call.
@@ -301,14 +327,7 @@ def prepare_decode_host(q_host, k_cache, v_cache, seq_lens_host, tok_begin_host,
             _dev(workspace, "workspace"), workspace.numel() * workspace.element_size(), _stream(stream), C.byref(desc))
     keep = (q_host, k_cache, v_cache, seq_lens_host, tok_begin_host, tok_end_host, host_partials_host, out_host, lse_host,
             workspace, desc, arr)
-    fn = lib().hg_attn_decode_host
-
-    def call(_keep=keep) -> None:
-        st = fn(*args)
-        if st != HG_OK:
-            _check(st, "hg_attn_decode_host")
-
-    return call
+    return _prepared(lib().hg_attn_decode_host, args, keep, "hg_attn_decode_host")
 
 
 def hg_kv_append(k_new, v_new, k_cache, v_cache, seq_lens, tok_end, desc: HgAttnDesc, stream=None) -> None:

@@ -55,6 +55,20 @@ class DeviceProblem:
         self.partial(stream)
         self.merge(host_partials, stream)
 
+    def prepare_step(self, host_partials, stream=None):
+        """``step`` with the arguments of both calls marshalled once: a callable for timing loops and decode loops
+        that keep their buffers.  Reflects the buffers and description as they are now."""
+        partial = hg.prepare_partial(self.q, self.kv["k"], self.kv["v"], self.seq_lens, self.tok_begin, self.tok_end,
+                                     self.o_part, self.m_part, self.l_part, self.desc, stream)
+        merge = hg.prepare_merge([(self.o_part, self.m_part, self.l_part)] + list(host_partials), self.out, self.lse,
+                                 self.desc, stream)
+
+        def step() -> None:
+            partial()
+            merge()
+
+        return step
+
     def alg_bytes(self) -> int:
         """Algorithmic bytes of one step: the slice's K and V once per KV head, plus q, the block-table
         entries of resident pages, the partials written and read back, and out/lse."""

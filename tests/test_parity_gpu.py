@@ -516,3 +516,27 @@ def test_a_slice_longer_than_num_chunks_is_cut_to_its_first_chunks(G):
     from oracle import hg_oracle as O
     ref_out, ref_lse = O.full_batch(ref.q, ref.K, ref.V, w.dtype, w.tok_begin, kept_end)
     check_output(prob.out, prob.lse, ref_out, ref_lse, "cut")
+
+
+def test_prepared_calls_are_the_same_calls():
+    """prepare_partial / prepare_merge / DeviceProblem.prepare_step marshal once; the launches are identical."""
+    w = wl(Hq=8, Hkv=2)
+    ref = OracleRef(w)
+    prob = DeviceProblem(w, DEV)
+    host = ref.host_partials_device(DEV)
+    prob.step(host)
+    torch.cuda.synchronize()
+    want_o, want_out, want_lse = prob.o_part.clone(), prob.out.clone(), prob.lse.clone()
+    for t in (prob.o_part, prob.m_part, prob.l_part, prob.out, prob.lse):
+        t.fill_(float("nan"))
+    step = prob.prepare_step(host)
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    assert torch.equal(prob.o_part, want_o) and torch.equal(prob.out, want_out) and torch.equal(prob.lse, want_lse)
+    bad = pkg.prepare_merge([(prob.o_part, prob.m_part, prob.l_part)], prob.out, prob.lse,
+                            prob.make_desc(w.chunk_tokens, prob.NC))
+    bad()                                                   # a fresh description: still fine
+    with pytest.raises(ValueError):
+        pkg.prepare_partial(prob.q.cpu(), prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end,
+                            prob.o_part, prob.m_part, prob.l_part, prob.desc)
