@@ -127,7 +127,8 @@ struct LaunchCache {
 };
 
 template <int D, bool BF16, int MODE>
-static hg_status launch_partial_t(const CUtensorMap& tk, const CUtensorMap& tv, PartialParams p, cudaStream_t st) {
+static hg_status launch_partial_t(const CUtensorMap& tk, const CUtensorMap& tv, PartialParams p, cudaStream_t st,
+                                  bool counter_is_zero) {
     static LaunchCache cache;                     // zero-initialised
     const size_t smem = (size_t)p.stages * (2 * TILE_T * D * 2 + 8 * D * 2) + 1024;     // per stage: K tile, V tile, q rows
     auto kern = partial_kernel<D, BF16, MODE>;
@@ -154,6 +155,11 @@ static hg_status launch_partial_t(const CUtensorMap& tk, const CUtensorMap& tv, 
         const long long slots = (long long)p.NC * Y * p.B;
         const long long resident = (long long)cache.sms[dev].load(std::memory_order_relaxed) * per_sm;
         grid = dim3((unsigned)(slots < resident ? slots : resident), 1, 1);
+        if (slots <= resident) p.sched = nullptr;     // at most one item per CTA: nothing to hand out, no counter to clear
+    }
+    if (p.sched && !counter_is_zero && cudaMemsetAsync(p.sched, 0, sizeof(int32_t), st) != cudaSuccess) {
+        cudaGetLastError();
+        return HG_ERR_CUDA;
     }
     kern<<<grid, THREADS, smem, st>>>(tk, tv, p);
     return cudaGetLastError() == cudaSuccess ? HG_OK : HG_ERR_CUDA;
@@ -161,9 +167,12 @@ static hg_status launch_partial_t(const CUtensorMap& tk, const CUtensorMap& tv, 
 
 template <int MODE>
 static hg_status launch_partial_m(int D, bool bf16, const CUtensorMap& tk, const CUtensorMap& tv, const PartialParams& p,
-                                  cudaStream_t st) {
-    if (D == 128) return bf16 ? launch_partial_t<128, true, MODE>(tk, tv, p, st) : launch_partial_t<128, false, MODE>(tk, tv, p, st);
-    return bf16 ? launch_partial_t<64, true, MODE>(tk, tv, p, st) : launch_partial_t<64, false, MODE>(tk, tv, p, st);
+                                  cudaStream_t st, bool counter_is_zero) {
+    if (D == 128)
+        return bf16 ? launch_partial_t<128, true, MODE>(tk, tv, p, st, counter_is_zero)
+                    : launch_partial_t<128, false, MODE>(tk, tv, p, st, counter_is_zero);
+    return bf16 ? launch_partial_t<64, true, MODE>(tk, tv, p, st, counter_is_zero)
+                : launch_partial_t<64, false, MODE>(tk, tv, p, st, counter_is_zero);
 }
 
 static hg_status run_partial(int mode, const void* q, const void* k, const void* v, const int32_t* seq_lens,
@@ -201,15 +210,11 @@ static hg_status run_partial(int mode, const void* q, const void* k, const void*
     p.test_stall = (d->flags & HG_FLAG_TEST_STALL) ? 1 : 0;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     p.sched = p.persistent && env_int("HG_ATTN_DYNAMIC", 1, 0, 1) ? desc_sched(d) : nullptr;
-    if (p.sched && !counter_is_zero && cudaMemsetAsync(p.sched, 0, sizeof(int32_t), cs) != cudaSuccess) {
-        cudaGetLastError();
-        return HG_ERR_CUDA;
-    }
     const bool bf16 = d->dtype == HG_DTYPE_BF16;
     switch (mode) {
-        case MODE_MHA: return launch_partial_m<MODE_MHA>(d->head_dim, bf16, tk, tv, p, cs);
-        case MODE_GQA: return launch_partial_m<MODE_GQA>(d->head_dim, bf16, tk, tv, p, cs);
-        default: return launch_partial_m<MODE_PROBE>(d->head_dim, bf16, tk, tv, p, cs);
+        case MODE_MHA: return launch_partial_m<MODE_MHA>(d->head_dim, bf16, tk, tv, p, cs, counter_is_zero);
+        case MODE_GQA: return launch_partial_m<MODE_GQA>(d->head_dim, bf16, tk, tv, p, cs, counter_is_zero);
+        default: return launch_partial_m<MODE_PROBE>(d->head_dim, bf16, tk, tv, p, cs, counter_is_zero);
     }
 }
 
