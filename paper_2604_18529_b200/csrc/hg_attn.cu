@@ -260,6 +260,15 @@ static hg_status run_merge(const hg_partial_src* src, int32_t n_src, float* out,
     cfg.numAttrs = na;
     auto launch = [&](auto k128, auto k64) { return d->head_dim == 128 ? cudaLaunchKernelEx(&cfg, k128, p) : cudaLaunchKernelEx(&cfg, k64, p); };
     cudaError_t e;
+    // many short rows: a warp per row, eight rows per CTA
+    if (rows >= 2048 && p.total <= 64 && env_int("HG_ATTN_MERGE_ROWS", 1, 0, 1)) {
+        cfg.gridDim = dim3((unsigned)((rows + 7) / 8));
+        cfg.blockDim = dim3(256);
+        e = d->head_dim == 128 ? cudaLaunchKernelEx(&cfg, merge_rows_kernel<128>, p, rows)
+                               : cudaLaunchKernelEx(&cfg, merge_rows_kernel<64>, p, rows);
+        if (e != cudaSuccess) { cudaGetLastError(); return HG_ERR_CUDA; }
+        return HG_OK;
+    }
     switch (cluster) {
         case 8: e = launch(merge_kernel<128, 256, 8>, merge_kernel<64, 256, 8>); break;
         case 4: e = launch(merge_kernel<128, 256, 4>, merge_kernel<64, 256, 4>); break;

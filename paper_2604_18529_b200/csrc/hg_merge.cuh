@@ -7,7 +7,7 @@
 // M_w grows; each lane holds D/32 contiguous output components.  The warps' triples, then the
 // cluster's CTAs' triples, are combined the same way in fixed order, and one division finishes
 // out = sum w o / sum w l and lse = M + ln sum w l.  No atomics: bit-reproducible for a given launch
-// shape.
+// shape.  A second kernel, one warp per row, serves large batches of short rows.
 #pragma once
 
 #include <cooperative_groups.h>
@@ -142,6 +142,71 @@ __global__ void __launch_bounds__(THREADS_) merge_kernel(const MergeParams p) {
         p.out[(size_t)row * D + tid] = empty ? 0.f : o / Lsum;
         if (tid == 0 && p.lse) p.lse[row] = empty ? NEG_INF : M + logf(Lsum);
     }
+}
+
+// Many short rows (a large batch, few chunks each): one WARP per (sequence, query head), eight rows per CTA.
+// The warp sweeps its row's partials in order, four loads in flight, with the same running-maximum rule as
+// above; no shared memory, no barrier.
+template <int D>
+__global__ void __launch_bounds__(256) merge_rows_kernel(const MergeParams p, int rows) {
+    constexpr int VEC = D / 32;
+    const float NEG_INF = __int_as_float(0xff800000);
+    const int lane = threadIdx.x & 31;
+    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+#if __CUDA_ARCH__ >= 900
+    cudaGridDependencySynchronize();
+#endif
+    if (row >= rows) return;
+    float acc[VEC];
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) acc[v] = 0.f;
+    float lsum = 0.f, M = NEG_INF;
+    for (int s = 0; s < p.n_src; ++s) {
+        const int nc = p.nc[s];
+        const float* ms = p.m[s] + (size_t)row * nc;
+        const float* ls = p.l[s] + (size_t)row * nc;
+        const float* os = p.o[s] + (size_t)row * nc * D;
+        for (int i0 = 0; i0 < nc; i0 += 4) {
+            float mi[4], li[4], ov[4][VEC];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = i0 + u;
+                const bool in = i < nc;
+                mi[u] = in ? ms[i] : NEG_INF;
+                li[u] = in ? ls[i] : 0.f;
+                const bool live = in && mi[u] != NEG_INF;
+                const float* orow = os + (size_t)(in ? i : 0) * D + lane * VEC;
+                if constexpr (VEC == 4) {
+                    const float4 v = live ? *reinterpret_cast<const float4*>(orow) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    ov[u][0] = v.x; ov[u][1] = v.y; ov[u][2] = v.z; ov[u][3] = v.w;
+                } else {
+                    const float2 v = live ? *reinterpret_cast<const float2*>(orow) : make_float2(0.f, 0.f);
+                    ov[u][0] = v.x; ov[u][1] = v.y;
+                }
+            }
+            const float m4 = fmaxf(fmaxf(mi[0], mi[1]), fmaxf(mi[2], mi[3]));
+            if (m4 == NEG_INF) continue;
+            if (m4 > M) {
+                const float r = __expf(M - m4);
+                lsum *= r;
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) acc[v] *= r;
+                M = m4;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float w = mi[u] == NEG_INF ? 0.f : __expf(mi[u] - M);
+                lsum = fmaf(w, li[u], lsum);
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) acc[v] = fmaf(w, ov[u][v], acc[v]);
+            }
+        }
+    }
+    const bool empty = (M == NEG_INF);
+    float* out = p.out + (size_t)row * D + lane * VEC;
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) out[v] = empty ? 0.f : acc[v] / lsum;
+    if (lane == 0 && p.lse) p.lse[row] = empty ? NEG_INF : M + logf(lsum);
 }
 
 }  // namespace hg

@@ -540,3 +540,25 @@ def test_prepared_calls_are_the_same_calls():
     with pytest.raises(ValueError):
         pkg.prepare_partial(prob.q.cpu(), prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end,
                             prob.o_part, prob.m_part, prob.l_part, prob.desc)
+
+
+@pytest.mark.parametrize("D,G", [(128, 4), (64, 1)])
+def test_many_short_rows_take_the_warp_per_row_merge(D, G, monkeypatch):
+    """A large batch of short sequences: thousands of (sequence, head) rows with a handful of partials each are
+    merged a warp per row; same result as the CTA-per-row kernel up to summation order."""
+    rng = np.random.default_rng(3)
+    B, Hkv = 300, 2
+    lens = [int(rng.integers(40, 330)) for _ in range(B)]
+    tb = [int(rng.integers(0, L // 2)) for L in lens]
+    te = [int(rng.integers(L // 2, L + 1)) for L in lens]
+    te[5] = tb[5]                                              # an empty slice among them
+    w = W.AttnWorkload("rows", B, Hkv * G * 4, Hkv, D, "f16", lens, tb, te, page_size=16, chunk_tokens=128, seed=41)
+    assert w.B * w.Hq >= 2048
+    prob, ref, _ = run_and_check(w)
+    out_rows, lse_rows = prob.out.clone(), prob.lse.clone()
+    monkeypatch.setenv("HG_ATTN_MERGE_ROWS", "0")
+    prob.merge(ref.host_partials_device(DEV))
+    torch.cuda.synchronize()
+    check_output(prob.out, prob.lse, ref.out, ref.lse, "cta per row")
+    assert (prob.out - out_rows).abs().max().item() <= 1e-5 * max(1.0, out_rows.abs().max().item())
+    assert torch.equal(torch.isinf(prob.lse), torch.isinf(lse_rows))
