@@ -38,7 +38,7 @@ constexpr int THREADS = CONSUMER_THREADS + 32;
 constexpr int MAX_STAGES = 8;
 constexpr int MAX_CHUNK_PAGES = 512;       // chunk_tokens / page_size, any schedule
 constexpr int PERSIST_CHUNK_PAGES = 256;   // ... for the persistent schedule (page ids are double-buffered)
-constexpr int PERSIST_MAX_BATCH = 512;     // sequences the in-kernel item scan handles
+constexpr int PERSIST_MAX_BATCH = 1536;    // sequences the in-kernel item scan handles
 
 enum { MODE_MHA = 0, MODE_GQA = 1, MODE_PROBE = 2 };
 
@@ -71,9 +71,8 @@ struct Control {
     int pages[MAX_CHUNK_PAGES];          // persistent schedule: two buffers, at 0 and at MAX_CHUNK_PAGES / 2
     float red_m[2][32];                  // per-warp running maxima / exp-sums of an item, double-buffered by item parity
     float red_l[2][32];
+    int scan[8];                         // per-warp totals of the set-up scan
     int cum[PERSIST_MAX_BATCH + 1];      // cum[b] = number of items of sequences < b
-    int tb[PERSIST_MAX_BATCH];           // clamped slice of every sequence
-    int te[PERSIST_MAX_BATCH];
 };
 static_assert(PERSIST_CHUNK_PAGES <= MAX_CHUNK_PAGES / 2, "page-id double buffer");
 
@@ -106,7 +105,8 @@ __device__ __forceinline__ void set_range(const PartialParams& p, Item& it, int 
     it.ntiles = it.hi > it.lo ? (it.hi + TILE_T - 1) / TILE_T - it.tile0 : 0;
 }
 
-// Item i of the persistent schedule: items are ordered by (b, y, c); everything it needs is in shared memory.
+// Item i of the persistent schedule: items are ordered by (b, y, c).  Only the producer decodes (it looks ahead, so the
+// three range loads are off the critical path); consumers get the decoded item with the item's first stage.
 __device__ __forceinline__ Item decode_item(const PartialParams& p, const Control& ctl, int i) {
     int lo = 0, hi = p.B;                 // largest b with cum[b] <= i
     while (hi - lo > 1) {
@@ -115,8 +115,8 @@ __device__ __forceinline__ Item decode_item(const PartialParams& p, const Contro
     }
     Item it;
     it.b = lo;
-    const int tb = ctl.tb[lo], te = ctl.te[lo];
-    const int nc = max(te > tb ? min((te + p.C - 1) / p.C - tb / p.C, p.NC) : 0, 1);
+    int tb, te;
+    const int nc = max(seq_chunks(p, lo, tb, te), 1);
     const int r = i - ctl.cum[lo];
     it.y = r / nc;
     it.c = r - it.y * nc;
@@ -139,6 +139,7 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
 
     extern __shared__ uint8_t smem_raw[];
     __shared__ Control ctl;
+    __shared__ Item sitem[MAX_STAGES];   // the decoded item, written by the producer with the item's first stage
     const uint32_t stage0 = (smem_u32(smem_raw) + 1023u) & ~1023u;   // the swizzle pattern is anchored at 1024 bytes
     uint8_t* const stage0_ptr = smem_raw + (stage0 - smem_u32(smem_raw));
 
@@ -171,25 +172,27 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
     }
     int n_items = 1, item_step = 1, item_first = 0;
     if (p.persistent) {
-        // cum[b+1] = sum_{b' <= b} nc_b' * Y : one warp, each lane a contiguous block of sequences
-        if (warp == 0) {
-            const int per = (p.B + 31) / 32;
-            const int b0 = min(p.B, lane * per), b1 = min(p.B, b0 + per);
-            int sum = 0;
-            for (int b = b0; b < b1; ++b) { int tb, te; sum += seq_chunks(p, b, tb, te) * Y; }
-            int incl = sum;
+        // cum[b+1] = sum_{b' <= b} nc_b' * Y : every thread a contiguous block of sequences, warp scan, then the
+        // warps' totals through shared memory
+        const int per = (p.B + THREADS - 1) / THREADS;
+        const int b0 = min(p.B, tid * per), b1 = min(p.B, b0 + per);
+        int sum = 0;
+        for (int b = b0; b < b1; ++b) { int tb, te; sum += seq_chunks(p, b, tb, te) * Y; }
+        int incl = sum;
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int v = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += v;
-            }
-            int run = incl - sum;
-            if (lane == 0) ctl.cum[0] = 0;
-            for (int b = b0; b < b1; ++b) {
-                int tb, te;
-                run += seq_chunks(p, b, tb, te) * Y;
-                ctl.cum[b + 1] = run; ctl.tb[b] = tb; ctl.te[b] = te;
-            }
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) ctl.scan[warp] = incl;
+        __syncthreads();
+        int run = incl - sum;
+        for (int w2 = 0; w2 < warp; ++w2) run += ctl.scan[w2];
+        if (tid == 0) ctl.cum[0] = 0;
+        for (int b = b0; b < b1; ++b) {
+            int tb, te;
+            run += seq_chunks(p, b, tb, te) * Y;
+            ctl.cum[b + 1] = run;
         }
         __syncthreads();
         n_items = ctl.cum[p.B];
@@ -343,6 +346,7 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 const uint32_t qbytes = (MODE != MODE_PROBE && it == 0) ? (uint32_t)q_heads * D * 2u : 0u;
                 if (lane == 0) {
                     ctl.sdesc[s] = make_int2(i_cur, it);
+                    if (it == 0) sitem[s] = cur;
                     mbar_arrive_expect_tx(&ctl.full[s], nvalid * box_bytes + qbytes);
                 }
                 __syncwarp();
@@ -395,8 +399,7 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
             // while the first stage is on its way
             for (int sl = blockIdx.x; sl < p.B * Y; sl += gridDim.x) {
                 const int b = sl / Y, y = sl - b * Y;
-                const int tb = ctl.tb[b], te = ctl.te[b];
-                const int nc = te > tb ? min((te + p.C - 1) / p.C - tb / p.C, p.NC) : 0;
+                const int nc = (ctl.cum[b + 1] - ctl.cum[b]) / Y;
                 const int ne = p.NC - nc;                 // empty slots per head
                 if (ne <= 0) continue;
                 if constexpr (MODE == MODE_PROBE) {
@@ -454,8 +457,8 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
         Item cur;
         cur.b = cur.y = cur.c = cur.lo = cur.hi = cur.tile0 = cur.ntiles = 0;
         int hb = 0, nheads = 1, h0 = 0, par = 1;
-        auto begin_item = [&](int i) {
-            cur = get_item(i);
+        auto begin_item = [&](int s) {
+            cur = sitem[s];
             par ^= 1;
             hb = cur.y % p.head_blocks;
             const int g = cur.y / p.head_blocks;
@@ -469,7 +472,7 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 int2 d;
                 const int s = next_stage(d);
                 if (s < 0) break;
-                if (d.y == 0) { begin_item(d.x); probe_x = 0u; }
+                if (d.y == 0) { begin_item(s); probe_x = 0u; }
                 const uint32_t base = stage0 + s * STAGE_BYTES;
                 const int tokbase = (cur.tile0 + d.y) * TILE_T;
 #pragma unroll
@@ -508,7 +511,7 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 const int s = next_stage(d);
                 if (s < 0) break;
                 if (d.y == 0) {
-                    begin_item(d.x);
+                    begin_item(s);
                     const uint32_t qs = stage0 + s * STAGE_BYTES + 2 * TILE_BYTES;
 #pragma unroll
                     for (int hh = 0; hh < HALVES; ++hh) {
@@ -626,7 +629,7 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 const int s = next_stage(d);
                 if (s < 0) break;
                 if (d.y == 0) {
-                    begin_item(d.x);
+                    begin_item(s);
                     // b0 = q[head quad][16 ks + 2 tq + {0,1}], b1 = the same + 8; heads past the group read as zero
                     const bool live = hb * 8 + quad < p.G;
                     const uint32_t qs = stage0 + s * STAGE_BYTES + 2 * TILE_BYTES + quad * (D * 2);

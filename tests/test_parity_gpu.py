@@ -327,8 +327,10 @@ def test_without_a_work_counter_items_are_dealt_round_robin():
 
 # ---- shapes beyond what the persistent schedule keeps in shared memory fall back to one CTA per item ------------
 
-def test_large_batch_uses_the_per_item_grid():
-    B = 530                                              # more sequences than the in-kernel item scan handles
+@pytest.mark.parametrize("B", [530, 1536, 1540])
+def test_large_batches(B):
+    # up to 1536 sequences the in-kernel item scan (every thread several sequences) feeds the persistent schedule;
+    # beyond that the same kernel runs with one CTA per item
     lens = [40 + (7 * i) % 150 for i in range(B)]
     tb = [(3 * i) % 30 for i in range(B)]
     w = wl(B=B, Hq=2, Hkv=1, D=64, seq_lens=lens, tok_begin=tb, tok_end=lens, chunk_tokens=64, seed=77)
