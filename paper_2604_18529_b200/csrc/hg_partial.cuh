@@ -118,8 +118,17 @@ __device__ __forceinline__ Item decode_item(const PartialParams& p, const Contro
     int tb, te;
     const int nc = max(seq_chunks(p, lo, tb, te), 1);
     const int r = i - ctl.cum[lo];
-    it.y = r / nc;
-    it.c = r - it.y * nc;
+    if (p.head_blocks == 1) {
+        it.y = r / nc;
+        it.c = r - it.y * nc;
+    } else {
+        // groups of more than 8 query heads: the head blocks of one (KV head, chunk) sit next to each other in the
+        // order, so they are taken at about the same time and the second reader finds part of the tiles in L2
+        const int per_g = nc * p.head_blocks;
+        const int g = r / per_g, rem = r - g * per_g;
+        it.c = rem / p.head_blocks;
+        it.y = g * p.head_blocks + (rem - it.c * p.head_blocks);
+    }
     set_range(p, it, tb, te);
     return it;
 }
