@@ -194,13 +194,14 @@ static hg_status run_partial(int mode, const void* q, const void* k, const void*
     st = make_maps(d, k, v, &tk, &tv);
     if (st != HG_OK) return st;
     const int G = d->num_q_heads / d->num_kv_heads;
-    if (mode != MODE_PROBE) mode = (G == 1) ? MODE_MHA : MODE_GQA;
+    // groups of up to 8 query heads: one MMA head block per item; larger groups: items of 16 heads (two blocks)
+    if (mode != MODE_PROBE) mode = (G == 1) ? MODE_MHA : (G <= 8 || !env_int("HG_ATTN_GQA16", 1, 0, 1) ? MODE_GQA : MODE_GQA2);
     p.q = q; p.seq_lens = seq_lens; p.tok_begin = tok_begin; p.tok_end = tok_end; p.block_table = d->block_table;
     p.o_part = o_part; p.m_part = m_part; p.l_part = l_part; p.sink = sink; p.status = d->status;
     p.B = d->batch; p.Hq = d->num_q_heads; p.Hkv = d->num_kv_heads; p.G = G;
     p.page_size = d->page_size; p.page_shift = ilog2_exact(d->page_size); p.max_pages = d->max_pages;
     p.num_pages = d->num_pages; p.C = d->chunk_tokens; p.NC = d->num_chunks;
-    p.head_blocks = (mode == MODE_GQA) ? (G + 7) / 8 : 1;
+    p.head_blocks = (mode == MODE_GQA) ? (G + 7) / 8 : (mode == MODE_GQA2 ? (G + 15) / 16 : 1);
     const float scale = d->scale > 0.f ? d->scale : 1.0f / sqrtf((float)d->head_dim);
     p.scale_log2 = scale * 1.4426950408889634f;
     p.stages = env_int("HG_ATTN_STAGES", d->head_dim == 128 ? 3 : 6, 2, MAX_STAGES);   // 96 KB of ring: 2 CTAs per SM
@@ -214,6 +215,7 @@ static hg_status run_partial(int mode, const void* q, const void* k, const void*
     switch (mode) {
         case MODE_MHA: return launch_partial_m<MODE_MHA>(d->head_dim, bf16, tk, tv, p, cs, counter_is_zero);
         case MODE_GQA: return launch_partial_m<MODE_GQA>(d->head_dim, bf16, tk, tv, p, cs, counter_is_zero);
+        case MODE_GQA2: return launch_partial_m<MODE_GQA2>(d->head_dim, bf16, tk, tv, p, cs, counter_is_zero);
         default: return launch_partial_m<MODE_PROBE>(d->head_dim, bf16, tk, tv, p, cs, counter_is_zero);
     }
 }

@@ -40,7 +40,7 @@ constexpr int MAX_CHUNK_PAGES = 512;       // chunk_tokens / page_size, any sche
 constexpr int PERSIST_CHUNK_PAGES = 256;   // ... for the persistent schedule (page ids are double-buffered)
 constexpr int PERSIST_MAX_BATCH = 1536;    // sequences the in-kernel item scan handles
 
-enum { MODE_MHA = 0, MODE_GQA = 1, MODE_PROBE = 2 };
+enum { MODE_MHA = 0, MODE_GQA = 1, MODE_PROBE = 2, MODE_GQA2 = 3 };   // GQA2: items of 16 query heads (two MMA head blocks)
 
 struct PartialParams {
     const void* q;
@@ -69,8 +69,8 @@ struct Control {
     int2 sdesc[MAX_STAGES];              // what a filled stage holds: x = item index (-1: no more work), y = tile in item
     int abort_flag;
     int pages[MAX_CHUNK_PAGES];          // persistent schedule: two buffers, at 0 and at MAX_CHUNK_PAGES / 2
-    float red_m[2][32];                  // per-warp running maxima / exp-sums of an item, double-buffered by item parity
-    float red_l[2][32];
+    float red_m[2][64];                  // per-warp running maxima / exp-sums of an item (4 warps x up to 16 heads),
+    float red_l[2][64];                  // double-buffered by item parity
     int scan[8];                         // per-warp totals of the set-up scan
     int cum[PERSIST_MAX_BATCH + 1];      // cum[b] = number of items of sequences < b
 };
@@ -144,6 +144,9 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
     constexpr int NV = 8 * HALVES;     // MHA: d-components owned by a lane
     constexpr int KSTEPS = D / 16;     // GQA: 16-wide steps along d
     constexpr float LN2 = 0.6931471805599453f;
+    constexpr bool GQA = MODE == MODE_GQA || MODE == MODE_GQA2;
+    constexpr int NB = MODE == MODE_GQA2 ? 2 : 1;        // MMA head blocks (8 query heads each) per item
+    constexpr int HPI = 8 * NB;                          // query heads per item
     const float NEG_INF = __int_as_float(0xff800000);
 
     extern __shared__ uint8_t smem_raw[];
@@ -237,8 +240,8 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 if (tid == 0) p.sink[((size_t)it.b * p.Hkv + it.y) * p.NC + it.c] = 0u;
             } else {
                 const int hb = it.y % p.head_blocks, g = it.y / p.head_blocks;
-                const int nh = (MODE == MODE_GQA) ? min(8, p.G - hb * 8) : 1;
-                const int hq0 = (MODE == MODE_GQA) ? g * p.G + hb * 8 : g;
+                const int nh = GQA ? min(HPI, p.G - hb * HPI) : 1;
+                const int hq0 = GQA ? g * p.G + hb * HPI : g;
                 for (int i = tid; i < nh * D; i += THREADS)
                     p.o_part[(((size_t)it.b * p.Hq + hq0 + i / D) * p.NC + it.c) * D + i % D] = 0.f;
                 if (tid < nh) {
@@ -341,8 +344,8 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 }
             };
             const int g = cur.y / p.head_blocks;
-            const int q_heads = (MODE == MODE_GQA) ? min(8, p.G - (cur.y % p.head_blocks) * 8) : 1;
-            const int q_head0 = (MODE == MODE_GQA) ? g * p.G + (cur.y % p.head_blocks) * 8 : g;
+            const int q_heads = GQA ? min(HPI, p.G - (cur.y % p.head_blocks) * HPI) : 1;
+            const int q_head0 = GQA ? g * p.G + (cur.y % p.head_blocks) * HPI : g;
             for (int it = 0; it < cur.ntiles; ++it) {              // one stage = K tile + V tile of 64 tokens
                 int okw = 1;
                 if (lane == 0) okw = mbar_wait(&ctl.empty[s], ph ^ 1u, abort_flag) ? 1 : 0;
@@ -352,7 +355,8 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 int phys = -1;
                 if (isv < 2 && t0j < cur.hi && t0j + R > cur.lo) phys = pages[(t0j >> p.page_shift) - page0];
                 const uint32_t nvalid = __popc(__ballot_sync(0xffffffffu, phys >= 0));   // K and V boxes
-                const uint32_t qbytes = (MODE != MODE_PROBE && it == 0) ? (uint32_t)q_heads * D * 2u : 0u;
+                // (items of 16 heads fetch their query rows themselves: the stage's q slot holds 8)
+                const uint32_t qbytes = (MODE != MODE_PROBE && NB == 1 && it == 0) ? (uint32_t)q_heads * D * 2u : 0u;
                 if (lane == 0) {
                     ctl.sdesc[s] = make_int2(i_cur, it);
                     if (it == 0) sitem[s] = cur;
@@ -415,8 +419,8 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                     for (int i = tid; i < ne; i += CONSUMER_THREADS) p.sink[((size_t)b * p.Hkv + y) * p.NC + nc + i] = 0u;
                 } else {
                     const int hb = y % p.head_blocks, g = y / p.head_blocks;
-                    const int nh = (MODE == MODE_GQA) ? min(8, p.G - hb * 8) : 1;
-                    const int hq0 = (MODE == MODE_GQA) ? g * p.G + hb * 8 : g;
+                    const int nh = GQA ? min(HPI, p.G - hb * HPI) : 1;
+                    const int hq0 = GQA ? g * p.G + hb * HPI : g;
                     for (int i = tid; i < nh * ne * D; i += CONSUMER_THREADS) {
                         const int e = i / D, hh = e / ne, cc = nc + e % ne;
                         p.o_part[(((size_t)b * p.Hq + hq0 + hh) * p.NC + cc) * D + i % D] = 0.f;
@@ -448,9 +452,12 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
             if (lane == 0) mbar_arrive(&ctl.empty[s]);
         };
         // Scratch of the item epilogue: consumer warp w2 parks its state in the memory of its own 16 K rows of
-        // the item's last stage (nobody else reads those rows): 2 KB per 64-element column half.
+        // the item's last stage (nobody else reads those rows): 2 KB per 64-element column half; a second block of 8
+        // heads goes to its 16 V rows of the same stage.
         auto warp_scratch = [&](int s, int w2, int float_idx) -> float* {
-            return reinterpret_cast<float*>(stage0_ptr + (size_t)s * STAGE_BYTES + row_off(16 * w2) +
+            const int blk = float_idx / (8 * D);         // 0: the warp's K rows, 1 (items of 16 heads): its V rows
+            float_idx -= blk * 8 * D;
+            return reinterpret_cast<float*>(stage0_ptr + (size_t)s * STAGE_BYTES + (size_t)blk * TILE_BYTES + row_off(16 * w2) +
                                             (uint32_t)(float_idx >> 9) * half_stride) + (float_idx & 511);
         };
         // Waits for the next filled stage; returns its ring position, or -1 when there is no more work (or the
@@ -471,8 +478,8 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
             par ^= 1;
             hb = cur.y % p.head_blocks;
             const int g = cur.y / p.head_blocks;
-            nheads = (MODE == MODE_GQA) ? min(8, p.G - hb * 8) : 1;
-            h0 = (MODE == MODE_GQA) ? g * p.G + hb * 8 : g;      // first query head of this item
+            nheads = GQA ? min(HPI, p.G - hb * HPI) : 1;
+            h0 = GQA ? g * p.G + hb * HPI : g;                // first query head of this item
         };
 
         if constexpr (MODE == MODE_PROBE) {
@@ -624,8 +631,9 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
             }
         } else {
             // ----------------------- GQA (tensor cores) -----------------------
-            uint32_t qb[KSTEPS][2];      // q^T as the B operand of S^T = K q^T
-            float m_run[2] = {NEG_INF, NEG_INF}, l_run[2] = {0.f, 0.f}, oacc[KSTEPS][4];
+            // NB blocks of 8 query heads share every K and V fragment loaded from the tile.
+            uint32_t qb[NB][KSTEPS][2];  // q^T as the B operand of S^T = K q^T
+            float m_run[NB][2], l_run[NB][2], oacc[NB][KSTEPS][4];
             // ldmatrix row addresses for this lane
             const int a_row = row0 + (lane & 7) + ((lane >> 3) & 1) * 8;   // K: matrices (rows, rows+8) x (k lo, k hi)
             const int a_kc = lane >> 4;
@@ -640,16 +648,30 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 if (d.y == 0) {
                     begin_item(s);
                     // b0 = q[head quad][16 ks + 2 tq + {0,1}], b1 = the same + 8; heads past the group read as zero
-                    const bool live = hb * 8 + quad < p.G;
-                    const uint32_t qs = stage0 + s * STAGE_BYTES + 2 * TILE_BYTES + quad * (D * 2);
 #pragma unroll
-                    for (int ks = 0; ks < KSTEPS; ++ks) {
-                        qb[ks][0] = live ? lds32(qs + (ks * 8 + tq) * 4) : 0u;
-                        qb[ks][1] = live ? lds32(qs + (ks * 8 + 4 + tq) * 4) : 0u;
+                    for (int nb = 0; nb < NB; ++nb) {
+                        const bool live = hb * HPI + nb * 8 + quad < p.G;
+                        if constexpr (NB == 1) {
+                            const uint32_t qs = stage0 + s * STAGE_BYTES + 2 * TILE_BYTES + quad * (D * 2);
+#pragma unroll
+                            for (int ks = 0; ks < KSTEPS; ++ks) {
+                                qb[nb][ks][0] = live ? lds32(qs + (ks * 8 + tq) * 4) : 0u;
+                                qb[nb][ks][1] = live ? lds32(qs + (ks * 8 + 4 + tq) * 4) : 0u;
+                            }
+                        } else {
+                            // 16 heads do not fit the stage's q slot: each lane reads its 2 x KSTEPS words from global memory
+                            const uint32_t* qg = reinterpret_cast<const uint32_t*>(
+                                reinterpret_cast<const uint16_t*>(p.q) + ((size_t)cur.b * p.Hq + (live ? h0 + nb * 8 + quad : 0)) * D);
+#pragma unroll
+                            for (int ks = 0; ks < KSTEPS; ++ks) {
+                                qb[nb][ks][0] = live ? __ldg(qg + ks * 8 + tq) : 0u;
+                                qb[nb][ks][1] = live ? __ldg(qg + ks * 8 + 4 + tq) : 0u;
+                            }
+                        }
+                        m_run[nb][0] = m_run[nb][1] = NEG_INF; l_run[nb][0] = l_run[nb][1] = 0.f;
+#pragma unroll
+                        for (int u = 0; u < KSTEPS; ++u) { oacc[nb][u][0] = oacc[nb][u][1] = oacc[nb][u][2] = oacc[nb][u][3] = 0.f; }
                     }
-                    m_run[0] = m_run[1] = NEG_INF; l_run[0] = l_run[1] = 0.f;
-#pragma unroll
-                    for (int u = 0; u < KSTEPS; ++u) { oacc[u][0] = oacc[u][1] = oacc[u][2] = oacc[u][3] = 0.f; }
                 }
                 const int tokbase = (cur.tile0 + d.y) * TILE_T;
                 const int tA = tokbase + row0 + quad, tB = tA + 8;
@@ -657,45 +679,53 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 const bool edge = tokbase < cur.lo || tokbase + TILE_T > cur.hi;
                 const uint32_t kbase = stage0 + s * STAGE_BYTES, vbase = kbase + TILE_BYTES;
 
-                // ---- S^T (16 tokens x 8 heads) ----
-                float sc[4] = {0.f, 0.f, 0.f, 0.f};
+                // ---- S^T (16 tokens x 8 heads per block) ----
+                float sc[NB][4];
+#pragma unroll
+                for (int nb = 0; nb < NB; ++nb) sc[nb][0] = sc[nb][1] = sc[nb][2] = sc[nb][3] = 0.f;
 #pragma unroll
                 for (int ks = 0; ks < KSTEPS; ++ks) {
                     const int ch = 2 * ks + a_kc;   // 16-byte chunk index along d
                     uint32_t a[4];
                     ldmatrix_x4(a, kbase + a_off + (ch >> 3) * half_stride + (((ch & 7) ^ (a_row & 7)) << 4));
-                    mma_16816<BF16>(sc, a, qb[ks][0], qb[ks][1]);
-                }
-                // sc[0], sc[1]: token tA, heads 2tq, 2tq+1; sc[2], sc[3]: token tB
-                float s2[4];
-                s2[0] = vA ? sc[0] * p.scale_log2 : NEG_INF; s2[1] = vA ? sc[1] * p.scale_log2 : NEG_INF;
-                s2[2] = vB ? sc[2] * p.scale_log2 : NEG_INF; s2[3] = vB ? sc[3] * p.scale_log2 : NEG_INF;
-                float mx[2] = {fmaxf(s2[0], s2[2]), fmaxf(s2[1], s2[3])};
 #pragma unroll
-                for (int o = 4; o <= 16; o <<= 1) {
-                    mx[0] = fmaxf(mx[0], __shfl_xor_sync(0xffffffffu, mx[0], o));
-                    mx[1] = fmaxf(mx[1], __shfl_xor_sync(0xffffffffu, mx[1], o));
+                    for (int nb = 0; nb < NB; ++nb) mma_16816<BF16>(sc[nb], a, qb[nb][ks][0], qb[nb][ks][1]);
                 }
-                float corr[2], msafe[2];
+                float corr[NB][2];
+                uint32_t bh0[NB], bh1[NB], bl0[NB], bl1[NB];
 #pragma unroll
-                for (int hc = 0; hc < 2; ++hc) {
-                    const float m_new = fmaxf(m_run[hc], mx[hc]);
-                    msafe[hc] = (m_new == NEG_INF) ? 0.f : m_new;
-                    corr[hc] = fast_exp2(m_run[hc] - msafe[hc]);
-                    m_run[hc] = m_new;
-                }
-                float pr[4];
-                pr[0] = fast_exp2(s2[0] - msafe[0]); pr[1] = fast_exp2(s2[1] - msafe[1]);
-                pr[2] = fast_exp2(s2[2] - msafe[0]); pr[3] = fast_exp2(s2[3] - msafe[1]);
-                l_run[0] = l_run[0] * corr[0] + pr[0] + pr[2];   // per-lane sums over its own two token rows
-                l_run[1] = l_run[1] * corr[1] + pr[1] + pr[3];
+                for (int nb = 0; nb < NB; ++nb) {
+                    // sc[0], sc[1]: token tA, heads 2tq, 2tq+1 of the block; sc[2], sc[3]: token tB
+                    float s2[4];
+                    s2[0] = vA ? sc[nb][0] * p.scale_log2 : NEG_INF; s2[1] = vA ? sc[nb][1] * p.scale_log2 : NEG_INF;
+                    s2[2] = vB ? sc[nb][2] * p.scale_log2 : NEG_INF; s2[3] = vB ? sc[nb][3] * p.scale_log2 : NEG_INF;
+                    float mx[2] = {fmaxf(s2[0], s2[2]), fmaxf(s2[1], s2[3])};
+#pragma unroll
+                    for (int o = 4; o <= 16; o <<= 1) {
+                        mx[0] = fmaxf(mx[0], __shfl_xor_sync(0xffffffffu, mx[0], o));
+                        mx[1] = fmaxf(mx[1], __shfl_xor_sync(0xffffffffu, mx[1], o));
+                    }
+                    float msafe[2];
+#pragma unroll
+                    for (int hc = 0; hc < 2; ++hc) {
+                        const float m_new = fmaxf(m_run[nb][hc], mx[hc]);
+                        msafe[hc] = (m_new == NEG_INF) ? 0.f : m_new;
+                        corr[nb][hc] = fast_exp2(m_run[nb][hc] - msafe[hc]);
+                        m_run[nb][hc] = m_new;
+                    }
+                    float pr[4];
+                    pr[0] = fast_exp2(s2[0] - msafe[0]); pr[1] = fast_exp2(s2[1] - msafe[1]);
+                    pr[2] = fast_exp2(s2[2] - msafe[0]); pr[3] = fast_exp2(s2[3] - msafe[1]);
+                    l_run[nb][0] = l_run[nb][0] * corr[nb][0] + pr[0] + pr[2];   // per-lane sums over its own two token rows
+                    l_run[nb][1] = l_run[nb][1] * corr[nb][1] + pr[1] + pr[3];
 
-                // P^T as the B operand of O^T += V^T P^T, as hi + lo 16-bit terms
-                const uint32_t hiA = pack2<BF16>(pr[0], pr[1]), hiB = pack2<BF16>(pr[2], pr[3]);
-                const float2 fA = unpack2<BF16>(hiA), fB = unpack2<BF16>(hiB);
-                const uint32_t loA = pack2<BF16>(pr[0] - fA.x, pr[1] - fA.y), loB = pack2<BF16>(pr[2] - fB.x, pr[3] - fB.y);
-                const uint32_t bh0 = movmatrix_trans(hiA), bh1 = movmatrix_trans(hiB);
-                const uint32_t bl0 = movmatrix_trans(loA), bl1 = movmatrix_trans(loB);
+                    // P^T as the B operand of O^T += V^T P^T, as hi + lo 16-bit terms
+                    const uint32_t hiA = pack2<BF16>(pr[0], pr[1]), hiB = pack2<BF16>(pr[2], pr[3]);
+                    const float2 fA = unpack2<BF16>(hiA), fB = unpack2<BF16>(hiB);
+                    const uint32_t loA = pack2<BF16>(pr[0] - fA.x, pr[1] - fA.y), loB = pack2<BF16>(pr[2] - fB.x, pr[3] - fB.y);
+                    bh0[nb] = movmatrix_trans(hiA); bh1[nb] = movmatrix_trans(hiB);
+                    bl0[nb] = movmatrix_trans(loA); bl1[nb] = movmatrix_trans(loB);
+                }
 
                 // ---- O^T ----
                 if (edge) {
@@ -709,50 +739,59 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 }
 #pragma unroll
                 for (int mt = 0; mt < KSTEPS; ++mt) {
-                    oacc[mt][0] *= corr[0]; oacc[mt][1] *= corr[1]; oacc[mt][2] *= corr[0]; oacc[mt][3] *= corr[1];
                     const int ch = 2 * mt + v_dc;
                     uint32_t a[4];
                     ldmatrix_x4_trans(a, vbase + v_off + (ch >> 3) * half_stride + (((ch & 7) ^ (v_row & 7)) << 4));
-                    mma_16816<BF16>(oacc[mt], a, bh0, bh1);
-                    mma_16816<BF16>(oacc[mt], a, bl0, bl1);
+#pragma unroll
+                    for (int nb = 0; nb < NB; ++nb) {
+                        oacc[nb][mt][0] *= corr[nb][0]; oacc[nb][mt][1] *= corr[nb][1];
+                        oacc[nb][mt][2] *= corr[nb][0]; oacc[nb][mt][3] *= corr[nb][1];
+                        mma_16816<BF16>(oacc[nb][mt], a, bh0[nb], bh1[nb]);
+                        mma_16816<BF16>(oacc[nb][mt], a, bl0[nb], bl1[nb]);
+                    }
                 }
                 if (d.y + 1 < cur.ntiles) { release(s, edge); continue; }
 
                 // ---- item epilogue: merge the 4 warp states (the item's last stage is the scratch) ----
 #pragma unroll
-                for (int o = 4; o <= 16; o <<= 1) {
-                    l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], o);
-                    l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], o);
-                }
-                if (quad == 0) {
-                    ctl.red_m[par][warp * 8 + 2 * tq] = m_run[0]; ctl.red_m[par][warp * 8 + 2 * tq + 1] = m_run[1];
-                    ctl.red_l[par][warp * 8 + 2 * tq] = l_run[0]; ctl.red_l[par][warp * 8 + 2 * tq + 1] = l_run[1];
-                }
-                {   // this warp's [8 heads][D] into its own rows; heads 2tq and 2tq+1 sit in the same 2 KB part
-                    float* const lane_base = warp_scratch(s, warp, (2 * tq) * D + quad);
+                for (int nb = 0; nb < NB; ++nb) {
+#pragma unroll
+                    for (int o = 4; o <= 16; o <<= 1) {
+                        l_run[nb][0] += __shfl_xor_sync(0xffffffffu, l_run[nb][0], o);
+                        l_run[nb][1] += __shfl_xor_sync(0xffffffffu, l_run[nb][1], o);
+                    }
+                    if (quad == 0) {
+                        const int e = warp * HPI + nb * 8 + 2 * tq;
+                        ctl.red_m[par][e] = m_run[nb][0]; ctl.red_m[par][e + 1] = m_run[nb][1];
+                        ctl.red_l[par][e] = l_run[nb][0]; ctl.red_l[par][e + 1] = l_run[nb][1];
+                    }
+                    // this warp's [8 heads][D] of the block into its own rows; heads 2tq and 2tq+1 sit in the same 2 KB part
+                    float* const lane_base = warp_scratch(s, warp, (nb * 8 + 2 * tq) * D + quad);
 #pragma unroll
                     for (int mt = 0; mt < KSTEPS; ++mt) {
-                        lane_base[mt * 16] = oacc[mt][0];
-                        lane_base[D + mt * 16] = oacc[mt][1];
-                        lane_base[mt * 16 + 8] = oacc[mt][2];
-                        lane_base[D + mt * 16 + 8] = oacc[mt][3];
+                        lane_base[mt * 16] = oacc[nb][mt][0];
+                        lane_base[D + mt * 16] = oacc[nb][mt][1];
+                        lane_base[mt * 16 + 8] = oacc[nb][mt][2];
+                        lane_base[D + mt * 16 + 8] = oacc[nb][mt][3];
                     }
                 }
                 if (!consumer_sync()) break;
-                {   // thread -> (head, D/16 consecutive components): the four warp states of one head, weighted
+                // thread -> (head, D/16 consecutive components): the four warp states of one head, weighted
+#pragma unroll
+                for (int nb = 0; nb < NB; ++nb) {
                     constexpr int PER = D / 16;
-                    const int hh = tid >> 4, dbase = (tid & 15) * PER;
+                    const int hh = nb * 8 + (tid >> 4), dbase = (tid & 15) * PER;
                     if (hh < nheads) {
                         float mw[CONSUMER_WARPS], M = NEG_INF, lsum = 0.f;
 #pragma unroll
-                        for (int w2 = 0; w2 < CONSUMER_WARPS; ++w2) { mw[w2] = ctl.red_m[par][w2 * 8 + hh]; M = fmaxf(M, mw[w2]); }
+                        for (int w2 = 0; w2 < CONSUMER_WARPS; ++w2) { mw[w2] = ctl.red_m[par][w2 * HPI + hh]; M = fmaxf(M, mw[w2]); }
                         float accv[PER];
 #pragma unroll
                         for (int v = 0; v < PER; ++v) accv[v] = 0.f;
 #pragma unroll
                         for (int w2 = 0; w2 < CONSUMER_WARPS; ++w2) {
                             const float w = fast_exp2(mw[w2] - M);                 // M is finite: the item has tokens
-                            lsum = fmaf(w, ctl.red_l[par][w2 * 8 + hh], lsum);
+                            lsum = fmaf(w, ctl.red_l[par][w2 * HPI + hh], lsum);
                             const float4* src = reinterpret_cast<const float4*>(warp_scratch(s, w2, hh * D + dbase));
 #pragma unroll
                             for (int v4 = 0; v4 < PER / 4; ++v4) {

@@ -564,3 +564,17 @@ def test_many_short_rows_take_the_warp_per_row_merge(D, G, monkeypatch):
     check_output(prob.out, prob.lse, ref.out, ref.lse, "cta per row")
     assert (prob.out - out_rows).abs().max().item() <= 1e-5 * max(1.0, out_rows.abs().max().item())
     assert torch.equal(torch.isinf(prob.lse), torch.isinf(lse_rows))
+
+
+@pytest.mark.parametrize("G", [9, 12, 16, 24])
+def test_groups_of_more_than_8_heads_either_way(G, monkeypatch):
+    """Groups above 8 query heads run as items of 16 heads (two MMA head blocks sharing every tile read); the
+    older form - one item per block of 8 - stays selectable.  Both match the oracle and each other."""
+    w = wl(B=2, Hq=G, Hkv=1, D=128, dtype="bf16", seq_lens=[900, 300], tok_begin=[70, 0], tok_end=[900, 217],
+           chunk_tokens=256, seed=300 + G, outlier_frac=0.01)
+    prob, ref, _ = run_and_check(w)
+    a_out, a_o = prob.out.clone(), prob.o_part.clone()
+    monkeypatch.setenv("HG_ATTN_GQA16", "0")
+    prob2, _, _ = run_and_check(w)
+    assert (prob2.out - a_out).abs().max().item() <= 1e-5 * max(1.0, a_out.abs().max().item())
+    assert (prob2.o_part - a_o).abs().max().item() <= 1e-4 * max(1.0, a_o.abs().max().item())
