@@ -1,6 +1,6 @@
 // Split-KV decode attention partials over a paged 16-bit KV pool (sm_100a).
 //
-// A work item is (sequence b, KV head g [, block of 8 query heads], chunk c).  Persistent CTAs take
+// A work item is (sequence b, KV head g [, block of 8 or 16 query heads], chunk c).  Persistent CTAs take
 // items from the list of non-empty items, dynamically through a global counter when the caller
 // provides one, else round-robin; the producer warp is the only scheduler, and every filled stage
 // carries a descriptor telling the consumers what it holds.  Within a CTA the producer streams, per
@@ -16,6 +16,9 @@
 //               tensor-core MMAs (tokens are the M dimension, heads the N dimension, nothing padded
 //               for a group of 8).  P is fed as hi + lo 16-bit terms, so its rounding error is ~2^-17
 //               (bf16) / ~2^-22 (fp16) instead of one 16-bit ulp.
+//   MODE_GQA2   groups of more than 8 query heads: items of 16 heads, i.e. two such head blocks that share
+//               every K and V fragment read from the tile (their query rows come straight from global memory,
+//               the second block's epilogue state parks in the warp's V rows).
 //   MODE_PROBE  same loads, no attention math: folds the slice's bytes into a checksum.
 //
 // With p.persistent == 0 the grid is (NC, Hkv * head_blocks, B) and every CTA handles the one item
