@@ -578,3 +578,38 @@ def test_groups_of_more_than_8_heads_either_way(G, monkeypatch):
     prob2, _, _ = run_and_check(w)
     assert (prob2.out - a_out).abs().max().item() <= 1e-5 * max(1.0, a_out.abs().max().item())
     assert (prob2.o_part - a_o).abs().max().item() <= 1e-4 * max(1.0, a_o.abs().max().item())
+
+
+@pytest.mark.parametrize("G", [1, 4, 16])
+def test_explicit_scale_overrides_the_default(G):
+    from oracle import hg_oracle as O
+    w = wl(Hq=2 * G, Hkv=2, seed=500 + G)
+    scale = 0.043
+    prob = DeviceProblem(w, DEV)
+    prob.desc = prob.make_desc(w.chunk_tokens, prob.NC, scale=scale)
+    prob.step([])
+    torch.cuda.synchronize()
+    q, K, V = bits(w.q()), bits(w.kv_logical("k")), bits(w.kv_logical("v"))
+    rm, rl, ro = O.chunked_partials(q, K, V, w.dtype, w.tok_begin, w.tok_end, w.chunk_tokens, prob.NC, scale=scale)
+    check_partials(prob.o_part.reshape(-1, w.D), prob.m_part.reshape(-1), prob.l_part.reshape(-1),
+                   rm.reshape(-1), rl.reshape(-1), ro.reshape(-1, w.D), "scale")
+    ref_out, ref_lse = O.full_batch(q, K, V, w.dtype, w.tok_begin, w.tok_end, scale=scale)
+    check_output(prob.out, prob.lse, ref_out, ref_lse, "scale")
+    # and it is not the default
+    d_out, _ = O.full_batch(q, K, V, w.dtype, w.tok_begin, w.tok_end)
+    assert np.abs(d_out - ref_out).max() > 1e-2
+
+
+@pytest.mark.parametrize("G", [1, 4])
+def test_ranges_reaching_outside_the_sequence_are_clipped(G):
+    """tok_begin below 0 and tok_end above seq_len mean "from the start" and "to the end": rows past seq_len are never
+    attended even when the caller's range covers them."""
+    w = wl(Hq=2 * G, Hkv=2, seq_lens=[700, 333], tok_begin=[130, 0], tok_end=[700, 333], seed=61)
+    ref = OracleRef(w)
+    prob = DeviceProblem(w, DEV, poison_tail=True)
+    prob.tok_begin = torch.tensor([130, -7], dtype=torch.int32, device=DEV)
+    prob.tok_end = torch.tensor([700 + 500, 333 + 1], dtype=torch.int32, device=DEV)
+    prob.step(ref.host_partials_device(DEV))
+    torch.cuda.synchronize()
+    assert int(prob.status.item()) == hg.HG_DEV_OK
+    check_output(prob.out, prob.lse, ref.out, ref.lse, "clipped")
