@@ -41,7 +41,8 @@ constexpr int THREADS = CONSUMER_THREADS + 32;
 constexpr int MAX_STAGES = 8;
 constexpr int MAX_CHUNK_PAGES = 512;       // chunk_tokens / page_size, any schedule
 constexpr int PERSIST_CHUNK_PAGES = 256;   // ... for the persistent schedule (page ids are double-buffered)
-constexpr int PERSIST_MAX_BATCH = 1536;    // sequences the in-kernel item scan handles
+constexpr int PERSIST_MAX_BATCH = 1024;    // sequences the in-kernel item scan handles (its table is 4 bytes each; two CTAs
+                                           // of three 34 KB stages leave an SM about 2 KB of shared memory to spare)
 
 enum { MODE_MHA = 0, MODE_GQA = 1, MODE_PROBE = 2, MODE_GQA2 = 3 };   // GQA2: items of 16 query heads (two MMA head blocks)
 

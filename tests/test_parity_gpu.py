@@ -327,9 +327,9 @@ def test_without_a_work_counter_items_are_dealt_round_robin():
 
 # ---- shapes beyond what the persistent schedule keeps in shared memory fall back to one CTA per item ------------
 
-@pytest.mark.parametrize("B", [530, 1536, 1540])
+@pytest.mark.parametrize("B", [530, 1024, 1030])
 def test_large_batches(B):
-    # up to 1536 sequences the in-kernel item scan (every thread several sequences) feeds the persistent schedule;
+    # up to 1024 sequences the in-kernel item scan (every thread several sequences) feeds the persistent schedule;
     # beyond that the same kernel runs with one CTA per item
     lens = [40 + (7 * i) % 150 for i in range(B)]
     tb = [(3 * i) % 30 for i in range(B)]
