@@ -21,6 +21,7 @@ from .binding import (  # noqa: F401
     prepare_merge,
     prepare_partial,
     hg_attn_decode_static,
+    hg_attn_suggest_chunk,
     hg_attn_workspace_bytes,
     hg_status_string,
     hg_kv_read_probe,

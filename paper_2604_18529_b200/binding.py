@@ -235,6 +235,17 @@ def hg_attn_merge(partials, out, lse, desc: HgAttnDesc, stream=None) -> None:
     _check(st, "hg_attn_merge")
 
 
+def hg_attn_suggest_chunk(total_tokens: int, num_q_heads: int, num_kv_heads: int, page_size: int) -> int:
+    """A chunk size (tokens) for a problem with that many GPU-resident token positions in total."""
+    f = lib().hg_attn_suggest_chunk
+    f.argtypes = [C.c_int64, C.c_int32, C.c_int32, C.c_int32]
+    f.restype = C.c_int32
+    n = int(f(total_tokens, num_q_heads, num_kv_heads, page_size))
+    if n == 0:
+        raise HgError(HG_ERR_INVALID_ARG, "hg_attn_suggest_chunk")
+    return n
+
+
 def hg_attn_workspace_bytes(desc: HgAttnDesc, n_host_partials: int = 0) -> int:
     n = int(lib().hg_attn_workspace_bytes(C.byref(desc), n_host_partials))
     if n == 0:

@@ -382,6 +382,22 @@ hg_status hg_attn_partial_from_logits(const float* logits, const void* v_rows, c
     return bf16 ? launch(logits_partial_kernel<64, true>) : launch(logits_partial_kernel<64, false>);
 }
 
+int32_t hg_attn_suggest_chunk(int64_t total_tokens, int32_t num_q_heads, int32_t num_kv_heads, int32_t page_size) {
+    if (total_tokens < 0 || num_kv_heads < 1 || num_q_heads < 1 || num_q_heads % num_kv_heads) return 0;
+    const int shift = ilog2_exact(page_size);
+    if (shift < 4 || shift > 8) return 0;
+    const int G = num_q_heads / num_kv_heads;
+    const int64_t rows = (int64_t)num_kv_heads * (G <= 8 ? 1 : (G + 15) / 16);     // items per chunk of one sequence
+    const int64_t target_items = 2000;            // about seven per resident CTA of a 148-SM device
+    const int unit = page_size > TILE_T ? page_size : TILE_T;
+    int64_t chunk = total_tokens * rows / target_items;
+    chunk = (chunk + unit - 1) / unit * unit;
+    const int64_t lo = 128 > unit ? 128 : unit, hi = 2048;
+    if (chunk < lo) chunk = lo;
+    if (chunk > hi) chunk = hi;
+    return (int32_t)chunk;
+}
+
 size_t hg_attn_workspace_bytes(const hg_attn_desc* desc, int32_t n_host_partials) {
     if (check_desc(desc, true) != HG_OK || n_host_partials < 0) return 0;
     return plan_workspace(desc, n_host_partials, HG_MAX_MERGE_SRC).total;
