@@ -613,3 +613,29 @@ def test_ranges_reaching_outside_the_sequence_are_clipped(G):
     torch.cuda.synchronize()
     assert int(prob.status.item()) == hg.HG_DEV_OK
     check_output(prob.out, prob.lse, ref.out, ref.lse, "clipped")
+
+
+def test_two_streams_with_their_own_workspaces_do_not_disturb_each_other():
+    """Two decode loops on two streams, each with its own workspace (and so its own work counter), interleaved
+    launch by launch: every result is the one the loop gets alone.  (No launch waits for another.)"""
+    ws_list, probs, wants, outs = [], [], [], []
+    for i, G in enumerate((1, 4)):
+        w = wl(Hq=8 * G, Hkv=8, seq_lens=[3000, 1777], tok_begin=[100, 0], tok_end=[3000, 1700], chunk_tokens=64, seed=700 + i)
+        assert sum(w.chunk_grid(b)[1] for b in range(w.B)) * w.Hkv > 296      # more items than resident CTAs: the counter is in use
+        prob = DeviceProblem(w, DEV)
+        prob.step([])
+        torch.cuda.synchronize()
+        probs.append(prob)
+        wants.append((prob.out.clone(), prob.lse.clone()))
+        ws_list.append(torch.empty(pkg.hg_attn_workspace_bytes(prob.desc, 0), dtype=torch.uint8, device=DEV))
+        outs.append((torch.empty_like(prob.out), torch.empty_like(prob.lse)))
+    streams = [torch.cuda.Stream(device=DEV) for _ in probs]
+    torch.cuda.synchronize()
+    for _ in range(10):
+        for prob, ws, (out, lse), st in zip(probs, ws_list, outs, streams):
+            pkg.hg_attn_decode(prob.q, prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end, [], out, lse,
+                               ws, prob.desc, stream=st)
+    torch.cuda.synchronize()
+    for prob, (out, lse), (want_out, want_lse) in zip(probs, outs, wants):
+        assert int(prob.status.item()) == hg.HG_DEV_OK
+        assert torch.equal(out, want_out) and torch.equal(lse, want_lse)
