@@ -130,7 +130,7 @@ template <int D, bool BF16, int MODE>
 static hg_status launch_partial_t(const CUtensorMap& tk, const CUtensorMap& tv, PartialParams p, cudaStream_t st,
                                   bool counter_is_zero) {
     static LaunchCache cache;                     // zero-initialised
-    const size_t smem = (size_t)p.stages * (2 * TILE_T * D * 2 + 8 * D * 2) + 1024;     // per stage: K tile, V tile, q rows
+    const size_t smem = (size_t)p.stages * ((128 / D) * 2 * TILE_T * D * 2 + 8 * D * 2) + 1024;   // per stage: 128 / D x (K tile, V tile), q rows
     auto kern = partial_kernel<D, BF16, MODE>;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return HG_ERR_CUDA; }
@@ -204,7 +204,7 @@ static hg_status run_partial(int mode, const void* q, const void* k, const void*
     p.head_blocks = (mode == MODE_GQA) ? (G + 7) / 8 : (mode == MODE_GQA2 ? (G + 15) / 16 : 1);
     const float scale = d->scale > 0.f ? d->scale : 1.0f / sqrtf((float)d->head_dim);
     p.scale_log2 = scale * 1.4426950408889634f;
-    p.stages = env_int("HG_ATTN_STAGES", d->head_dim == 128 ? 3 : 6, 2, MAX_STAGES);   // 96 KB of ring: 2 CTAs per SM
+    p.stages = env_int("HG_ATTN_STAGES", 3, 2, MAX_STAGES);   // 3 x 32 KB of K and V (plus q rows): 2 CTAs per SM
     // persistent schedule unless the batch or the chunk's page list exceeds what the kernel keeps in shared memory
     p.persistent = (d->batch <= PERSIST_MAX_BATCH && d->chunk_tokens / d->page_size <= PERSIST_CHUNK_PAGES)
                        ? env_int("HG_ATTN_PERSISTENT", 1, 0, 1) : 0;

@@ -4,7 +4,7 @@
 // items from the list of non-empty items, dynamically through a global counter when the caller
 // provides one, else round-robin; the producer warp is the only scheduler, and every filled stage
 // carries a descriptor telling the consumers what it holds.  Within a CTA the producer streams, per
-// 64-token step, the K tile and the V tile of the item (64 x D each) from HBM into one stage of a
+// step of 64 tokens (128 at D = 64: two tile pairs), the K tile and the V tile of the item (64 x D each) from HBM into one stage of a
 // shared-memory ring with TMA tensor loads - one 5-D box per (page, tensor), 128-byte swizzled - and
 // runs ahead across item boundaries, so the ring never drains between items.  Four consumer warps
 // each own 16 token rows of every tile and keep a private online-softmax state (running max,
@@ -144,7 +144,9 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
     constexpr int HALVES = D / 64;
     constexpr int TILE_BYTES = TILE_T * D * 2;
     constexpr int Q_BYTES = 8 * D * 2;            // the item's query rows (up to 8 heads), present in an item's first stage
-    constexpr int STAGE_BYTES = 2 * TILE_BYTES + Q_BYTES;   // K tile, V tile, q
+    constexpr int SUB = 128 / D;                  // 64-token tiles per stage: a stage is 32 KB of K and V at either head dim,
+    constexpr int PAIR_BYTES = 2 * TILE_BYTES;    // so the per-stage hand-shakes cost the same per byte (K tile, V tile)
+    constexpr int STAGE_BYTES = SUB * PAIR_BYTES + Q_BYTES;   // SUB x (K tile, V tile), q
     constexpr int NV = 8 * HALVES;     // MHA: d-components owned by a lane
     constexpr int KSTEPS = D / 16;     // GQA: 16-wide steps along d
     constexpr float LN2 = 0.6931471805599453f;
@@ -275,7 +277,8 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
         const uint64_t policy = l2_evict_first_policy();
         const int nbox = TILE_T >> rshift;           // boxes per tile: 4, 2 or 1
         const int j = lane & (nbox - 1);             // this lane's box
-        const int isv = lane >> (6 - rshift);        // 0: K tile, 1: V tile (lanes >= 2 * nbox idle)
+        const int isv = (lane >> (6 - rshift)) & 1;  // 0: K tile, 1: V tile
+        const int sub = lane >> (7 - rshift);        // which of the stage's tiles (lanes with sub >= SUB idle)
         constexpr int PER_LANE = PERSIST_CHUNK_PAGES / 32;
         const bool dynamic = p.persistent && p.sched != nullptr;
 
@@ -350,14 +353,14 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
             const int g = cur.y / p.head_blocks;
             const int q_heads = GQA ? min(HPI, p.G - (cur.y % p.head_blocks) * HPI) : 1;
             const int q_head0 = GQA ? g * p.G + (cur.y % p.head_blocks) * HPI : g;
-            for (int it = 0; it < cur.ntiles; ++it) {              // one stage = K tile + V tile of 64 tokens
+            for (int it = 0; it < cur.ntiles; it += SUB) {         // one stage = SUB x (K tile + V tile of 64 tokens)
                 int okw = 1;
                 if (lane == 0) okw = mbar_wait(&ctl.empty[s], ph ^ 1u, abort_flag) ? 1 : 0;
                 okw = __shfl_sync(0xffffffffu, okw, 0);
                 if (!okw) { alive = false; break; }
-                const int t0j = (cur.tile0 + it) * TILE_T + j * R;
+                const int t0j = (cur.tile0 + it + sub) * TILE_T + j * R;
                 int phys = -1;
-                if (isv < 2 && t0j < cur.hi && t0j + R > cur.lo) phys = pages[(t0j >> p.page_shift) - page0];
+                if (sub < SUB && it + sub < cur.ntiles && t0j < cur.hi && t0j + R > cur.lo) phys = pages[(t0j >> p.page_shift) - page0];
                 const uint32_t nvalid = __popc(__ballot_sync(0xffffffffu, phys >= 0));   // K and V boxes
                 // (items of 16 heads fetch their query rows themselves: the stage's q slot holds 8)
                 const uint32_t qbytes = (MODE != MODE_PROBE && NB == 1 && it == 0) ? (uint32_t)q_heads * D * 2u : 0u;
@@ -368,10 +371,10 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 }
                 __syncwarp();
                 if (qbytes && lane == 31)        // the item's query rows travel with its first stage
-                    bulk_load(stage0_ptr + (size_t)s * STAGE_BYTES + 2 * TILE_BYTES,
+                    bulk_load(stage0_ptr + (size_t)s * STAGE_BYTES + SUB * PAIR_BYTES,
                               reinterpret_cast<const uint16_t*>(p.q) + ((size_t)cur.b * p.Hq + q_head0) * D, qbytes, &ctl.full[s]);
                 if (phys >= 0) {
-                    uint8_t* dst = stage0_ptr + (size_t)s * STAGE_BYTES + isv * TILE_BYTES + j * box_bytes;
+                    uint8_t* dst = stage0_ptr + (size_t)s * STAGE_BYTES + sub * PAIR_BYTES + isv * TILE_BYTES + j * box_bytes;
                     tma_load_5d(dst, isv ? &tmV : &tmK, &ctl.full[s], 0, t0j & (p.page_size - 1), 0, g, phys, policy);
                 }
                 ++issued;
@@ -493,8 +496,9 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 const int s = next_stage(d);
                 if (s < 0) break;
                 if (d.y == 0) { begin_item(s); probe_x = 0u; }
-                const uint32_t base = stage0 + s * STAGE_BYTES;
-                const int tokbase = (cur.tile0 + d.y) * TILE_T;
+                for (int sub = 0; sub < SUB && d.y + sub < cur.ntiles; ++sub) {
+                const uint32_t base = stage0 + s * STAGE_BYTES + sub * PAIR_BYTES;
+                const int tokbase = (cur.tile0 + d.y + sub) * TILE_T;
 #pragma unroll
                 for (int u = 0; u < 8 * HALVES; ++u) {
                     // K and V: 16 rows x HALVES x 8 chunks each per warp; a quarter-warp reads one 128-byte row segment
@@ -506,7 +510,8 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                         probe_x ^= v.x ^ v.y ^ v.z ^ v.w;
                     }
                 }
-                if (d.y + 1 < cur.ntiles) { release(s, false); continue; }
+                }
+                if (d.y + SUB < cur.ntiles) { release(s, false); continue; }
                 // item epilogue, with the item's last stage as scratch
 #pragma unroll
                 for (int o = 16; o; o >>= 1) probe_x ^= __shfl_xor_sync(0xffffffffu, probe_x, o);
@@ -532,7 +537,7 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 if (s < 0) break;
                 if (d.y == 0) {
                     begin_item(s);
-                    const uint32_t qs = stage0 + s * STAGE_BYTES + 2 * TILE_BYTES;
+                    const uint32_t qs = stage0 + s * STAGE_BYTES + SUB * PAIR_BYTES;
 #pragma unroll
                     for (int hh = 0; hh < HALVES; ++hh) {
                         uint4 raw = lds128(qs + hh * 128 + li * 16);
@@ -545,11 +550,12 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
 #pragma unroll
                     for (int u = 0; u < NV; ++u) o[u] = 0.f;
                 }
-                const int tokbase = (cur.tile0 + d.y) * TILE_T;
+                for (int sub = 0; sub < SUB && d.y + sub < cur.ntiles; ++sub) {
+                const int tokbase = (cur.tile0 + d.y + sub) * TILE_T;
                 bool valid[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) { const int t = tokbase + rbase + k; valid[k] = t >= cur.lo && t < cur.hi; }
-                const uint32_t kbase = stage0 + s * STAGE_BYTES, vbase = kbase + TILE_BYTES;
+                const uint32_t kbase = stage0 + s * STAGE_BYTES + sub * PAIR_BYTES, vbase = kbase + TILE_BYTES;
 
                 // ---- K tile: 4 logits per lane group ----
                 float acc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -604,7 +610,8 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                         oo[6] = fmaf(pk[k], dd.x, oo[6]); oo[7] = fmaf(pk[k], dd.y, oo[7]);
                     }
                 }
-                if (d.y + 1 < cur.ntiles) { release(s, false); continue; }
+                }
+                if (d.y + SUB < cur.ntiles) { release(s, false); continue; }
 
                 // ---- item epilogue: merge the 16 row-group states (parked in the item's last stage) ----
                 const int slot = warp * 4 + gi;
@@ -656,7 +663,7 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                     for (int nb = 0; nb < NB; ++nb) {
                         const bool live = hb * HPI + nb * 8 + quad < p.G;
                         if constexpr (NB == 1) {
-                            const uint32_t qs = stage0 + s * STAGE_BYTES + 2 * TILE_BYTES + quad * (D * 2);
+                            const uint32_t qs = stage0 + s * STAGE_BYTES + SUB * PAIR_BYTES + quad * (D * 2);
 #pragma unroll
                             for (int ks = 0; ks < KSTEPS; ++ks) {
                                 qb[nb][ks][0] = live ? lds32(qs + (ks * 8 + tq) * 4) : 0u;
@@ -677,11 +684,14 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                         for (int u = 0; u < KSTEPS; ++u) { oacc[nb][u][0] = oacc[nb][u][1] = oacc[nb][u][2] = oacc[nb][u][3] = 0.f; }
                     }
                 }
-                const int tokbase = (cur.tile0 + d.y) * TILE_T;
+                bool wrote = false;
+                for (int sub = 0; sub < SUB && d.y + sub < cur.ntiles; ++sub) {
+                const int tokbase = (cur.tile0 + d.y + sub) * TILE_T;
                 const int tA = tokbase + row0 + quad, tB = tA + 8;
                 const bool vA = tA >= cur.lo && tA < cur.hi, vB = tB >= cur.lo && tB < cur.hi;
                 const bool edge = tokbase < cur.lo || tokbase + TILE_T > cur.hi;
-                const uint32_t kbase = stage0 + s * STAGE_BYTES, vbase = kbase + TILE_BYTES;
+                wrote |= edge;
+                const uint32_t kbase = stage0 + s * STAGE_BYTES + sub * PAIR_BYTES, vbase = kbase + TILE_BYTES;
 
                 // ---- S^T (16 tokens x 8 heads per block) ----
                 float sc[NB][4];
@@ -754,7 +764,8 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                         mma_16816<BF16>(oacc[nb][mt], a, bl0[nb], bl1[nb]);
                     }
                 }
-                if (d.y + 1 < cur.ntiles) { release(s, edge); continue; }
+                }
+                if (d.y + SUB < cur.ntiles) { release(s, wrote); continue; }
 
                 // ---- item epilogue: merge the 4 warp states (the item's last stage is the scratch) ----
 #pragma unroll
