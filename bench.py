@@ -29,8 +29,8 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the partial kernel, from the ncu
 # captures summarised under profiles/ (None until a capture of that workload exists)
 NCU_TRAFFIC_BYTES = {
-    # profiles/partial_kernel_opt13b.md: two sequences captured (805.54 MB read + 4.74 MB written), x 4
-    "opt13b": 4 * (805_537_024 + 4_742_400),
+    # profiles/partial_kernel_opt13b.md: two sequences captured (805.55 MB read + 5.01 MB written), x 4
+    "opt13b": 4 * (805_546_496 + 5_009_664),
     # profiles/partial_kernel_llama70b.md: the full launch captured
     "llama70b": 1_718_226_000 + 7_822_080,
     # profiles/partial_kernel_opt30b.md: one of the four sequences captured (1879.14 MB read + 3.87 MB written), x 4
