@@ -59,6 +59,13 @@ typedef enum hg_dtype { HG_DTYPE_F16 = 0, HG_DTYPE_BF16 = 1 } hg_dtype;
                                  stage, so every wait runs into its time limit (about 2 s); the call then
                                  reports HG_DEV_WAIT_TIMEOUT through *status and returns normally */
 
+#define HG_FLAG_SPARSE_EMPTY 2u /* empty chunk slots get m = -inf and l = 0 only; their o rows are left as they
+                                   are (hg_attn_merge never reads the o of an empty partial).  For batches that
+                                   mix long and short sequences: num_chunks is set by the longest one, and
+                                   zero-filling every short sequence's unused slots can cost more than the
+                                   attention itself.  hg_attn_decode and its variants always work this way on
+                                   their own workspace. */
+
 /* values the kernels may write to *hg_attn_desc.status (device word, optional) */
 #define HG_DEV_OK 0
 #define HG_DEV_WAIT_TIMEOUT 1 /* a bounded on-chip barrier wait ran out; the call's results are invalid.

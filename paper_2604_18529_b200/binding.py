@@ -22,6 +22,7 @@ HG_DTYPE_F16, HG_DTYPE_BF16 = 0, 1
 HG_DEV_OK, HG_DEV_WAIT_TIMEOUT, HG_DEV_BAD_PAGE = 0, 1, 2
 HG_MAX_MERGE_SRC = 8
 HG_FLAG_TEST_STALL = 1
+HG_FLAG_SPARSE_EMPTY = 2
 HG_STATIC_SCRATCH_BYTES = 8 << 20
 
 

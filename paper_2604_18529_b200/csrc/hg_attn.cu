@@ -209,6 +209,7 @@ static hg_status run_partial(int mode, const void* q, const void* k, const void*
     p.persistent = (d->batch <= PERSIST_MAX_BATCH && d->chunk_tokens / d->page_size <= PERSIST_CHUNK_PAGES)
                        ? env_int("HG_ATTN_PERSISTENT", 1, 0, 1) : 0;
     p.test_stall = (d->flags & HG_FLAG_TEST_STALL) ? 1 : 0;
+    p.sparse_empty = (d->flags & HG_FLAG_SPARSE_EMPTY) ? 1 : 0;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     p.sched = p.persistent && env_int("HG_ATTN_DYNAMIC", 1, 0, 1) ? desc_sched(d) : nullptr;
     const bool bf16 = d->dtype == HG_DTYPE_BF16;
@@ -262,8 +263,8 @@ static hg_status run_merge(const hg_partial_src* src, int32_t n_src, float* out,
     cfg.numAttrs = na;
     auto launch = [&](auto k128, auto k64) { return d->head_dim == 128 ? cudaLaunchKernelEx(&cfg, k128, p) : cudaLaunchKernelEx(&cfg, k64, p); };
     cudaError_t e;
-    // many short rows: a warp per row, eight rows per CTA
-    if (rows >= 2048 && p.total <= 64 && env_int("HG_ATTN_MERGE_ROWS", 1, 0, 1)) {
+    // many rows: a warp per row, eight rows per CTA
+    if (rows >= 2048 && env_int("HG_ATTN_MERGE_ROWS", 1, 0, 1)) {
         cfg.gridDim = dim3((unsigned)((rows + 7) / 8));
         cfg.blockDim = dim3(256);
         e = d->head_dim == 128 ? cudaLaunchKernelEx(&cfg, merge_rows_kernel<128>, p, rows)
@@ -422,6 +423,7 @@ static hg_status decode_impl(const void* q, const void* k_cache, const void* v_c
     memcpy(&dd, desc, desc->struct_size < sizeof dd ? desc->struct_size : sizeof dd);
     dd.struct_size = sizeof dd;
     dd.sched_counter = reinterpret_cast<int32_t*>(ws + w.sched);       // the workspace provides the work counter
+    dd.flags |= HG_FLAG_SPARSE_EMPTY;                                  // the chunk partials are private to this call and its merge
     st = run_partial(MODE_MHA, q, k_cache, v_cache, seq_lens, tok_begin, tok_end, o_part, m_part, l_part, nullptr, stream, &dd,
                      counter_is_zero);
     if (st != HG_OK) return st;

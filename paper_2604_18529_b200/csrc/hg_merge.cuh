@@ -144,9 +144,10 @@ __global__ void __launch_bounds__(THREADS_) merge_kernel(const MergeParams p) {
     }
 }
 
-// Many short rows (a large batch, few chunks each): one WARP per (sequence, query head), eight rows per CTA.
-// The warp sweeps its row's partials in order, four loads in flight, with the same running-maximum rule as
-// above; no shared memory, no barrier.
+// Many rows (a large batch): one WARP per (sequence, query head), eight rows per CTA.  The warp reads 32 slot
+// maxima at a time, one per lane, and visits only the slots that hold something, in order, four loads in flight -
+// so the many empty slots that short sequences have next to a long one cost almost nothing.  Same
+// running-maximum rule as above; no shared memory, no barrier.
 template <int D>
 __global__ void __launch_bounds__(256) merge_rows_kernel(const MergeParams p, int rows) {
     constexpr int VEC = D / 32;
@@ -166,39 +167,44 @@ __global__ void __launch_bounds__(256) merge_rows_kernel(const MergeParams p, in
         const float* ms = p.m[s] + (size_t)row * nc;
         const float* ls = p.l[s] + (size_t)row * nc;
         const float* os = p.o[s] + (size_t)row * nc * D;
-        for (int i0 = 0; i0 < nc; i0 += 4) {
-            float mi[4], li[4], ov[4][VEC];
+        for (int i0 = 0; i0 < nc; i0 += 32) {
+            const float mine = i0 + lane < nc ? ms[i0 + lane] : NEG_INF;
+            uint32_t live = __ballot_sync(0xffffffffu, mine != NEG_INF);
+            while (live) {
+                float mi[4], li[4], ov[4][VEC];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int i = i0 + u;
-                const bool in = i < nc;
-                mi[u] = in ? ms[i] : NEG_INF;
-                li[u] = in ? ls[i] : 0.f;
-                const bool live = in && mi[u] != NEG_INF;
-                const float* orow = os + (size_t)(in ? i : 0) * D + lane * VEC;
-                if constexpr (VEC == 4) {
-                    const float4 v = live ? *reinterpret_cast<const float4*>(orow) : make_float4(0.f, 0.f, 0.f, 0.f);
-                    ov[u][0] = v.x; ov[u][1] = v.y; ov[u][2] = v.z; ov[u][3] = v.w;
-                } else {
-                    const float2 v = live ? *reinterpret_cast<const float2*>(orow) : make_float2(0.f, 0.f);
-                    ov[u][0] = v.x; ov[u][1] = v.y;
+                for (int u = 0; u < 4; ++u) {                  // the next four live slots (warp-uniform)
+                    const bool in = live != 0u;
+                    const int src = in ? __ffs(live) - 1 : 0;
+                    if (in) live &= live - 1u;
+                    mi[u] = __shfl_sync(0xffffffffu, mine, src);
+                    if (!in) mi[u] = NEG_INF;
+                    const int i = i0 + src;
+                    li[u] = in ? ls[i] : 0.f;
+                    const float* orow = os + (size_t)i * D + lane * VEC;
+                    if constexpr (VEC == 4) {
+                        const float4 v = in ? *reinterpret_cast<const float4*>(orow) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        ov[u][0] = v.x; ov[u][1] = v.y; ov[u][2] = v.z; ov[u][3] = v.w;
+                    } else {
+                        const float2 v = in ? *reinterpret_cast<const float2*>(orow) : make_float2(0.f, 0.f);
+                        ov[u][0] = v.x; ov[u][1] = v.y;
+                    }
                 }
-            }
-            const float m4 = fmaxf(fmaxf(mi[0], mi[1]), fmaxf(mi[2], mi[3]));
-            if (m4 == NEG_INF) continue;
-            if (m4 > M) {
-                const float r = __expf(M - m4);
-                lsum *= r;
+                const float m4 = fmaxf(fmaxf(mi[0], mi[1]), fmaxf(mi[2], mi[3]));
+                if (m4 > M) {
+                    const float r = __expf(M - m4);            // 0 while M is still -inf
+                    lsum *= r;
 #pragma unroll
-                for (int v = 0; v < VEC; ++v) acc[v] *= r;
-                M = m4;
-            }
+                    for (int v = 0; v < VEC; ++v) acc[v] *= r;
+                    M = m4;
+                }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const float w = mi[u] == NEG_INF ? 0.f : __expf(mi[u] - M);
-                lsum = fmaf(w, li[u], lsum);
+                for (int u = 0; u < 4; ++u) {
+                    const float w = mi[u] == NEG_INF ? 0.f : __expf(mi[u] - M);
+                    lsum = fmaf(w, li[u], lsum);
 #pragma unroll
-                for (int v = 0; v < VEC; ++v) acc[v] = fmaf(w, ov[u][v], acc[v]);
+                    for (int v = 0; v < VEC; ++v) acc[v] = fmaf(w, ov[u][v], acc[v]);
+                }
             }
         }
     }

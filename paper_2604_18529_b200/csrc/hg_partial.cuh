@@ -62,6 +62,7 @@ struct PartialParams {
     int C, NC, stages, head_blocks;
     int persistent;
     int test_stall;           // HG_FLAG_TEST_STALL: the producer never fills a stage
+    int sparse_empty;         // HG_FLAG_SPARSE_EMPTY: empty chunk slots get m and l only, their o rows stay untouched
     int32_t* sched;           // zeroed work counter: items are handed out dynamically (NULL: round-robin)
     float scale_log2;         // logit scale * log2(e)
 };
@@ -248,8 +249,9 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 const int hb = it.y % p.head_blocks, g = it.y / p.head_blocks;
                 const int nh = GQA ? min(HPI, p.G - hb * HPI) : 1;
                 const int hq0 = GQA ? g * p.G + hb * HPI : g;
-                for (int i = tid; i < nh * D; i += THREADS)
-                    p.o_part[(((size_t)it.b * p.Hq + hq0 + i / D) * p.NC + it.c) * D + i % D] = 0.f;
+                if (!p.sparse_empty)
+                    for (int i = tid; i < nh * D; i += THREADS)
+                        p.o_part[(((size_t)it.b * p.Hq + hq0 + i / D) * p.NC + it.c) * D + i % D] = 0.f;
                 if (tid < nh) {
                     p.m_part[((size_t)it.b * p.Hq + hq0 + tid) * p.NC + it.c] = NEG_INF;
                     p.l_part[((size_t)it.b * p.Hq + hq0 + tid) * p.NC + it.c] = 0.f;
@@ -428,10 +430,11 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                     const int hb = y % p.head_blocks, g = y / p.head_blocks;
                     const int nh = GQA ? min(HPI, p.G - hb * HPI) : 1;
                     const int hq0 = GQA ? g * p.G + hb * HPI : g;
-                    for (int i = tid; i < nh * ne * D; i += CONSUMER_THREADS) {
-                        const int e = i / D, hh = e / ne, cc = nc + e % ne;
-                        p.o_part[(((size_t)b * p.Hq + hq0 + hh) * p.NC + cc) * D + i % D] = 0.f;
-                    }
+                    if (!p.sparse_empty)
+                        for (int i = tid; i < nh * ne * D; i += CONSUMER_THREADS) {
+                            const int e = i / D, hh = e / ne, cc = nc + e % ne;
+                            p.o_part[(((size_t)b * p.Hq + hq0 + hh) * p.NC + cc) * D + i % D] = 0.f;
+                        }
                     for (int i = tid; i < nh * ne; i += CONSUMER_THREADS) {
                         const int hh = i / ne, cc = nc + i % ne;
                         p.m_part[((size_t)b * p.Hq + hq0 + hh) * p.NC + cc] = NEG_INF;

@@ -639,3 +639,32 @@ def test_two_streams_with_their_own_workspaces_do_not_disturb_each_other():
     for prob, (out, lse), (want_out, want_lse) in zip(probs, outs, wants):
         assert int(prob.status.item()) == hg.HG_DEV_OK
         assert torch.equal(out, want_out) and torch.equal(lse, want_lse)
+
+
+@pytest.mark.parametrize("G", [1, 4])
+def test_sparse_empty_slots_for_mixed_batches(G):
+    """A batch of one long and several short sequences: num_chunks follows the long one.  With HG_FLAG_SPARSE_EMPTY
+    the short sequences' unused slots get m = -inf and l = 0 and their o rows are not touched; the merge never
+    reads them.  hg_attn_decode works that way by itself."""
+    lens = [2500, 90, 130, 64, 300]
+    w = wl(B=5, Hq=2 * G, Hkv=2, seq_lens=lens, tok_begin=[0, 10, 0, 0, 37], tok_end=lens, chunk_tokens=128, seed=88)
+    ref = OracleRef(w)
+    prob = DeviceProblem(w, DEV)
+    prob.desc = prob.make_desc(w.chunk_tokens, prob.NC, flags=hg.HG_FLAG_SPARSE_EMPTY)
+    prob.o_part.fill_(float("nan")); prob.m_part.fill_(7.0); prob.l_part.fill_(7.0)
+    prob.step(ref.host_partials_device(DEV))
+    torch.cuda.synchronize()
+    check_output(prob.out, prob.lse, ref.out, ref.lse, "sparse")
+    for b in range(1, w.B):
+        n = w.chunk_grid(b)[1]
+        assert n < prob.NC
+        assert torch.isinf(prob.m_part[b, :, n:]).all() and (prob.l_part[b, :, n:] == 0).all()
+        assert torch.isnan(prob.o_part[b, :, n:]).all()                    # left alone
+        assert not torch.isnan(prob.o_part[b, :, :n]).any()
+    ws = torch.full((pkg.hg_attn_workspace_bytes(prob.desc, 2),), 0xFF, dtype=torch.uint8, device=DEV)   # NaN patterns
+    out, lse = torch.empty_like(prob.out), torch.empty_like(prob.lse)
+    plain = prob.make_desc(w.chunk_tokens, prob.NC)
+    pkg.hg_attn_decode(prob.q, prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end,
+                       ref.host_partials_device(DEV), out, lse, ws, plain)
+    torch.cuda.synchronize()
+    assert torch.equal(out, prob.out) and torch.equal(lse, prob.lse)
