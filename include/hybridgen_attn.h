@@ -115,7 +115,8 @@ typedef struct hg_attn_desc {
     int32_t* status;           /* dev, optional: receives HG_DEV_* if a kernel detects a problem */
     int32_t* sched_counter;    /* dev, optional, 4 bytes: when given, hg_attn_partial zeroes it on the stream and
                                   its CTAs draw work items from it dynamically (better balance on ragged
-                                  batches); NULL: items are dealt round-robin.  Must not be shared by calls
+                                  batches); NULL: items are dealt round-robin.  Left alone when the problem has no
+                                  more items than the device has resident CTAs.  Must not be shared by calls
                                   that may overlap on the GPU.  Present when struct_size covers it. */
 } hg_attn_desc;
 
@@ -135,7 +136,7 @@ typedef struct hg_partial_src {
  *   q          dev [B][Hq][D], dtype as desc->dtype, 16-byte aligned
  *   k_cache    dev K pool, v_cache dev V pool (addressing above)
  *   seq_lens   dev int32 [B]   cached tokens per sequence
- *   tok_begin  dev int32 [B]   0 <= tok_begin <= tok_end <= seq_len
+ *   tok_begin  dev int32 [B]   0 <= tok_begin <= tok_end <= seq_len; values outside are clipped to [0, seq_len]
  *   tok_end    dev int32 [B]
  *   o_part     dev float [B][Hq][NC][D]  out: sum_t e^{s_t - m} V_t
  *   m_part     dev float [B][Hq][NC]     out: exact fp32 chunk maximum of the scaled logits
@@ -158,6 +159,7 @@ hg_status hg_attn_partial(const void* q, const void* k_cache, const void* v_cach
  *   partials  host array of n_src sources (n_src >= 1); each source's arrays are dev memory
  *   out       dev float [B][Hq][D]   sum_i w_i o_i / sum_i w_i l_i,  w_i = e^{m_i - max_j m_j}
  *   lse       dev float [B][Hq]      max_j m_j + ln sum_i w_i l_i   (may be NULL)
+ * A partial with m = -inf is empty: it contributes nothing and its o row is never read.
  * Only batch, num_q_heads and head_dim of desc are used.  n_src <= HG_MAX_MERGE_SRC.
  */
 #define HG_MAX_MERGE_SRC 8
