@@ -161,6 +161,20 @@ static hg_status launch_partial_t(const CUtensorMap& tk, const CUtensorMap& tv, 
         cudaGetLastError();
         return HG_ERR_CUDA;
     }
+    if ((!p.sched || counter_is_zero) && env_int("HG_ATTN_PDL", 1, 0, 1)) {
+        // no memset sits between this launch and the kernel before it in the stream: launch as a programmatic
+        // dependent, so that block scheduling and the input-free part of the set-up overlap that kernel's tail
+        p.pdl_wait = 1;
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof cfg);
+        cfg.gridDim = grid; cfg.blockDim = dim3(THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, kern, tk, tv, p) != cudaSuccess) { cudaGetLastError(); return HG_ERR_CUDA; }
+        return HG_OK;
+    }
     kern<<<grid, THREADS, smem, st>>>(tk, tv, p);
     return cudaGetLastError() == cudaSuccess ? HG_OK : HG_ERR_CUDA;
 }

@@ -46,6 +46,7 @@ __global__ void __launch_bounds__(THREADS_) merge_kernel(const MergeParams p) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
 #if __CUDA_ARCH__ >= 900
+    cudaTriggerProgrammaticLaunchCompletion();  // a partial kernel launched as a dependent may set up meanwhile
     cudaGridDependencySynchronize();            // partials may come from the kernel launched just before
 #endif
 
@@ -155,6 +156,7 @@ __global__ void __launch_bounds__(256) merge_rows_kernel(const MergeParams p, in
     const int lane = threadIdx.x & 31;
     const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
 #if __CUDA_ARCH__ >= 900
+    cudaTriggerProgrammaticLaunchCompletion();  // a partial kernel launched as a dependent may set up meanwhile
     cudaGridDependencySynchronize();
 #endif
     if (row >= rows) return;

@@ -63,6 +63,7 @@ struct PartialParams {
     int persistent;
     int test_stall;           // HG_FLAG_TEST_STALL: the producer never fills a stage
     int sparse_empty;         // HG_FLAG_SPARSE_EMPTY: empty chunk slots get m and l only, their o rows stay untouched
+    int pdl_wait;             // launched as a programmatic dependent: wait for the preceding kernel before reading any input
     int32_t* sched;           // zeroed work counter: items are handed out dynamically (NULL: round-robin)
     float scale_log2;         // logit scale * log2(e)
 };
@@ -168,18 +169,11 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int Y = p.Hkv * p.head_blocks;
 
-    // Loads whose answers are needed a little later are issued first, so that their round trips overlap the
-    // set-up: the status word (a wait that timed out earlier in this call, or a word the caller left set,
-    // means: do not queue behind it), and this CTA's second work item (its first is its own block index).
-    const int32_t status_at_entry = p.status ? *reinterpret_cast<volatile int32_t*>(p.status) : HG_DEV_OK;
-    int early_request = 0;
+    // ---- set-up that touches no input: barriers, tensor-map prefetch ------------------------------------
     if (tid == CONSUMER_THREADS) {
         prefetch_tensormap(&tmK);                    // the descriptors are on their way long before the first load
         prefetch_tensormap(&tmV);
-        if (p.persistent && p.sched && !p.test_stall) early_request = (int)gridDim.x + atomicAdd(p.sched, 1);
     }
-
-    // ---- set-up: barriers, and for the persistent schedule the item counts per sequence ---------------
     if (tid == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(&ctl.full[s], 1);
@@ -189,6 +183,20 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
         ctl.abort_flag = 0;
         fence_barrier_init();
     }
+#if __CUDA_ARCH__ >= 900
+    // launched while the kernel before it in the stream was still running: everything above overlapped that
+    // kernel's tail; nothing it may have written is read before this returns
+    if (p.pdl_wait) cudaGridDependencySynchronize();
+#endif
+
+    // Loads whose answers are needed a little later are issued first, so that their round trips overlap the
+    // scan below: the status word (a wait that timed out earlier in this call, or a word the caller left set,
+    // means: do not queue behind it), and this CTA's second work item (its first is its own block index).
+    const int32_t status_at_entry = p.status ? *reinterpret_cast<volatile int32_t*>(p.status) : HG_DEV_OK;
+    int early_request = 0;
+    if (tid == CONSUMER_THREADS && p.persistent && p.sched && !p.test_stall) early_request = (int)gridDim.x + atomicAdd(p.sched, 1);
+
+    // ---- for the persistent schedule the item counts per sequence -------------------------------------------
     int n_items = 1, item_step = 1, item_first = 0;
     if (p.persistent) {
         // cum[b+1] = sum_{b' <= b} nc_b' * Y : every thread a contiguous block of sequences, warp scan, then the
