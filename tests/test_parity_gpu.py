@@ -668,3 +668,27 @@ def test_sparse_empty_slots_for_mixed_batches(G):
                        ref.host_partials_device(DEV), out, lse, ws, plain)
     torch.cuda.synchronize()
     assert torch.equal(out, prob.out) and torch.equal(lse, prob.lse)
+
+
+def test_the_readme_decode_flow():
+    """The dozen lines of the README: suggest a chunk size, describe the pool by its tensor strides, decode."""
+    G = 4
+    w = wl(Hq=2 * G, Hkv=2, seq_lens=[1900, 777], tok_begin=[300, 0], tok_end=[1900, 700], seed=404)
+    ref = OracleRef(w)
+    kv = w.build_device_kv(DEV)
+    k_pool, v_pool, block_table = kv["k"], kv["v"], kv["block_table"]
+    assert k_pool.shape == (kv["num_pages"], w.Hkv, w.page_size, w.D)
+    chunk = pkg.hg_attn_suggest_chunk(w.gpu_tokens, w.Hq, w.Hkv, w.page_size)
+    max_chunks = max(-(-e // chunk) - b // chunk for b, e in zip(w.tok_begin, w.tok_end))
+    desc = pkg.attn_desc(batch=w.B, num_q_heads=w.Hq, num_kv_heads=w.Hkv, head_dim=w.D, dtype=torch.float16,
+                         page_size=w.page_size, num_pages=k_pool.shape[0], page_stride=k_pool.stride(0),
+                         head_stride=k_pool.stride(1), tok_stride=k_pool.stride(2), block_table=block_table,
+                         max_pages=block_table.shape[1], chunk_tokens=chunk, num_chunks=max_chunks)
+    ws = torch.empty(pkg.hg_attn_workspace_bytes(desc, 2), dtype=torch.uint8, device=DEV)
+    out = torch.empty(w.B, w.Hq, w.D, device=DEV)
+    lse = torch.empty(w.B, w.Hq, device=DEV)
+    i32 = lambda x: torch.tensor(x, dtype=torch.int32, device=DEV)
+    pkg.hg_attn_decode(w.q(DEV), k_pool, v_pool, i32(w.seq_lens), i32(w.tok_begin), i32(w.tok_end),
+                       ref.host_partials_device(DEV), out, lse, ws, desc)
+    torch.cuda.synchronize()
+    check_output(out, lse, ref.out, ref.lse, "readme")
