@@ -10,7 +10,7 @@ from typing import List, Optional, Tuple
 import torch
 
 from . import binding as hg
-from .workload import AttnWorkload, torch_dtype
+from .workload import AttnWorkload
 
 
 class DeviceProblem:

@@ -1,5 +1,4 @@
 """Helpers for the GPU-vs-oracle parity tests: oracle references for a workload and error measures."""
-import math
 
 import numpy as np
 import torch

@@ -1,7 +1,6 @@
 """Host-side companions (logits calculator, selection, gather, feedback scheduler) against the oracle and the
 plain statements in oracle/hg_policy.py.  CPU only."""
 import itertools
-import math
 
 import numpy as np
 import pytest

@@ -91,7 +91,6 @@ def test_decode_loop_with_append_eviction_and_exact_hybrid_attention():
     """The cache's whole life: every step appends the new token's K/V on the GPU; when a slice outgrows its
     budget the oldest tokens move to the host store; attention is the hybrid step with K large enough to take
     every host token, so each step must equal monolithic attention over the whole sequence so far."""
-    import dataclasses
     import paper_2604_18529_b200 as pkg
     from test_kv_residency_gpu import poison_future_rows, rows_at
     G, steps, budget, evict_n = 2, 12, 200, 64

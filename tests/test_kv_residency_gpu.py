@@ -3,7 +3,6 @@ oldest tokens to the host and attending over the shrunk slice.  Data movement is
 the logical rows of the workload generator, attention against the oracle."""
 import dataclasses
 
-import numpy as np
 import pytest
 import torch
 

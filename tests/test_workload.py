@@ -2,7 +2,6 @@
 table and the logical rows describe the same cache.  CPU only."""
 import dataclasses
 
-import numpy as np
 import pytest
 import torch
 
