@@ -82,7 +82,7 @@ class HybridAttentionStep:
         self.copy_stream = torch.cuda.Stream(device=dev)
         self.ev = {n: torch.cuda.Event(enable_timing=True) for n in ("g0", "g1", "t0", "t1", "h1")}
         self.history: List[StepRecord] = []
-        self._plan_k, self._plan_pos = -1, None
+        self._plan_k, self._plan_pos, self._plan_n, self._ranking = -1, None, None, None
         self.set_host_tokens(self.n_host)
 
     def set_host_tokens(self, n_host: torch.Tensor) -> None:
@@ -92,6 +92,18 @@ class HybridAttentionStep:
         if self.n_host_max > self.capacity:
             raise ValueError("more host tokens than the host rows hold")
         self.n_rows = self.n_host.repeat_interleave(self.Hkv).contiguous()
+        self._plan_k = -1
+
+    def set_pre_qk_ranking(self, ranking: Optional[torch.Tensor]) -> None:
+        """A ranked candidate list for Pre-QK^T selection, most important first: int32 ``[B][Hkv][R]`` of host token
+        indices, -1 padded at the end (Section 4.5: any predictor - positions, accumulated scores, head
+        importance - reduces to such a list; the selector takes its first K entries).  ``None`` goes back to
+        the built-in position rule (sinks + most recent host tokens)."""
+        if ranking is not None:
+            if ranking.dtype != torch.int32 or ranking.dim() != 3 or ranking.shape[:2] != (self.B, self.Hkv):
+                raise ValueError("ranking must be int32 [B][Hkv][R]")
+            ranking = ranking.contiguous()
+        self._ranking = ranking
         self._plan_k = -1
 
     def set_operating_point(self, k: int, strategy: int) -> None:
@@ -105,13 +117,21 @@ class HybridAttentionStep:
         logits = self.p_logits[:B * Hq * k].view(B, Hq, k)
         vsel = self.p_vsel[:B * Hkv * k * D].view(B, Hkv, k, D)
         n_sel = self.p_nsel
-        if self._plan_k != k:                       # counts and the position-based set depend on k alone: kept between steps
-            torch.minimum(self.n_host, torch.tensor(k, dtype=torch.int32), out=n_sel)
+        if self._plan_k != k:                       # counts and the Pre-QK^T set depend on k alone: kept between steps
+            n_post = torch.minimum(self.n_host, torch.tensor(k, dtype=torch.int32))
+            n_pre = n_post.clone()
             pos = torch.full((B, Hkv, k), -1, dtype=torch.int32)
-            for b in range(B):
-                sel = H.hg_host_select_positions(int(self.n_host[b]), self.sinks, max(k - self.sinks, 0), k)
-                pos[b, :, : len(sel)] = sel
-            self._plan_k, self._plan_pos = k, pos
+            if self._ranking is not None:
+                # the first K candidates of the caller's list; a sequence offers as many as every one of its heads has
+                take = self._ranking[:, :, :k]
+                pos[:, :, : take.shape[2]] = take
+                n_pre = torch.minimum(n_pre, (take >= 0).sum(dim=2).min(dim=1).values.to(torch.int32))
+            else:
+                for b in range(B):
+                    sel = H.hg_host_select_positions(int(self.n_host[b]), self.sinks, max(k - self.sinks, 0), k)
+                    pos[b, :, : len(sel)] = sel
+            self._plan_k, self._plan_pos, self._plan_n = k, pos, (n_post, n_pre)
+        n_sel.copy_(self._plan_n[0 if self.strategy == POST_QK and self.n_host_max > 0 else 1])
         sel_desc = H.host_desc(self.k_host, Hq, k, scale=self.desc.scale, threads=self.threads)
         if self.strategy == POST_QK and self.n_host_max > 0:
             n_max = self.n_host_max

@@ -134,3 +134,35 @@ def test_decode_loop_with_append_eviction_and_exact_hybrid_attention():
             assert np.linalg.norm(out - ref_out) / np.linalg.norm(ref_out) <= OUT_REL_L2, s
             assert np.abs(lse - ref_lse).max() <= LSE_ABS, s
     assert evictions >= 3 and tb[0] > tb[1] >= 0
+
+
+def test_pre_qk_selection_from_a_callers_ranking():
+    """The token selector takes any ranked candidate list (Section 4.5): here a list built from an earlier
+    Post-QK^T step's choice, padded with -1 where a head has fewer candidates."""
+    G = 2
+    w = W.AttnWorkload("rank", 2, 2 * G, 2, 128, "f16", [1200, 500], [800, 300], [1200, 500], page_size=16,
+                       chunk_tokens=128, seed=77)
+    q_t, K_t, V_t = w.q(), w.kv_logical("k"), w.kv_logical("v")
+    prob = DeviceProblem(w, DEV)
+    eng = hybrid.HybridAttentionStep(prob.desc, K_t, V_t, torch.tensor(w.tok_begin, dtype=torch.int32), k_min=48, k_max=48,
+                                     k_step=16, handoff_chunk=32, device=DEV)
+    q, K, V = bits(q_t), bits(K_t), bits(V_t)
+    args = (prob.q, q_t, prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end, prob.out, prob.lse)
+    with torch.cuda.device(DEV):
+        eng.step(*args)                                            # Post-QK^T: the 48 best per KV head
+        ranking = torch.full((w.B, w.Hkv, 64), -1, dtype=torch.int32)
+        ranking[:, :, :48] = eng.idx.flip(2)                       # some order; what matters is which 48 come first
+        ranking[1, 1, 40:] = -1                                    # one head of sequence 1 offers only 40
+        eng.set_pre_qk_ranking(ranking)
+        eng.set_operating_point(48, hybrid.PRE_QK)
+        eng.step(*args)
+    assert eng.n_sel.tolist() == [48, 40]
+    assert torch.equal(eng.idx[0], ranking[0, :, :48]) and torch.equal(eng.idx[1, :, :40], ranking[1, :, :40])
+    ref_out, ref_lse = reference(w, q, K, V, eng.idx, eng.n_sel, G)
+    out, lse = prob.out.double().cpu().numpy(), prob.lse.double().cpu().numpy()
+    assert np.abs(out - ref_out).max() <= OUT_MAX_ABS and np.abs(lse - ref_lse).max() <= LSE_ABS
+    with torch.cuda.device(DEV):
+        eng.set_pre_qk_ranking(None)                               # back to sinks + recent window
+        eng.set_operating_point(48, hybrid.PRE_QK)
+        eng.step(*args)
+    assert eng.idx[0, 0, :4].tolist() == [0, 1, 2, 3] and eng.n_sel.tolist() == [48, 48]
