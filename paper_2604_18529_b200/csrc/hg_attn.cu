@@ -12,6 +12,7 @@
 #include <string.h>
 
 #include <atomic>
+#include <type_traits>
 
 #include "hg_kvcache.cuh"
 #include "hg_logits.cuh"
@@ -382,7 +383,9 @@ hg_status hg_attn_partial_from_logits(const float* logits, const void* v_rows, c
     p.logits = logits; p.v_rows = v_rows; p.n_sel = n_sel; p.o_part = o_part; p.m_part = m_part; p.l_part = l_part;
     p.B = d->batch; p.Hq = d->num_q_heads; p.Hkv = d->num_kv_heads; p.G = p.Hq / p.Hkv; p.K = d->max_selected;
     p.chunk = d->chunk_tokens; p.NC = d->num_chunks;
-    const size_t smem = ((size_t)8 * p.chunk + (size_t)LG_WARPS * 8 * d->head_dim) * sizeof(float);
+    // heads per pass over the V rows: the smallest of 1, 2, 4, 8 that covers the group (8 for larger groups)
+    const int nh = p.G >= 8 ? 8 : (p.G > 2 ? 4 : p.G);
+    const size_t smem = ((size_t)nh * p.chunk + (size_t)LG_WARPS * nh * d->head_dim) * sizeof(float);
     dim3 grid((unsigned)p.NC, (unsigned)p.Hkv, (unsigned)p.B);
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     const bool bf16 = d->dtype == HG_DTYPE_BF16;
@@ -394,8 +397,19 @@ hg_status hg_attn_partial_from_logits(const float* logits, const void* v_rows, c
         kern<<<grid, LG_THREADS, smem, cs>>>(p);
         return cudaGetLastError() == cudaSuccess ? HG_OK : HG_ERR_CUDA;
     };
-    if (d->head_dim == 128) return bf16 ? launch(logits_partial_kernel<128, true>) : launch(logits_partial_kernel<128, false>);
-    return bf16 ? launch(logits_partial_kernel<64, true>) : launch(logits_partial_kernel<64, false>);
+    auto pick = [&](auto dtag, auto btag) -> hg_status {
+        constexpr int DD = decltype(dtag)::value;
+        constexpr bool BB = decltype(btag)::value;
+        switch (nh) {
+            case 1: return launch(logits_partial_kernel<DD, BB, 1>);
+            case 2: return launch(logits_partial_kernel<DD, BB, 2>);
+            case 4: return launch(logits_partial_kernel<DD, BB, 4>);
+            default: return launch(logits_partial_kernel<DD, BB, 8>);
+        }
+    };
+    if (d->head_dim == 128)
+        return bf16 ? pick(std::integral_constant<int, 128>{}, std::true_type{}) : pick(std::integral_constant<int, 128>{}, std::false_type{});
+    return bf16 ? pick(std::integral_constant<int, 64>{}, std::true_type{}) : pick(std::integral_constant<int, 64>{}, std::false_type{});
 }
 
 int32_t hg_attn_suggest_chunk(int64_t total_tokens, int32_t num_q_heads, int32_t num_kv_heads, int32_t page_size) {

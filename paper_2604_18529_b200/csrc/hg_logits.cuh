@@ -4,7 +4,7 @@
 // them into the same (m, l, o) partial that hg_attn_partial produces for GPU-resident tokens, so the
 // merge kernel treats both sides alike.  q.K^T is skipped; only V is streamed.
 //
-// Grid (chunk, KV head, sequence), 256 threads.  Per block of up to 8 query heads of the group: the
+// Grid (chunk, KV head, sequence), 256 threads.  Per block of up to NH (1, 2, 4 or 8) query heads of the group: the
 // chunk's logits go to shared memory, warp h finds head h's maximum and turns its logits into
 // p = e^{s - m} in place (and their sum l); then the 8 warps stride over the chunk's tokens, each lane
 // owning D/32 components of every head's o, reading each V row once for all heads; a fixed-order
@@ -29,13 +29,14 @@ struct LogitsParams {
     int B, Hq, Hkv, G, K, chunk, NC;
 };
 
-template <int D, bool BF16>
+// NH: query heads handled per pass over the chunk's V rows (1, 2, 4 or 8; a group of G heads takes ceil(G / NH) passes)
+template <int D, bool BF16, int NH>
 __global__ void __launch_bounds__(LG_THREADS) logits_partial_kernel(const LogitsParams p) {
     constexpr int VEC = D / 32;                       // components per lane
     extern __shared__ float lg_smem[];
-    float* const s_p = lg_smem;                       // [8 heads][chunk]  logits, then p
-    float* const s_red = lg_smem + 8 * p.chunk;       // [8 warps][8 heads][D]
-    __shared__ float s_m[8], s_l[8];
+    float* const s_p = lg_smem;                       // [NH heads][chunk]  logits, then p
+    float* const s_red = lg_smem + NH * p.chunk;      // [8 warps][NH heads][D]
+    __shared__ float s_m[NH], s_l[NH];
     const float NEG_INF = __int_as_float(0xff800000);
 
     const int c = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
@@ -45,8 +46,8 @@ __global__ void __launch_bounds__(LG_THREADS) logits_partial_kernel(const Logits
     const int nt = max(t1 - t0, 0);
     const uint16_t* vbase = reinterpret_cast<const uint16_t*>(p.v_rows) + ((size_t)b * p.Hkv + g) * (size_t)p.K * D;
 
-    for (int hb = 0; hb * 8 < p.G; ++hb) {
-        const int h0 = g * p.G + hb * 8, nh = min(8, p.G - hb * 8);
+    for (int hb = 0; hb * NH < p.G; ++hb) {
+        const int h0 = g * p.G + hb * NH, nh = min(NH, p.G - hb * NH);
         // ---- logits of this head block into shared memory -------------------------------------------
         for (int i = tid; i < nh * nt; i += LG_THREADS) {
             const int hh = i / nt, t = i - hh * nt;
@@ -72,9 +73,9 @@ __global__ void __launch_bounds__(LG_THREADS) logits_partial_kernel(const Logits
         }
         __syncthreads();
         // ---- o[h][d] = sum_t p[h][t] V[t][d]: each V row read once for all heads of the block -----------
-        float acc[8][VEC];
+        float acc[NH][VEC];
 #pragma unroll
-        for (int hh = 0; hh < 8; ++hh)
+        for (int hh = 0; hh < NH; ++hh)
 #pragma unroll
             for (int v = 0; v < VEC; ++v) acc[hh][v] = 0.f;
         constexpr int UNROLL = 8;                                  // V rows in flight per warp
@@ -102,8 +103,8 @@ __global__ void __launch_bounds__(LG_THREADS) logits_partial_kernel(const Logits
                     vv[2] = bb.x; vv[3] = bb.y;
                 }
 #pragma unroll
-                for (int hh = 0; hh < 8; ++hh) {
-                    if (hh < nh) {
+                for (int hh = 0; hh < NH; ++hh) {
+                    if (NH == 1 || hh < nh) {
                         const float pv = s_p[hh * p.chunk + t];       // broadcast read
                         if (pv != 0.f) {                              // unselected slots (and their V rows) never enter the sum
 #pragma unroll
@@ -114,10 +115,10 @@ __global__ void __launch_bounds__(LG_THREADS) logits_partial_kernel(const Logits
             }
         }
 #pragma unroll
-        for (int hh = 0; hh < 8; ++hh) {
-            if (hh < nh) {
+        for (int hh = 0; hh < NH; ++hh) {
+            if (NH == 1 || hh < nh) {
 #pragma unroll
-                for (int v = 0; v < VEC; ++v) s_red[((size_t)warp * 8 + hh) * D + lane * VEC + v] = acc[hh][v];
+                for (int v = 0; v < VEC; ++v) s_red[((size_t)warp * NH + hh) * D + lane * VEC + v] = acc[hh][v];
             }
         }
         __syncthreads();
@@ -125,7 +126,7 @@ __global__ void __launch_bounds__(LG_THREADS) logits_partial_kernel(const Logits
             const int hh = i / D, d = i - hh * D;
             float o = 0.f;
 #pragma unroll
-            for (int w = 0; w < LG_WARPS; ++w) o += s_red[((size_t)w * 8 + hh) * D + d];
+            for (int w = 0; w < LG_WARPS; ++w) o += s_red[((size_t)w * NH + hh) * D + d];
             const size_t slot = ((size_t)b * p.Hq + h0 + hh) * p.NC + c;
             p.o_part[slot * D + d] = o;
             if (d == 0) { p.m_part[slot] = s_m[hh]; p.l_part[slot] = s_l[hh]; }
