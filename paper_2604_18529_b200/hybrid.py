@@ -40,6 +40,8 @@ class HybridAttentionStep:
 
     ``desc`` describes the GPU slice (as for ``hg_attn_partial``); ``k_host`` / ``v_host`` are the host-held
     rows ``[B][T][Hkv][D]`` (any strides, D contiguous) of which the first ``n_host[b]`` are valid.
+    For batches that mix long and short sequences build ``desc`` with ``flags=HG_FLAG_SPARSE_EMPTY``: the
+    chunk partials here are private to the step, so their empty slots need no zero-filled ``o`` rows.
     """
 
     def __init__(self, desc: hg.HgAttnDesc, k_host: torch.Tensor, v_host: torch.Tensor, n_host: torch.Tensor,
