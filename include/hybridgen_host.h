@@ -12,6 +12,8 @@
  *                             last `window` tokens
  *   hg_host_gather_rows       gathers the selected tokens' V rows into a staging buffer for the transfer
  *   hg_sched_init / _update   the Feedback Scheduler policy (Algorithm 1)
+ *   hg_host_tier_*            host memory bound to one NUMA node, the mechanism under the semantic-aware
+ *                             placement of Section 4.4 (K rows in CPU DRAM, V rows in a far tier)
  */
 #ifndef HYBRIDGEN_HOST_H_
 #define HYBRIDGEN_HOST_H_
@@ -91,6 +93,26 @@ int32_t hg_host_select_positions(int32_t n_tokens, int32_t sinks, int32_t window
  */
 hg_status hg_host_gather_rows(const void* rows, const int32_t* idx, const int32_t* n_sel, void* dst,
                               const hg_host_desc* desc);
+
+/*
+ * Tiered host memory (Section 4.4).  The paper keeps the K rows, which the CPU reads, in CPU DRAM and the
+ * V rows, which only ever travel to the GPU, in a slower and larger tier (CXL-attached memory appears to
+ * Linux as a NUMA node without CPUs), by binding allocations to nodes.  These calls are that mechanism:
+ * page-aligned anonymous memory whose pages may live on `node` only.
+ *
+ *   hg_host_tier_alloc    bytes > 0, node >= 0.  HG_ERR_INVALID_ARG for a node the machine does not have,
+ *                         HG_ERR_UNSUPPORTED where the kernel refuses the binding, HG_OK and *out otherwise.
+ *                         The memory is zero-filled on first touch; register it with the CUDA runtime to
+ *                         make transfers from it asynchronous.
+ *   hg_host_tier_free     ptr and bytes as allocated.
+ *   hg_host_tier_node_of  the node on which the page holding ptr lives now; -1 when it has not been touched
+ *                         yet or cannot be told.
+ *   hg_host_tier_nodes    number of NUMA nodes with memory that are on line (at least 1).
+ */
+hg_status hg_host_tier_alloc(size_t bytes, int32_t node, void** out);
+void hg_host_tier_free(void* ptr, size_t bytes);
+int32_t hg_host_tier_node_of(const void* ptr);
+int32_t hg_host_tier_nodes(void);
 
 /* Feedback Scheduler (Algorithm 1). */
 typedef enum hg_sched_strategy { HG_SCHED_POST_QK = 0, HG_SCHED_PRE_QK = 1 } hg_sched_strategy;

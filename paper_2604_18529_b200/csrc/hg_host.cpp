@@ -6,6 +6,12 @@
 #include <string.h>
 
 #include <pthread.h>
+#include <stdio.h>
+#if defined(__linux__)
+#include <sys/mman.h>
+#include <sys/syscall.h>
+#include <unistd.h>
+#endif
 
 #include <algorithm>
 #include <atomic>
@@ -445,6 +451,81 @@ hg_status hg_host_gather_rows(const void* rows, const int32_t* idx, const int32_
         rows_written();
     });
     return HG_OK;
+}
+
+// ---- tiered host memory ---------------------------------------------------------------------------------------
+
+int32_t hg_host_tier_nodes(void) {
+#if defined(__linux__)
+    // /sys/devices/system/node/has_memory: a list like "0" or "0-1,3"
+    FILE* f = fopen("/sys/devices/system/node/has_memory", "r");
+    if (!f) return 1;
+    int count = 0, a = 0, b = 0;
+    char sep = 0;
+    while (fscanf(f, "%d", &a) == 1) {
+        b = a;
+        if (fscanf(f, "%c", &sep) == 1 && sep == '-') { if (fscanf(f, "%d", &b) != 1) b = a; if (fscanf(f, "%c", &sep) != 1) sep = 0; }
+        count += b - a + 1;
+        if (sep != ',') break;
+    }
+    fclose(f);
+    return count > 0 ? count : 1;
+#else
+    return 1;
+#endif
+}
+
+static bool node_has_memory(int node) {
+#if defined(__linux__)
+    char path[64];
+    snprintf(path, sizeof path, "/sys/devices/system/node/node%d/meminfo", node);
+    FILE* f = fopen(path, "r");
+    if (!f) return false;
+    fclose(f);
+    return true;
+#else
+    return node == 0;
+#endif
+}
+
+hg_status hg_host_tier_alloc(size_t bytes, int32_t node, void** out) {
+    if (!out || bytes == 0 || node < 0 || node >= 1024) return HG_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!node_has_memory(node)) return HG_ERR_INVALID_ARG;
+#if defined(__linux__)
+    void* p = mmap(nullptr, bytes, PROT_READ | PROT_WRITE, MAP_PRIVATE | MAP_ANONYMOUS, -1, 0);
+    if (p == MAP_FAILED) return HG_ERR_UNSUPPORTED;
+    unsigned long mask[16] = {0};                      // 1024 nodes
+    mask[node / (8 * sizeof(unsigned long))] |= 1ul << (node % (8 * sizeof(unsigned long)));
+    const long mpol_bind = 2;                          // MPOL_BIND: pages of this range come from the nodes in the mask only
+    if (syscall(SYS_mbind, p, bytes, mpol_bind, mask, (unsigned long)(sizeof mask * 8), 0u) != 0) {
+        munmap(p, bytes);
+        return HG_ERR_UNSUPPORTED;
+    }
+    *out = p;
+    return HG_OK;
+#else
+    return HG_ERR_UNSUPPORTED;
+#endif
+}
+
+void hg_host_tier_free(void* ptr, size_t bytes) {
+#if defined(__linux__)
+    if (ptr && bytes) munmap(ptr, bytes);
+#endif
+}
+
+int32_t hg_host_tier_node_of(const void* ptr) {
+#if defined(__linux__)
+    if (!ptr) return -1;
+    void* page = reinterpret_cast<void*>(reinterpret_cast<uintptr_t>(ptr) & ~(uintptr_t)4095);
+    int status = -1;
+    // move_pages with no target nodes only reports where each page is
+    if (syscall(SYS_move_pages, 0, 1ul, &page, nullptr, &status, 0) != 0) return -1;
+    return status >= 0 ? status : -1;
+#else
+    return -1;
+#endif
 }
 
 void hg_sched_init(hg_sched_state* st, int32_t k_min) {

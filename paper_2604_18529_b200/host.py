@@ -46,6 +46,14 @@ def _lib():
         L.hg_host_select_positions.restype = C.c_int32
         L.hg_host_gather_rows.argtypes = [vp, vp, vp, vp, C.POINTER(HgHostDesc)]
         L.hg_host_gather_rows.restype = C.c_int
+        L.hg_host_tier_alloc.argtypes = [C.c_size_t, C.c_int32, C.POINTER(vp)]
+        L.hg_host_tier_alloc.restype = C.c_int
+        L.hg_host_tier_free.argtypes = [vp, C.c_size_t]
+        L.hg_host_tier_free.restype = None
+        L.hg_host_tier_node_of.argtypes = [vp]
+        L.hg_host_tier_node_of.restype = C.c_int32
+        L.hg_host_tier_nodes.argtypes = []
+        L.hg_host_tier_nodes.restype = C.c_int32
         L.hg_sched_init.argtypes = [C.POINTER(HgSchedState), C.c_int32]
         L.hg_sched_init.restype = None
         L.hg_sched_update.argtypes = [C.POINTER(HgSchedState), C.c_double, C.c_double, C.c_double, C.c_int32, C.c_int32, C.c_int32]
@@ -129,3 +137,52 @@ class FeedbackScheduler:
     def update(self, t_gpu: float, t_cpu: float, t_tx: float):
         _lib().hg_sched_update(C.byref(self.state), t_gpu, t_cpu, t_tx, self.k_min, self.k_max, self.step)
         return self.state.k, self.state.strategy
+
+
+def hg_host_tier_nodes() -> int:
+    """NUMA nodes with memory on this machine."""
+    return int(_lib().hg_host_tier_nodes())
+
+
+class TierBuffer:
+    """A tensor whose memory is bound to one NUMA node (``hg_host_tier_alloc``), optionally registered with the
+    CUDA runtime so that copies from and to it are asynchronous DMA.  ``tensor`` views the memory; the buffer
+    must outlive every view and every copy in flight."""
+
+    def __init__(self, shape, dtype: torch.dtype, node: int, register: bool = False):
+        self.shape, self.dtype, self.node = tuple(shape), dtype, node
+        n = 1
+        for d in self.shape:
+            n *= d
+        self.nbytes = max(n * torch.empty(0, dtype=dtype).element_size(), 1)
+        ptr = C.c_void_p()
+        _check(_lib().hg_host_tier_alloc(self.nbytes, node, C.byref(ptr)), "hg_host_tier_alloc")
+        self.ptr = ptr.value
+        self._raw = (C.c_uint8 * self.nbytes).from_address(self.ptr)
+        self.tensor = torch.frombuffer(self._raw, dtype=dtype, count=n).view(self.shape)
+        self.registered = False
+        if register:
+            err = torch.cuda.cudart().cudaHostRegister(self.ptr, self.nbytes, 0)
+            if int(err) != 0:
+                self.free()
+                raise RuntimeError(f"cudaHostRegister failed: {err}")
+            self.registered = True
+
+    def node_of(self, byte_offset: int = 0) -> int:
+        return int(_lib().hg_host_tier_node_of(self.ptr + byte_offset))
+
+    def free(self) -> None:
+        if self.ptr:
+            if self.registered:
+                torch.cuda.cudart().cudaHostUnregister(self.ptr)
+                self.registered = False
+            self.tensor = None
+            self._raw = None
+            _lib().hg_host_tier_free(self.ptr, self.nbytes)
+            self.ptr = 0
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass

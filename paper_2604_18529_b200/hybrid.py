@@ -202,9 +202,22 @@ class HostKvStore:
     its oldest tokens in original order - row i is absolute token i, ``n[b]`` rows valid - i.e. the prefix
     ``[0, tok_begin[b])`` that the Eviction Engine (Section 4.2) has moved off the GPU."""
 
-    def __init__(self, batch: int, capacity: int, num_kv_heads: int, head_dim: int, dtype: torch.dtype):
-        self.k = torch.zeros(batch, capacity, num_kv_heads, head_dim, dtype=dtype).pin_memory()
-        self.v = torch.zeros(batch, capacity, num_kv_heads, head_dim, dtype=dtype).pin_memory()
+    def __init__(self, batch: int, capacity: int, num_kv_heads: int, head_dim: int, dtype: torch.dtype,
+                 k_node: Optional[int] = None, v_node: Optional[int] = None):
+        """``k_node`` / ``v_node``: NUMA nodes to bind the K rows and the V rows to (Section 4.4: keys, which the CPU
+        reads, in CPU DRAM; values, which only travel to the GPU, in the far tier); ``None`` leaves the placement
+        to the allocator.  Either way the rows are pinned."""
+        shape = (batch, capacity, num_kv_heads, head_dim)
+        self._tiers = []
+        def rows(node):
+            if node is None:
+                return torch.zeros(shape, dtype=dtype).pin_memory()
+            buf = H.TierBuffer(shape, dtype, node, register=True)
+            self._tiers.append(buf)
+            buf.tensor.zero_()
+            return buf.tensor
+        self.k = rows(k_node)
+        self.v = rows(v_node)
         self.n = torch.zeros(batch, dtype=torch.int32)
         self.capacity = capacity
 

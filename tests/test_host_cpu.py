@@ -194,3 +194,17 @@ def test_feedback_scheduler_follows_algorithm_1():
     for _ in range(20):
         s.update(1.0, 0.1, 0.1)
     assert s.state.k == 1024
+
+
+def test_tier_memory_is_bound_to_its_node():
+    assert H.hg_host_tier_nodes() >= 1
+    buf = H.TierBuffer((3, 1000, 64), torch.float16, node=0)
+    assert buf.node_of() == -1                                  # nothing touched yet: no page behind it
+    buf.tensor.fill_(1.5)
+    assert buf.node_of() == 0 and buf.node_of(buf.nbytes - 1) == 0
+    assert buf.tensor.shape == (3, 1000, 64) and float(buf.tensor.float().sum()) == 1.5 * 3 * 1000 * 64
+    buf.free()
+    with pytest.raises(H.HgError):
+        H.TierBuffer((16,), torch.float32, node=H.hg_host_tier_nodes() + 500)   # no such node
+    with pytest.raises(H.HgError):
+        H.TierBuffer((16,), torch.float32, node=-1)

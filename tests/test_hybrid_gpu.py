@@ -166,3 +166,30 @@ def test_pre_qk_selection_from_a_callers_ranking():
         eng.set_operating_point(48, hybrid.PRE_QK)
         eng.step(*args)
     assert eng.idx[0, 0, :4].tolist() == [0, 1, 2, 3] and eng.n_sel.tolist() == [48, 48]
+
+
+def test_host_store_on_bound_and_registered_tier_memory():
+    """K rows and V rows of the host tier bound to NUMA nodes (node 0 for both here: one node is all this machine
+    has) and registered with the CUDA runtime: eviction lands in them and the hybrid step reads them."""
+    import paper_2604_18529_b200 as pkg
+    G = 2
+    w = W.AttnWorkload("tier", 2, 2 * G, 2, 128, "f16", [500, 260], [0, 0], [500, 260], page_size=16, chunk_tokens=128, seed=321)
+    prob = DeviceProblem(w, DEV)
+    store = hybrid.HostKvStore(w.B, 256, w.Hkv, w.D, torch.float16, k_node=0, v_node=0)
+    with torch.cuda.device(DEV):
+        store.evict_from_gpu(prob.kv["k"], prob.kv["v"], prob.tok_begin, prob.tok_end, [200, 100], prob.desc)
+        assert prob.tok_begin.tolist() == [200, 100] == store.n.tolist()
+        for b in range(w.B):
+            for g in range(w.Hkv):
+                assert torch.equal(store.k[b, : int(store.n[b]), g], w.kv_rows("k", b, g, 0, int(store.n[b])))
+        assert store._tiers[0].node_of() == 0 and store._tiers[1].node_of() == 0
+        eng = hybrid.HybridAttentionStep(prob.desc, store.k, store.v, store.n, k_min=256, k_max=256, k_step=64, handoff_chunk=128,
+                                         device=DEV)
+        eng.step(prob.q, w.q(), prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end, prob.out, prob.lse)
+    q, K, V = bits(w.q()), bits(w.kv_logical("k")), bits(w.kv_logical("v"))
+    ref_out, ref_lse = O.full_batch(q, K, V, w.dtype, [0, 0], w.seq_lens)
+    out, lse = prob.out.double().cpu().numpy(), prob.lse.double().cpu().numpy()
+    assert np.abs(out - ref_out).max() <= OUT_MAX_ABS and np.abs(lse - ref_lse).max() <= LSE_ABS
+    del eng
+    for t in store._tiers:
+        t.free()
