@@ -242,7 +242,29 @@ def time_extras(w, prob, dev, steps):
                               "steps": [{"k": r.k, "strategy": "post_qk" if r.strategy == 0 else "pre_qk",
                                          "t_gpu_ms": round(r.t_gpu, 3), "t_cpu_ms": round(r.t_cpu, 3),
                                          "t_tx_ms": round(r.t_tx, 3), "t_step_ms": round(r.t_step, 3)} for r in recs]}
-        del eng, kh, vh
+        # the same step for 8 layers (one cache, a query per layer): layer after layer, and with the CPU stage of layer
+        # i + 1 on a host thread while the GPU handles layer i (the paper's pipelined execution)
+        L = 8
+        layers = [hybrid.HybridAttentionStep(prob.desc, kh, vh, torch.full((w.B,), n_h, dtype=torch.int32), k_min=128,
+                                             k_max=1024, k_step=128, sinks=4, device=dev) for _ in range(L)]
+        pipe = hybrid.HybridPipeline(layers)
+        qd = [prob.q] * L
+        qhs = [qh] * L
+        kvs = [(prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end)] * L
+        outs = [(torch.empty_like(prob.out), torch.empty_like(prob.lse)) for _ in range(L)]
+        times = {}
+        with torch.cuda.device(dev):
+            for mode in (False, True):
+                best = None
+                for _ in range(6):
+                    for e in layers:
+                        e.set_operating_point(128, hybrid.PRE_QK)
+                    ms = pipe.run(qd, qhs, kvs, outs, pipelined=mode)
+                    best = ms if best is None else min(best, ms)
+                times[mode] = best
+        out["hybrid_pipeline"] = {"layers": L, "k": 128, "strategy": "pre_qk", "layer_after_layer_ms": round(times[False], 3),
+                                  "pipelined_ms": round(times[True], 3)}
+        del eng, kh, vh, layers, pipe
     # ---- residency: evict 1024 oldest tokens per sequence into staging (state is restored between runs)
     max_evict = 1024
     k_out = torch.empty(w.B, max_evict, w.Hkv, w.D, dtype=dt, device=dev); v_out = torch.empty_like(k_out)

@@ -85,6 +85,7 @@ class HybridAttentionStep:
         self.ev = {n: torch.cuda.Event(enable_timing=True) for n in ("g0", "g1", "t0", "t1", "h1")}
         self.history: List[StepRecord] = []
         self._plan_k, self._plan_pos, self._plan_n, self._ranking = -1, None, None, None
+        self._pending = None
         self.set_host_tokens(self.n_host)
 
     def set_host_tokens(self, n_host: torch.Tensor) -> None:
@@ -152,22 +153,30 @@ class HybridAttentionStep:
         self.idx, self.n_sel = idx, n_sel.clone()
         return logits, vsel, n_sel
 
-    # ---- one step ---------------------------------------------------------------------------------------------
-    def step(self, q_dev, q_host, k_cache, v_cache, seq_lens, tok_begin, tok_end, out, lse) -> StepRecord:
-        B, Hq, Hkv, D = self.B, self.Hq, self.Hkv, self.D
-        k, ev = self.k, self.ev
+    # ---- one step, in the three pieces a pipeline needs -------------------------------------------------------------
+    def cpu_stage(self, q_host: torch.Tensor):
+        """Selection, logits and V-row gather for the current (K, strategy); host only, may run on another thread
+        while the GPU works on something else.  Returns what ``finish`` needs."""
+        t0 = time.perf_counter()
+        k = self.k
+        logits, vsel, n_sel = self._cpu_stage(q_host, k)
+        return k, logits, vsel, n_sel, (time.perf_counter() - t0) * 1e3
+
+    def launch_gpu(self, q_dev, k_cache, v_cache, seq_lens, tok_begin, tok_end) -> None:
+        """The GPU stage: partials of the GPU-resident tokens, enqueued on the current stream."""
         main = torch.cuda.current_stream(self.dev)
-        t_wall = time.perf_counter()
-        # GPU stage: enqueued first, runs while the host works
-        ev["g0"].record(main)
+        self.ev["g0"].record(main)
         hg.hg_attn_partial(q_dev, k_cache, v_cache, seq_lens, tok_begin, tok_end, self.o_part, self.m_part, self.l_part,
                            self.desc, main)
-        ev["g1"].record(main)
-        # CPU stage
-        t0 = time.perf_counter()
-        logits, vsel, n_sel = self._cpu_stage(q_host, k)
-        t_cpu = (time.perf_counter() - t0) * 1e3
-        # transfer and hand-off partials on the second stream
+        self.ev["g1"].record(main)
+
+    def finish(self, staged, out, lse) -> None:
+        """Transfer of the CPU stage's output, hand-off partials (second stream) and the merge (current stream);
+        everything is enqueued, nothing waited for."""
+        B, Hq, Hkv, D = self.B, self.Hq, self.Hkv, self.D
+        k, logits, vsel, n_sel, t_cpu = staged
+        ev = self.ev
+        main = torch.cuda.current_stream(self.dev)
         ld = hg.logits_desc(batch=B, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, dtype=self.dtype, max_selected=k,
                             chunk_tokens=self.chunk)
         ncs = ld.num_chunks
@@ -189,12 +198,69 @@ class HybridAttentionStep:
             ev["h1"].record(cs)
         main.wait_event(ev["h1"])
         hg.hg_attn_merge([(self.o_part, self.m_part, self.l_part), (h_o, h_m, h_l)], out, lse, self.desc, main)
-        main.synchronize()
-        rec = StepRecord(k=k, strategy=self.strategy, t_gpu=ev["g0"].elapsed_time(ev["g1"]), t_cpu=t_cpu,
-                         t_tx=ev["t0"].elapsed_time(ev["t1"]), t_step=(time.perf_counter() - t_wall) * 1e3)
+        self._pending = (k, self.strategy, t_cpu)
+
+    def collect(self, t_step_ms: float = 0.0, update: bool = True) -> StepRecord:
+        """After the stream has been synchronised: the step's record; with ``update`` Algorithm 1 moves (K, strategy)."""
+        k, strategy, t_cpu = self._pending
+        ev = self.ev
+        rec = StepRecord(k=k, strategy=strategy, t_gpu=ev["g0"].elapsed_time(ev["g1"]), t_cpu=t_cpu,
+                         t_tx=ev["t0"].elapsed_time(ev["t1"]), t_step=t_step_ms)
         self.history.append(rec)
-        self.k, self.strategy = self.sched.update(rec.t_gpu, rec.t_cpu, rec.t_tx)      # Algorithm 1, for the next step
+        if update:
+            self.k, self.strategy = self.sched.update(rec.t_gpu, rec.t_cpu, rec.t_tx)
         return rec
+
+    def step(self, q_dev, q_host, k_cache, v_cache, seq_lens, tok_begin, tok_end, out, lse) -> StepRecord:
+        """One layer by itself: GPU stage enqueued first, the CPU stage runs beside it on this thread."""
+        t_wall = time.perf_counter()
+        self.launch_gpu(q_dev, k_cache, v_cache, seq_lens, tok_begin, tok_end)
+        staged = self.cpu_stage(q_host)
+        self.finish(staged, out, lse)
+        torch.cuda.current_stream(self.dev).synchronize()
+        return self.collect((time.perf_counter() - t_wall) * 1e3)       # Algorithm 1, for the next step
+
+
+class HybridPipeline:
+    """Several layers run the way the paper's timeline shows (Section 4.3, workflow step 1): while the GPU works
+    on layer i, a host thread already runs the CPU stage of layer i + 1.  One ``HybridAttentionStep`` per layer
+    (each with its own buffers); the per-layer queries are inputs - deriving layer i + 1's query from layer i's
+    input is the paper's speculation, outside this package.  A single (K, strategy) serves all layers of a pass
+    and is updated once per pass from the mean latencies.
+    """
+
+    def __init__(self, layers: List[HybridAttentionStep]):
+        from concurrent.futures import ThreadPoolExecutor
+        self.layers = layers
+        self.pool = ThreadPoolExecutor(max_workers=1)
+
+    def run(self, q_dev: List[torch.Tensor], q_host: List[torch.Tensor], kv: List[tuple], outs: List[tuple],
+            pipelined: bool = True) -> float:
+        """``kv[i] = (k_cache, v_cache, seq_lens, tok_begin, tok_end)``, ``outs[i] = (out, lse)``.  Returns the wall
+        time of the pass in ms.  ``pipelined=False`` runs the same work layer after layer (for comparison)."""
+        L = self.layers
+        dev = L[0].dev
+        k, strategy = L[0].k, L[0].strategy
+        for e in L:
+            e.set_operating_point(k, strategy)
+        t0 = time.perf_counter()
+        fut = self.pool.submit(L[0].cpu_stage, q_host[0]) if pipelined else None
+        for i, e in enumerate(L):
+            e.launch_gpu(q_dev[i], *kv[i])
+            staged = fut.result() if pipelined else e.cpu_stage(q_host[i])
+            if pipelined and i + 1 < len(L):
+                fut = self.pool.submit(L[i + 1].cpu_stage, q_host[i + 1])     # overlaps layer i's GPU work and transfer
+            e.finish(staged, *outs[i])
+            if not pipelined:
+                torch.cuda.current_stream(dev).synchronize()
+        torch.cuda.current_stream(dev).synchronize()
+        ms = (time.perf_counter() - t0) * 1e3
+        recs = [e.collect(update=False) for e in L]
+        mean = lambda f: sum(getattr(r, f) for r in recs) / len(recs)
+        k, strategy = L[0].sched.update(mean("t_gpu"), mean("t_cpu"), mean("t_tx"))
+        for e in L:
+            e.set_operating_point(k, strategy)
+        return ms
 
 
 class HostKvStore:

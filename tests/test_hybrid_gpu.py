@@ -193,3 +193,43 @@ def test_host_store_on_bound_and_registered_tier_memory():
     del eng
     for t in store._tiers:
         t.free()
+
+
+def test_layer_pipeline_overlaps_cpu_stages_and_gives_the_same_results():
+    """Three layers (same cache, a query per layer): with the CPU stage of layer i + 1 running on a host thread
+    while the GPU handles layer i, every layer's result is what the layer-after-layer order gives, and equals
+    attention over the GPU slice plus the tokens that layer chose; one (K, strategy) per pass."""
+    G, L = 2, 3
+    w = W.AttnWorkload("pipe", 2, 2 * G, 2, 128, "f16", [1300, 600], [900, 350], [1300, 600], page_size=16,
+                       chunk_tokens=128, seed=555)
+    K_t, V_t = w.kv_logical("k"), w.kv_logical("v")
+    prob = DeviceProblem(w, DEV)
+    n_host = torch.tensor(w.tok_begin, dtype=torch.int32)
+    gen = torch.Generator().manual_seed(3)
+    q_host = [torch.randn(w.B, w.Hq, w.D, generator=gen).half() for _ in range(L)]
+    q_dev = [q.to(DEV) for q in q_host]
+    kv = [(prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end)] * L
+    layers = [hybrid.HybridAttentionStep(prob.desc, K_t, V_t, n_host, k_min=64, k_max=128, k_step=32, handoff_chunk=64,
+                                         host_threads=2, device=DEV) for _ in range(L)]
+    pipe = hybrid.HybridPipeline(layers)
+    Kb, Vb = bits(K_t), bits(V_t)
+    results = {}
+    for pipelined in (False, True):
+        for e in layers:
+            e.set_operating_point(64, hybrid.POST_QK)
+        outs = [(torch.empty_like(prob.out), torch.empty_like(prob.lse)) for _ in range(L)]
+        with torch.cuda.device(DEV):
+            ms = pipe.run(q_dev, q_host, kv, outs, pipelined=pipelined)
+        assert ms > 0
+        recs = [e.history[-1] for e in layers]
+        assert all(r.k == 64 and r.strategy == hybrid.POST_QK for r in recs)
+        mean = lambda f: sum(getattr(r, f) for r in recs) / L
+        want = P.feedback_scheduler_step(64, hybrid.POST_QK, mean("t_gpu"), mean("t_cpu"), mean("t_tx"), 64, 128, 32)
+        assert all((e.k, e.strategy) == want for e in layers)              # one operating point for all layers
+        for i, e in enumerate(layers):
+            ref_out, ref_lse = reference(w, bits(q_host[i]), Kb, Vb, e.idx, e.n_sel, G)
+            out, lse = outs[i][0].double().cpu().numpy(), outs[i][1].double().cpu().numpy()
+            assert np.abs(out - ref_out).max() <= OUT_MAX_ABS and np.abs(lse - ref_lse).max() <= LSE_ABS
+        results[pipelined] = [(o.clone(), l.clone()) for o, l in outs]
+    for (o0, l0), (o1, l1) in zip(results[False], results[True]):
+        assert torch.equal(o0, o1) and torch.equal(l0, l1)
