@@ -5,10 +5,18 @@ A step is one pass of the whole path over one batch of synthetic input: hg_attn_
 GPU-resident KV slice, then hg_attn_merge of the chunk partials with the partials of the host-held
 slice.  Prints ONE JSON line (rank 0).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME|all] [--repeats R] [--impl reference]
 
-N > 1 is launched under torchrun, one rank per GPU; every rank runs its own copy of the workload
-(independent sequences, no data-path collective): weak scaling.
+Without --workload the headline (value, roofline, e2e, cpu_baseline) is the largest single-GPU
+configuration, `opt30b`, and `config.workloads` carries one record per configuration (the four
+32K-1M-token ones with their roofline and end-to-end figures, `tiny` in microseconds only).  Every
+workload's timed pass of K steps is repeated R times; the headline is the median repeat.
+
+N > 1: one rank per GPU, each running its own copy of the workload (independent sequences, no
+data-path collective): weak scaling.  Started without a launcher (no WORLD_SIZE in the environment)
+the script starts its own N ranks through torch.distributed.run.  With N > 1 the line also carries
+`sharded`: the 1M-token configuration cut by token range over the N ranks, the one mode of the path
+with a real exchange step (an all-gather of one merged row per head into local memory).
 """
 import argparse
 import json
@@ -26,17 +34,16 @@ if ROOT not in sys.path:
 METRIC = "decode attention KV tokens/s"
 UNIT = "KV tokens/s"
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the partial kernel, from the ncu
-# captures summarised under profiles/ (None until a capture of that workload exists)
+HEADLINE = "opt30b"                      # the largest configuration that fits one GPU (7.5 GB of KV per step)
+LARGE = ("opt13b", "opt30b", "llama70b", "ragged")
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the partial kernel, one ncu capture per workload
+# (absent until a capture of that workload exists).  Traffic grows in proportion to the tokens processed, so a
+# capture of the first sequences is scaled to the full launch.
 NCU_TRAFFIC_BYTES = {
-    # profiles/partial_kernel_opt13b.md: two sequences captured (805.55 MB read + 5.01 MB written), x 4
-    "opt13b": 4 * (805_546_496 + 5_009_664),
-    # profiles/partial_kernel_llama70b.md: the full launch captured
-    "llama70b": 1_718_226_000 + 7_822_080,
-    # profiles/partial_kernel_opt30b.md: one of the four sequences captured (1879.14 MB read + 3.87 MB written), x 4
-    "opt30b": 4 * (1_879_144_000 + 3_870_464),
-    # profiles/partial_kernel_ragged.md: the full launch captured
-    "ragged": 951_494_144 + 8_356_864,
+    "opt13b": 4 * (805_546_496 + 5_009_664),          # two of the eight sequences captured, x 4
+    "llama70b": 1_718_226_000 + 7_822_080,            # the full launch captured
+    "opt30b": 4 * (1_879_144_000 + 3_870_464),        # one of the four sequences captured, x 4
+    "ragged": 951_494_144 + 8_356_864,                # the full launch captured
 }
 
 
@@ -64,12 +71,20 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+def launcher_command(args_list, n, port=None):
+    """The command that starts `n` ranks of this script on this node (one per GPU)."""
+    port = port or (29500 + os.getpid() % 1500)
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(args_list)
+
+
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed regions run."""
 
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, index):
         self.index, self.proc, self.lines = index, None, []
@@ -77,7 +92,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "25"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -88,29 +103,34 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append((time.time(), line.strip()))
 
-    def stop(self, t0, t1):
+    def window(self, t0, t1, fallback_all=True):
+        """Median SM clock, maximum clock and the throttle reasons seen between wall times t0 and t1."""
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            pass
-        rows = [l for t, l in self.lines if t0 - 0.05 <= t <= t1 + 0.2] or [l for _, l in self.lines]
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"], "samples": 0}
+        rows = [l for t, l in list(self.lines) if t0 - 0.03 <= t <= t1 + 0.05]
+        if not rows and fallback_all:
+            rows = [l for _, l in list(self.lines)]
         sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for l in rows:
             p = [x.strip() for x in l.split(",")]
             try:
                 sm.append(float(p[0])); mx.append(float(p[1]))
             except Exception:
                 continue
-            for n, v in zip(names, p[3:7]):
+            for n, v in zip(self.NAMES, p[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
                 "reasons": sorted(reasons), "samples": len(sm)}
+
+    def stop(self):
+        if self.proc is None:
+            return
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
 
 
 def oracle_sample(w, rows_budget, device):
@@ -171,7 +191,7 @@ def time_oracle(w, device, target_core_seconds=20.0):
     t0 = time.perf_counter()
     oracle_pass(w, items, threads)
     dt = time.perf_counter() - t0
-    return {"value": tokens / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+    return {"value": tokens / dt, "unit": UNIT, "cores": threads, "kind": "oracle", "workload": w.name,
             "sample": f"{len(items)} of {w.B * w.Hq} (sequence, head) rows, full GPU slice each, "
                       f"chunked PARTIAL + MERGE in fp64, {dt:.2f} s"}, items, tokens
 
@@ -297,7 +317,8 @@ def run_reference(args, rank, world):
     import torch
     from oracle import hg_oracle as O
     from paper_2604_18529_b200 import workload as W
-    w = W.make_workload(args.workload)
+    name = HEADLINE if args.workload in (None, "all") else args.workload
+    w = W.make_workload(name)
     dev = "cuda:0" if torch.cuda.is_available() else "cpu"
     threads = O.host_threads()
     items, tokens = oracle_sample(w, max(threads, 16), dev)
@@ -311,48 +332,39 @@ def run_reference(args, rank, world):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": args.workload, "sample": f"{len(items)} of {w.B * w.Hq} (sequence, head) rows per step"},
+            "config": {"workload": name, "sample": f"{len(items)} of {w.B * w.Hq} (sequence, head) rows per step"},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
                              "sample": f"{len(items)} rows x {args.steps} steps"},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", default="opt13b")
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--batch", type=int, default=0, help="keep only the first BATCH sequences (small profiling captures)")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--probe", action="store_true", help="also time the read-probe kernel")
-    ap.add_argument("--extras", action="store_true",
-                    help="also time the hand-off kernel, the host logits calculator and the residency operations")
-    args = ap.parse_args()
-    args.warmup = max(args.warmup, 3)
+class Ranks:
+    """This process's place in the job, its device and the barrier every timed region is bracketed by."""
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    if args.impl == "reference":
-        return run_reference(args, rank, world)
+    def __init__(self, rank, local_rank, world):
+        self.rank, self.local_rank, self.world = rank, local_rank, world
+        self.dev = f"cuda:{local_rank}"
 
+    def barrier(self):
+        import torch
+        import torch.distributed as dist
+        torch.cuda.synchronize()
+        if self.world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+
+def measure_workload(name, args, R, sampler):
+    """All timings of one workload on this rank's GPU; times are the maximum over ranks.  Returns the record of
+    `config.workloads` plus, under "_headline", what the top-level keys need (rank 0 only reads it)."""
     import torch
-    import torch.distributed as dist
     import paper_2604_18529_b200 as pkg
     from paper_2604_18529_b200 import workload as W
     from paper_2604_18529_b200.problem import DeviceProblem
 
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
-    torch.cuda.set_device(local_rank)
-    dev = f"cuda:{local_rank}"
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(dev))
-
-    w = W.make_workload(args.workload)
+    dev, K = R.dev, args.steps
+    w = W.make_workload(name)
     if args.batch:
         w = W.first_sequences(w, args.batch)
     prob = DeviceProblem(w, dev)
@@ -363,54 +375,50 @@ def main():
              torch.randn(w.B, w.Hq, 1, device=dev, generator=gen),
              torch.rand(w.B, w.Hq, 1, device=dev, generator=gen) + 1.0)]
     stream = torch.cuda.current_stream()
-
-    def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
     step = prob.prepare_step(host)          # both calls with their arguments marshalled once, as a decode loop would
+    torch.cuda.synchronize()
+    time.sleep(0.5)                         # input generation is heavy integer work: let the power average settle
     for _ in range(args.warmup):
         step()
     torch.cuda.synchronize()
     if int(prob.status.item()) != 0:
-        raise SystemExit(f"device status {int(prob.status.item())} after warm-up")
+        raise SystemExit(f"{name}: device status {int(prob.status.item())} after warm-up")
 
-    # ---- pass A: exactly K steps, device-timed ------------------------------------------------------
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.3)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    t_wall0 = time.time()
-    ev0.record(stream)
-    for _ in range(args.steps):
-        step()
-    ev1.record(stream)
-    barrier()
-    t_wall1 = time.time()
-    ms_total = ev0.elapsed_time(ev1)
+    # ---- pass A: exactly K steps between one pair of events, repeated ----------------------------------------
+    reps = []
+    for _ in range(max(1, args.repeats)):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        R.barrier()
+        t0 = time.time()
+        ev0.record(stream)
+        for _ in range(K):
+            step()
+        ev1.record(stream)
+        R.barrier()
+        t1 = time.time()
+        reps.append((ev0.elapsed_time(ev1), t0, t1))
+    rep_ms = max_over_ranks([r[0] for r in reps], dev)
+    order = sorted(range(len(rep_ms)), key=lambda i: rep_ms[i])
+    med = order[(len(order) - 1) // 2]       # the median repeat (the lower one of an even count)
+    ms_step = rep_ms[med] / K
 
-    # ---- pass B: K more steps with an event around every kernel (roofline of the dominant kernel) --------
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    # ---- pass B: K more steps with an event around every kernel (roofline of the dominant kernel) ----------
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    tb0 = time.time()
     for e in evs:
         e[0].record(stream); prob.partial(); e[1].record(stream); prob.merge(host); e[2].record(stream)
     torch.cuda.synchronize()
-    t_wall1 = time.time()
-    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
-    part_ms = [e[0].elapsed_time(e[1]) for e in evs]
-    merge_ms = [e[1].elapsed_time(e[2]) for e in evs]
+    tb1 = time.time()
+    part_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
+    merge_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
 
-    # ---- end to end: per-step data in pinned host memory, results read back ----------------------------------
+    # ---- end to end: per-step data in pinned host memory, results read back every step -----------------------
     pin = lambda t: t.cpu().pin_memory()
     q_h, sl_h, tb_h, te_h = pin(prob.q), pin(prob.seq_lens), pin(prob.tok_begin), pin(prob.tok_end)
     host_h = [tuple(pin(x) for x in src) for src in host]
     out_h = torch.empty(prob.out.shape, dtype=torch.float32).pin_memory()
     lse_h = torch.empty(prob.lse.shape, dtype=torch.float32).pin_memory()
     ws = torch.empty(pkg.hg_attn_workspace_bytes(prob.desc, 1), dtype=torch.uint8, device=dev)
-
     decode_host = pkg.prepare_decode_host(q_h, prob.kv["k"], prob.kv["v"], sl_h, tb_h, te_h, host_h, out_h, lse_h, ws,
                                           prob.desc)     # arguments marshalled once, as a decode loop would
 
@@ -420,23 +428,23 @@ def main():
 
     for _ in range(3):
         e2e_step()
-    barrier()
+    R.barrier()
     ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ee0.record(stream)
-    for _ in range(args.steps):
+    for _ in range(K):
         e2e_step()
     ee1.record(stream)
-    barrier()
-    e2e_ms = ee0.elapsed_time(ee1)
+    R.barrier()
+    (e2e_ms,) = max_over_ranks([ee0.elapsed_time(ee1)], dev)
     same = torch.equal(out_h, prob.out.cpu()) and torch.equal(lse_h, prob.lse.cpu())
     h2d = sum(t.numel() * t.element_size() for t in (q_h, sl_h, tb_h, te_h)) + \
         sum(t.numel() * t.element_size() for src in host_h for t in src)
     d2h = out_h.numel() * 4 + lse_h.numel() * 4
 
-    probe_ms = None
+    probe_us = None
     if args.probe:
         sink = torch.zeros(w.B, w.Hkv, prob.NC, dtype=torch.int32, device=dev)
-        pe = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
+        pe = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(K)]
         for _ in range(3):
             pkg.hg_kv_read_probe(prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end, sink, prob.desc)
         for e in pe:
@@ -444,51 +452,210 @@ def main():
             pkg.hg_kv_read_probe(prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end, sink, prob.desc)
             e[1].record(stream)
         torch.cuda.synchronize()
-        probe_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in pe)
+        probe_us = statistics.mean(e[0].elapsed_time(e[1]) for e in pe) * 1e3
+    extras = time_extras(w, prob, dev, K) if args.extras and R.rank == 0 and name != "tiny" else None
+    if int(prob.status.item()) != 0:
+        raise SystemExit(f"{name}: device status {int(prob.status.item())} after the timed passes")
 
-    extras = time_extras(w, prob, dev, args.steps) if args.extras and rank == 0 else None
-    ms_total, e2e_ms = max_over_ranks([ms_total, e2e_ms], dev)
+    tokens = w.gpu_tokens
+    kv_bytes = w.kv_bytes()
+    large = kv_bytes > 2 * 126e6
+    peak, peak_kind = measured_peak()
+    nchunks = sum(w.chunk_grid(b)[1] for b in range(w.B))
+    part_alg = kv_bytes + w.B * w.Hq * w.D * 2 + (prob.kv["num_pages"] * 4 if w.paged else 0) + w.Hq * nchunks * (w.D + 2) * 4
+    achieved = part_alg / (part_ms * 1e-3) / 1e9
+    step_gbs = prob.alg_bytes() / (ms_step * 1e-3) / 1e9
+    clocks_med = sampler.window(reps[med][1], reps[med][2]) if sampler else None
+    rec = {
+        "workload": w.name, "batch": w.B, "q_heads": w.Hq, "kv_heads": w.Hkv, "head_dim": w.D, "kv_dtype": w.dtype,
+        "context": max(w.seq_lens), "gpu_tokens": tokens, "page_size": w.page_size, "chunk_tokens": w.chunk_tokens,
+        "kv_bytes_per_step": kv_bytes,
+        "l2": "inputs larger than L2" if large else "inputs fit L2: launch-bound case, microseconds only",
+        "us_per_step": ms_step * 1e3, "ms_per_step": ms_step,
+        "repeats_ms_per_step": {"median": ms_step, "min": min(rep_ms) / K, "max": max(rep_ms) / K,
+                                "all": [m / K for m in rep_ms],
+                                "sm_mhz": [sampler.window(r[1], r[2], fallback_all=False)["sm_mhz"] if sampler else None
+                                           for r in reps]},
+        "kv_tokens_per_s": whole_job_value(tokens, R.world, ms_step),
+        "partial_us": part_ms * 1e3, "merge_us": merge_ms * 1e3,
+        "kernel_timing": "a second pass of K steps with CUDA events around each kernel; those events keep the merge "
+                         "from starting as a programmatic dependent inside the partial kernel's tail, so partial_us + "
+                         "merge_us can exceed the step time of the first pass",
+        "probe_us": probe_us, "extras": extras,
+        "clocks": clocks_med,
+        "e2e": {"value": whole_job_value(tokens, R.world, e2e_ms / K), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / K, "matches_device_path": bool(same),
+                "api": "hg_attn_decode_host via prepare_decode_host (KV pools stay device resident: they are the "
+                       "GPU's slice of the cache)"},
+    }
+    if large:
+        rec["step_gbs"] = step_gbs
+        rec["step_frac_of_8000"] = step_gbs / 8000.0
+        rec["roofline"] = {"bound": "hbm", "kernel": "partial_kernel", "achieved": achieved, "peak": peak,
+                           "peak_kind": f"{peak_kind} copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
+                           "frac_of_8000": achieved / 8000.0, "alg_bytes_per_launch": part_alg,
+                           "traffic": None if args.batch else NCU_TRAFFIC_BYTES.get(name)}
+    else:
+        # the contract asks for a roofline object on every line; for a launch-bound case it is context only
+        rec["roofline"] = {"bound": "hbm", "kernel": "partial_kernel", "achieved": achieved, "peak": peak,
+                           "peak_kind": f"{peak_kind} copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
+                           "frac_of_8000": achieved / 8000.0, "alg_bytes_per_launch": part_alg, "traffic": None,
+                           "note": "launch-bound: the inputs fit L2"}
+    rec["_headline"] = {"w": w, "ms_step": ms_step, "tokens": tokens, "wall": (reps[0][1], tb1)}
+    del prob, ws, host
+    torch.cuda.empty_cache()
+    return rec
 
-    if rank == 0:
-        tokens = w.gpu_tokens
-        ms_step = ms_total / args.steps
-        peak, peak_kind = measured_peak()
-        kv_bytes = w.kv_bytes()
-        nchunks = sum(w.chunk_grid(b)[1] for b in range(w.B))
-        part_alg = kv_bytes + w.B * w.Hq * w.D * 2 + (prob.kv["num_pages"] * 4 if w.paged else 0) + \
-            w.Hq * nchunks * (w.D + 2) * 4
-        part_avg = statistics.mean(part_ms)
-        achieved = part_alg / (part_avg * 1e-3) / 1e9
-        line = {
-            "metric": METRIC, "value": whole_job_value(tokens, world, ms_step), "unit": UNIT, "n_gpus": world,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": w.name, "batch": w.B, "q_heads": w.Hq, "kv_heads": w.Hkv, "head_dim": w.D,
-                       "kv_dtype": w.dtype, "context": max(w.seq_lens), "gpu_tokens": tokens, "page_size": w.page_size,
-                       "chunk_tokens": w.chunk_tokens, "kv_bytes_per_step": kv_bytes,
-                       "l2": "inputs larger than L2" if kv_bytes > 2 * 126e6 else "inputs fit L2 (launch-bound case)",
-                       "step_gbs": prob.alg_bytes() / (ms_step * 1e-3) / 1e9,
-                       "step_frac_of_8000": prob.alg_bytes() / (ms_step * 1e-3) / 1e9 / 8000.0,
-                       "partial_us": part_avg * 1e3, "merge_us": statistics.mean(merge_ms) * 1e3,
-                       "roofline_timing": "second pass of K steps with CUDA events around each kernel",
-                       "probe_us": None if probe_ms is None else probe_ms * 1e3, "extras": extras},
-            "roofline": {"bound": "hbm", "kernel": "partial_kernel", "achieved": achieved, "peak": peak,
-                         "peak_kind": f"{peak_kind} copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
-                         "frac_of_8000": achieved / 8000.0, "alg_bytes_per_launch": part_alg,
-                         "traffic": None if args.batch else NCU_TRAFFIC_BYTES.get(args.workload)},
-            "e2e": {"value": whole_job_value(tokens, world, e2e_ms / args.steps), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps, "matches_device_path": bool(same),
-                    "api": "hg_attn_decode_host via prepare_decode_host (KV pools stay device resident: they are the GPU's slice of the cache)"},
-            "gpu_launches": 2 * args.steps,
-            "clocks": clocks,
-        }
-        if not args.no_cpu_baseline and world == 1:
-            line["cpu_baseline"] = time_oracle(w, dev)[0]
-        elif world == 1:
-            line["cpu_baseline"] = None
-        print(json.dumps(line), flush=True)
-    if world > 1:
+
+def measure_sharded(args, R):
+    """The 1M-token configuration cut by token range over the ranks: local decode over this rank's range, one
+    all-gather of a merged row per (sequence, head) into local memory, local merge.  Times are max over ranks."""
+    import dataclasses
+    import torch
+    import torch.distributed as dist
+    from paper_2604_18529_b200 import sharded, workload as W
+    from paper_2604_18529_b200.problem import DeviceProblem
+
+    dev, K = R.dev, args.steps
+    w = W.make_workload("llama70b")
+    begins, ends = sharded.shard_ranges(w.tok_begin, w.tok_end, R.world, w.chunk_tokens)
+    mine = dataclasses.replace(w, name=f"llama70b[rank {R.rank}/{R.world}]", tok_begin=begins[R.rank], tok_end=ends[R.rank])
+    prob = DeviceProblem(mine, dev)          # only this rank's pages are resident
+    gen = torch.Generator(device=dev).manual_seed(w.seed)
+    host = [(torch.randn(w.B, w.Hq, 1, w.D, device=dev, generator=gen),
+             torch.randn(w.B, w.Hq, 1, device=dev, generator=gen),
+             torch.rand(w.B, w.Hq, 1, device=dev, generator=gen) + 1.0)] if R.rank == 0 else []
+    eng = sharded.TokenShardedDecode(prob.desc, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        eng.step(prob.q, prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end, host, prob.out, prob.lse)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    R.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(K):
+        step()
+    e1.record(stream)
+    R.barrier()
+    x0, x1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    x0.record(stream)
+    for _ in range(K):
+        if dist.is_initialized():
+            sharded.exchange_records(eng.record, None, eng.gathered)
+    x1.record(stream)
+    R.barrier()
+    step_ms, exch_ms = max_over_ranks([e0.elapsed_time(e1) / K, x0.elapsed_time(x1) / K], dev)
+    tokens = w.gpu_tokens
+    return {"workload": "llama70b", "split": "token ranges on the chunk grid, older tokens on lower ranks",
+            "ranks": R.world, "gpu_tokens_total": tokens, "tokens_this_rank": mine.gpu_tokens,
+            "ms_per_step": step_ms, "kv_tokens_per_s": tokens / (step_ms * 1e-3),
+            "exchange": "all-gather of B*Hq*(D+1) floats per rank into local memory, then hg_attn_merge over the ranks' rows",
+            "exchange_bytes_per_rank": int(eng.record.numel() * 4), "exchange_ms": exch_ms,
+            "exchange_share": exch_ms / step_ms if step_ms > 0 else None, "scaling": "strong"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="all", help="one of tiny, opt13b, opt30b, llama70b, ragged; or all (default)")
+    ap.add_argument("--repeats", type=int, default=5, help="times the K-step pass is repeated per workload")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=0, help="keep only the first BATCH sequences (small profiling captures)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sharded", action="store_true", help="add the token-sharded record even on one rank")
+    ap.add_argument("--probe", action="store_true", help="also time the read-probe kernel")
+    ap.add_argument("--extras", action="store_true",
+                    help="also time the hand-off kernel, the host logits calculator and the residency operations")
+    ap.add_argument("--launch-check", action="store_true",
+                    help="only start the ranks (gloo, no GPU needed) and print which ranks met; not a bench line")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started without a launcher: start the ranks, one per GPU; rank 0's line is this command's line
+        print(f"bench.py: starting {args.gpus} ranks through torch.distributed.run", file=sys.stderr, flush=True)
+        raise SystemExit(subprocess.call(launcher_command(sys.argv[1:], args.gpus), cwd=ROOT))
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.launch_check:
+        import torch.distributed as dist
+        dist.init_process_group("gloo")
+        seen = [None] * world
+        dist.all_gather_object(seen, rank)
+        got = max_over_ranks([float(rank)])
+        dist.barrier()
         dist.destroy_process_group()
+        if rank == 0:
+            print(json.dumps({"launch_check": True, "world": world, "ranks_seen": seen, "max_rank": got[0]}), flush=True)
+        return
+    if args.impl == "reference":
+        return run_reference(args, rank, world)
+
+    import torch
+    import torch.distributed as dist
+
+    print(f"bench.py: rank {rank} of {world}", file=sys.stderr, flush=True)
+    if not torch.cuda.is_available():
+        raise SystemExit(f"bench.py (rank {rank} of {world}) needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    R = Ranks(rank, local_rank, world)
+    if world > 1:
+        os.environ.setdefault("NCCL_DEBUG", "INFO")          # communicator lines (ranks, transport) stay visible
+        os.environ.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+        dist.init_process_group("nccl", device_id=torch.device(R.dev))
+
+    # the group-query configurations first: their consumer warps are the most clock-sensitive, and the 7.5 GB
+    # configuration leaves the board at its power cap for the measurements that follow it
+    names = ["tiny", "ragged", "llama70b", "opt13b", "opt30b"] if args.workload == "all" else [args.workload]
+    head_name = HEADLINE if args.workload == "all" else args.workload
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.3)
+    recs = {n: measure_workload(n, args, R, sampler) for n in names}
+    shard_rec = measure_sharded(args, R) if (world > 1 or args.sharded) and args.workload == "all" else None
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+    time.sleep(0.2)
+    head = recs[head_name]
+    hl = head.pop("_headline")
+    for r in recs.values():
+        r.pop("_headline", None)
+    sampler.stop()
+    config = {k: head[k] for k in ("workload", "batch", "q_heads", "kv_heads", "head_dim", "kv_dtype", "context", "gpu_tokens",
+                                  "page_size", "chunk_tokens", "kv_bytes_per_step", "l2", "partial_us", "merge_us",
+                                  "kernel_timing", "probe_us", "extras", "repeats_ms_per_step")}
+    config["step_gbs"] = head.get("step_gbs")
+    config["step_frac_of_8000"] = head.get("step_frac_of_8000")
+    config["headline"] = f"the median of {max(1, args.repeats)} repeats of {args.steps} steps of `{head['workload']}`"
+    if args.workload == "all":
+        config["workloads"] = [recs[n] for n in names]
+        config["min_step_frac_of_8000"] = min(recs[n]["step_frac_of_8000"] for n in LARGE)
+    line = {
+        "metric": METRIC, "value": head["kv_tokens_per_s"], "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": hl["ms_step"], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": config, "roofline": head["roofline"], "e2e": head["e2e"],
+        "gpu_launches": 2 * args.steps,
+        "clocks": head["clocks"],
+    }
+    if shard_rec is not None:
+        line["sharded"] = shard_rec
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = time_oracle(hl["w"], R.dev)[0]
+    elif world == 1:
+        line["cpu_baseline"] = None
+    print(json.dumps(line), flush=True)
 
 
 if __name__ == "__main__":

@@ -35,3 +35,28 @@ def test_bench_line_has_the_contract_keys():
     assert e["value"] > 0 and e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0 and e["matches_device_path"] is True
     assert d["gpu_launches"] == 2 * d["steps"]
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
+
+
+def test_default_line_covers_every_configuration_and_headlines_the_largest():
+    d = run_bench("--steps", "3", "--warmup", "3", "--repeats", "3", "--no-cpu-baseline", "--sharded")
+    c = d["config"]
+    assert c["workload"] == "opt30b" and d["dtype"] == "f32"
+    names = [r["workload"] for r in c["workloads"]]
+    assert sorted(names) == sorted(["tiny", "opt13b", "opt30b", "llama70b", "ragged"])
+    for r in c["workloads"]:
+        assert r["ms_per_step"] > 0 and r["partial_us"] > 0 and r["merge_us"] > 0 and r["e2e"]["matches_device_path"] is True
+        rp = r["repeats_ms_per_step"]
+        assert len(rp["all"]) == 3 and rp["min"] <= rp["median"] <= rp["max"] and len(rp["sm_mhz"]) == 3
+        assert set(r["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
+        if r["workload"] == "tiny":
+            assert "step_frac_of_8000" not in r and r["us_per_step"] > 0
+        else:
+            ro = r["roofline"]
+            assert 0.3 < r["step_frac_of_8000"] < 1.05 and ro["traffic"] > 0.99 * ro["alg_bytes_per_launch"]
+            assert abs(ro["frac"] - ro["achieved"] / ro["peak"]) < 1e-9
+    head = [r for r in c["workloads"] if r["workload"] == "opt30b"][0]
+    assert d["ms_per_step"] == head["ms_per_step"] and d["value"] == head["kv_tokens_per_s"]
+    assert d["roofline"] == head["roofline"] and d["e2e"] == head["e2e"]
+    assert c["min_step_frac_of_8000"] == min(r["step_frac_of_8000"] for r in c["workloads"] if r["workload"] != "tiny")
+    s = d["sharded"]
+    assert s["ranks"] == 1 and s["gpu_tokens_total"] == 419430 and s["tokens_this_rank"] == 419430 and s["ms_per_step"] > 0

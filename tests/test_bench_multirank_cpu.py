@@ -57,3 +57,44 @@ def test_reference_arm_runs_on_rank_zero_only(monkeypatch, capsys):
     line = json.loads(capsys.readouterr().out)
     assert line["impl"] == "reference" and line["value"] > 0 and line["cpu_baseline"]["kind"] == "oracle"
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["unit"] == "KV tokens/s"
+
+
+def _run_bench(*args):
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    return subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), *args], capture_output=True, text=True,
+                          timeout=600, cwd=ROOT, env=env)
+
+
+def test_gpus_n_starts_its_own_ranks():
+    """`bench.py --gpus 2` without a launcher starts two ranks itself; they meet over gloo and rank 0 alone prints."""
+    import json
+    out = _run_bench("--gpus", "2", "--launch-check")
+    assert out.returncode == 0, out.stderr[-2000:]
+    assert "starting 2 ranks" in out.stderr
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d == {"launch_check": True, "world": 2, "ranks_seen": [0, 1], "max_rank": 1.0}
+
+
+def test_gpus_n_without_cuda_fails_in_every_rank_after_the_spawn():
+    import torch
+    if torch.cuda.is_available():
+        import pytest
+        pytest.skip("a CUDA device is present: the ranks would run the bench")
+    out = _run_bench("--gpus", "2", "--steps", "1")
+    assert out.returncode != 0
+    assert "starting 2 ranks" in out.stderr
+    for r in (0, 1):
+        assert f"bench.py (rank {r} of 2) needs a CUDA device" in out.stderr
+    assert not [l for l in out.stdout.splitlines() if l.startswith("{")]
+
+
+def test_launcher_command_is_one_rank_per_gpu_on_loopback():
+    sys.path.insert(0, ROOT)
+    import bench
+    cmd = bench.launcher_command(["--gpus", "4", "--steps", "2"], 4, port=29999)
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"] and "--nproc-per-node=4" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[cmd.index("--master-port") + 1] == "29999"
+    assert cmd[-4:] == ["--gpus", "4", "--steps", "2"] and cmd[-5].endswith("bench.py")
