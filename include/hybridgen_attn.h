@@ -66,12 +66,15 @@ typedef enum hg_dtype { HG_DTYPE_F16 = 0, HG_DTYPE_BF16 = 1 } hg_dtype;
                                    attention itself.  hg_attn_decode and its variants always work this way on
                                    their own workspace. */
 
-/* values the kernels may write to *hg_attn_desc.status (device word, optional) */
+/* bits the kernels may set in *hg_attn_desc.status (device word, optional; several may be set at once) */
 #define HG_DEV_OK 0
 #define HG_DEV_WAIT_TIMEOUT 1 /* a bounded on-chip barrier wait ran out; the call's results are invalid.
-                                 While the word holds this value the kernels skip their work, so clear
-                                 it before the next call. */
-#define HG_DEV_BAD_PAGE 2     /* a block-table entry of a resident page was outside [0, num_pages) */
+                                 While this bit is set the kernels skip their work, so clear the word
+                                 before the next call. */
+#define HG_DEV_BAD_PAGE 2     /* a block-table entry of a resident page was outside [0, num_pages): the page was not
+                                 read and its tokens were left out of the partial, as if they were not resident */
+#define HG_DEV_RANGE 4        /* a slice reached past max_pages * page_size tokens, the end of its block-table row:
+                                 it was cut there (the partials cover [tok_begin, max_pages * page_size)) */
 
 /*
  * Problem description (host struct).
@@ -118,7 +121,21 @@ typedef struct hg_attn_desc {
                                   batches); NULL: items are dealt round-robin.  Left alone when the problem has no
                                   more items than the device has resident CTAs.  Must not be shared by calls
                                   that may overlap on the GPU.  Present when struct_size covers it. */
+    uint32_t tune;             /* HG_TUNE_* bits; 0 = the library's defaults.  Each bit switches one choice of the
+                                  schedule off; results do not depend on them (the tests show equal bits), speed
+                                  does.  Present when struct_size covers it, like the two fields below. */
+    int32_t tune_stages;       /* depth of the shared-memory ring of hg_attn_partial, 2..8; 0 = default (3) */
+    int32_t tune_ctas_per_sm;  /* upper limit on resident CTAs per SM for hg_attn_partial; 0 = as many as fit */
 } hg_attn_desc;
+
+/* bits of hg_attn_desc.tune */
+#define HG_TUNE_NO_PERSISTENT 1u     /* one CTA per work item instead of a persistent grid */
+#define HG_TUNE_NO_DYNAMIC 2u        /* deal items round-robin even when a work counter is given */
+#define HG_TUNE_NO_PDL 4u            /* no programmatic dependent launches */
+#define HG_TUNE_NO_MERGE_CLUSTER 8u  /* hg_attn_merge: never split a row over a thread-block cluster */
+#define HG_TUNE_NO_MERGE_ROWS 16u    /* hg_attn_merge: never use the warp-per-row kernel */
+#define HG_TUNE_NO_GQA16 32u         /* groups of more than 8 query heads as items of 8 heads, not 16 */
+#define HG_TUNE_NO_HOST_DIRECT 64u   /* hg_attn_decode_host: always stage through the workspace with copies */
 
 /* One source of partials for hg_attn_merge (host struct, dev pointers). */
 typedef struct hg_partial_src {
@@ -179,9 +196,12 @@ int32_t hg_attn_suggest_chunk(int64_t total_tokens, int32_t num_q_heads, int32_t
 /*
  * Bytes of device workspace hg_attn_decode / hg_attn_decode_host need for this problem
  * (chunk partials, plus staging for q, ranges, host partials and results in the _host form).
+ * n_host_partials is the total number of partials per (sequence, head) that the host sources of
+ * hg_attn_decode_host will carry: the sum of their nc fields (a source of nc = 3 counts 3), not the
+ * number of sources.  hg_attn_decode ignores it (its host partials are already on the device).
  * Returns 0 for an invalid description.
  */
-size_t hg_attn_workspace_bytes(const hg_attn_desc* desc, int32_t n_host_src);
+size_t hg_attn_workspace_bytes(const hg_attn_desc* desc, int32_t n_host_partials);
 
 /*
  * One pass of the whole path: hg_attn_partial into workspace, then hg_attn_merge of those
@@ -216,19 +236,22 @@ hg_status hg_attn_decode_host(const void* q_host, const void* k_cache, const voi
  * hg_attn_decode for callers that cannot allocate device memory.  (The paper has no counterpart:
  * this entry point exists for the embedding environment, not for the method.)
  *
- * Who needs it: code that runs where cudaMalloc is off limits - inside a CUDA-graph capture, in a
- * plugin whose host gives it a fixed memory budget and forbids further allocation, or in a
- * latency-critical decode loop that must not take the allocator's lock or trigger an implicit
- * device synchronisation.  Such a caller has the inputs and the output buffers but nowhere to put
- * the chunk partials that sit between the two kernels.
+ * Who needs it: code that runs where cudaMalloc is off limits - a plugin whose host gives it a
+ * fixed memory budget and forbids further allocation, a latency-critical decode loop that must
+ * not take the allocator's lock or trigger the implicit device synchronisation cudaFree brings,
+ * a component that is handed buffers by its framework and has no allocator of its own.  Such a
+ * caller has the inputs and the output buffers but nowhere to put the chunk partials that sit
+ * between the two kernels.
  *
  * Here those partials live in a fixed array inside the library's device image
  * (HG_STATIC_SCRATCH_BYTES bytes, reserved on every GPU that loads the library for as long as the
  * process lives).  Arguments and results are those of hg_attn_decode minus the workspace.
  *
- *   - Limit: batch * num_q_heads * num_chunks * (head_dim + 2) * 4 bytes (each of the three arrays
- *     rounded up to 256 bytes) must fit in HG_STATIC_SCRATCH_BYTES; a larger problem is refused with
- *     HG_ERR_WORKSPACE and nothing is launched.  Use bigger chunks or hg_attn_decode instead.
+ *   - Limit: with n = batch * num_q_heads * num_chunks, the three partial arrays - n * head_dim * 4
+ *     bytes of o and twice n * 4 bytes of m and l, each array rounded up to a multiple of 256 bytes -
+ *     must fit in HG_STATIC_SCRATCH_BYTES (exactly filling it is accepted); a larger problem is
+ *     refused with HG_ERR_WORKSPACE and nothing is launched.  Use bigger chunks or hg_attn_decode
+ *     instead.
  *   - The first call on each device looks up the array's device address (a symbol query, no
  *     allocation) with that device current.  Make that first call outside any stream capture.
  *   - Neither this call nor anything it calls uses cudaMalloc, cudaFree or an allocating library.

@@ -19,11 +19,13 @@ _lib = None
 
 HG_OK, HG_ERR_INVALID_ARG, HG_ERR_UNSUPPORTED, HG_ERR_CUDA, HG_ERR_WORKSPACE = 0, 1, 2, 3, 4
 HG_DTYPE_F16, HG_DTYPE_BF16 = 0, 1
-HG_DEV_OK, HG_DEV_WAIT_TIMEOUT, HG_DEV_BAD_PAGE = 0, 1, 2
+HG_DEV_OK, HG_DEV_WAIT_TIMEOUT, HG_DEV_BAD_PAGE, HG_DEV_RANGE = 0, 1, 2, 4
 HG_MAX_MERGE_SRC = 8
 HG_FLAG_TEST_STALL = 1
 HG_FLAG_SPARSE_EMPTY = 2
 HG_STATIC_SCRATCH_BYTES = 8 << 20
+(HG_TUNE_NO_PERSISTENT, HG_TUNE_NO_DYNAMIC, HG_TUNE_NO_PDL, HG_TUNE_NO_MERGE_CLUSTER, HG_TUNE_NO_MERGE_ROWS,
+ HG_TUNE_NO_GQA16, HG_TUNE_NO_HOST_DIRECT) = 1, 2, 4, 8, 16, 32, 64
 
 
 class HgError(RuntimeError):
@@ -53,6 +55,9 @@ class HgAttnDesc(C.Structure):
         ("flags", C.c_uint32),
         ("status", C.c_void_p),
         ("sched_counter", C.c_void_p),
+        ("tune", C.c_uint32),
+        ("tune_stages", C.c_int32),
+        ("tune_ctas_per_sm", C.c_int32),
     ]
 
 
@@ -166,7 +171,8 @@ def attn_desc(*, batch: int, num_q_heads: int, num_kv_heads: int, head_dim: int,
               num_pages: int, page_stride: int, head_stride: int, tok_stride: int,
               block_table: Optional[torch.Tensor], max_pages: int, chunk_tokens: int, num_chunks: int,
               scale: float = 0.0, status: Optional[torch.Tensor] = None, flags: int = 0,
-              sched_counter: Optional[torch.Tensor] = None) -> HgAttnDesc:
+              sched_counter: Optional[torch.Tensor] = None, tune: int = 0, tune_stages: int = 0,
+              tune_ctas_per_sm: int = 0) -> HgAttnDesc:
     """Fill an ``hg_attn_desc``.  ``block_table`` (int32 CUDA [B][max_pages]), ``status`` and
     ``sched_counter`` (int32 CUDA scalars) are kept alive by the returned object."""
     d = HgAttnDesc()
@@ -180,6 +186,7 @@ def attn_desc(*, batch: int, num_q_heads: int, num_kv_heads: int, head_dim: int,
     d.scale, d.flags = scale, flags
     d.status = _dev(status, "status", torch.int32)
     d.sched_counter = _dev(sched_counter, "sched_counter", torch.int32)
+    d.tune, d.tune_stages, d.tune_ctas_per_sm = tune, tune_stages, tune_ctas_per_sm
     d._keep = (block_table, status, sched_counter)
     return d
 
@@ -269,8 +276,8 @@ def hg_attn_decode(q, k_cache, v_cache, seq_lens, tok_begin, tok_end, host_parti
 
 def hg_attn_decode_static(q, k_cache, v_cache, seq_lens, tok_begin, tok_end, host_partials, out, lse,
                           desc: HgAttnDesc, stream=None) -> None:
-    """``hg_attn_decode`` for callers that may not allocate device memory (graph capture, fixed-budget
-    plugins, allocator-free decode loops): the chunk partials go to a fixed 8 MiB array inside the
+    """``hg_attn_decode`` for callers that may not allocate device memory (fixed-budget plugins,
+    allocator-free decode loops, components without an allocator): the chunk partials go to a fixed 8 MiB array inside the
     library instead of a caller workspace.  Raises ``HgError`` (workspace) if the problem's partials do
     not fit.  All calls on a device share that array, so calls that could overlap on the GPU must be
     serialised; make the first call on a device outside any stream capture."""

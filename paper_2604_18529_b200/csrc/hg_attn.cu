@@ -8,7 +8,6 @@
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stddef.h>
-#include <stdlib.h>
 #include <string.h>
 
 #include <atomic>
@@ -30,7 +29,7 @@ static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 // The optional trailing field, for callers compiled against a shorter struct.
 static int32_t* desc_sched(const hg_attn_desc* d) {
-    return d->struct_size >= sizeof(hg_attn_desc) ? d->sched_counter : nullptr;
+    return d->struct_size >= offsetof(hg_attn_desc, sched_counter) + sizeof(int32_t*) ? d->sched_counter : nullptr;
 }
 
 static int ilog2_exact(int v) {
@@ -112,11 +111,19 @@ static hg_status make_maps(const hg_attn_desc* d, const void* k, const void* v, 
 
 // ---- launches ---------------------------------------------------------------------------------------
 
-static int env_int(const char* name, int dflt, int lo, int hi) {
-    const char* s = getenv(name);
-    if (!s || !*s) return dflt;
-    int v = atoi(s);
-    return v < lo ? lo : (v > hi ? hi : v);
+// The optional tuning fields (all defaults when the caller's struct ends before them).
+struct Tune {
+    uint32_t bits;
+    int stages, ctas_per_sm;
+    bool off(uint32_t bit) const { return (bits & bit) != 0; }
+};
+
+static Tune desc_tune(const hg_attn_desc* d) {
+    Tune t = {0u, 0, 0};
+    if (d->struct_size >= offsetof(hg_attn_desc, tune_ctas_per_sm) + sizeof(int32_t)) {
+        t.bits = d->tune; t.stages = d->tune_stages; t.ctas_per_sm = d->tune_ctas_per_sm;
+    }
+    return t;
 }
 
 // Per kernel instantiation and device: the shared-memory opt-in that is in force and the occupancy it gives.
@@ -129,7 +136,7 @@ struct LaunchCache {
 
 template <int D, bool BF16, int MODE>
 static hg_status launch_partial_t(const CUtensorMap& tk, const CUtensorMap& tv, PartialParams p, cudaStream_t st,
-                                  bool counter_is_zero) {
+                                  bool counter_is_zero, const Tune& tune) {
     static LaunchCache cache;                     // zero-initialised
     const size_t smem = (size_t)p.stages * ((128 / D) * 2 * TILE_T * D * 2 + 8 * D * 2) + 1024;   // per stage: 128 / D x (K tile, V tile), q rows
     auto kern = partial_kernel<D, BF16, MODE>;
@@ -152,7 +159,7 @@ static hg_status launch_partial_t(const CUtensorMap& tk, const CUtensorMap& tv, 
     if (p.persistent) {
         // one wave of resident CTAs; each takes items from the schedule
         int per_sm = cache.per_sm[dev].load(std::memory_order_relaxed);
-        per_sm = env_int("HG_ATTN_CTAS_PER_SM", per_sm, 1, per_sm);
+        if (tune.ctas_per_sm >= 1 && tune.ctas_per_sm < per_sm) per_sm = tune.ctas_per_sm;
         const long long slots = (long long)p.NC * Y * p.B;
         const long long resident = (long long)cache.sms[dev].load(std::memory_order_relaxed) * per_sm;
         grid = dim3((unsigned)(slots < resident ? slots : resident), 1, 1);
@@ -162,7 +169,7 @@ static hg_status launch_partial_t(const CUtensorMap& tk, const CUtensorMap& tv, 
         cudaGetLastError();
         return HG_ERR_CUDA;
     }
-    if ((!p.sched || counter_is_zero) && env_int("HG_ATTN_PDL", 1, 0, 1)) {
+    if ((!p.sched || counter_is_zero) && !tune.off(HG_TUNE_NO_PDL)) {
         // no memset sits between this launch and the kernel before it in the stream: launch as a programmatic
         // dependent, so that block scheduling and the input-free part of the set-up overlap that kernel's tail
         p.pdl_wait = 1;
@@ -182,12 +189,12 @@ static hg_status launch_partial_t(const CUtensorMap& tk, const CUtensorMap& tv, 
 
 template <int MODE>
 static hg_status launch_partial_m(int D, bool bf16, const CUtensorMap& tk, const CUtensorMap& tv, const PartialParams& p,
-                                  cudaStream_t st, bool counter_is_zero) {
+                                  cudaStream_t st, bool counter_is_zero, const Tune& tune) {
     if (D == 128)
-        return bf16 ? launch_partial_t<128, true, MODE>(tk, tv, p, st, counter_is_zero)
-                    : launch_partial_t<128, false, MODE>(tk, tv, p, st, counter_is_zero);
-    return bf16 ? launch_partial_t<64, true, MODE>(tk, tv, p, st, counter_is_zero)
-                : launch_partial_t<64, false, MODE>(tk, tv, p, st, counter_is_zero);
+        return bf16 ? launch_partial_t<128, true, MODE>(tk, tv, p, st, counter_is_zero, tune)
+                    : launch_partial_t<128, false, MODE>(tk, tv, p, st, counter_is_zero, tune);
+    return bf16 ? launch_partial_t<64, true, MODE>(tk, tv, p, st, counter_is_zero, tune)
+                : launch_partial_t<64, false, MODE>(tk, tv, p, st, counter_is_zero, tune);
 }
 
 static hg_status run_partial(int mode, const void* q, const void* k, const void* v, const int32_t* seq_lens,
@@ -209,8 +216,9 @@ static hg_status run_partial(int mode, const void* q, const void* k, const void*
     st = make_maps(d, k, v, &tk, &tv);
     if (st != HG_OK) return st;
     const int G = d->num_q_heads / d->num_kv_heads;
+    const Tune tune = desc_tune(d);
     // groups of up to 8 query heads: one MMA head block per item; larger groups: items of 16 heads (two blocks)
-    if (mode != MODE_PROBE) mode = (G == 1) ? MODE_MHA : (G <= 8 || !env_int("HG_ATTN_GQA16", 1, 0, 1) ? MODE_GQA : MODE_GQA2);
+    if (mode != MODE_PROBE) mode = (G == 1) ? MODE_MHA : (G <= 8 || tune.off(HG_TUNE_NO_GQA16) ? MODE_GQA : MODE_GQA2);
     p.q = q; p.seq_lens = seq_lens; p.tok_begin = tok_begin; p.tok_end = tok_end; p.block_table = d->block_table;
     p.o_part = o_part; p.m_part = m_part; p.l_part = l_part; p.sink = sink; p.status = d->status;
     p.B = d->batch; p.Hq = d->num_q_heads; p.Hkv = d->num_kv_heads; p.G = G;
@@ -219,20 +227,20 @@ static hg_status run_partial(int mode, const void* q, const void* k, const void*
     p.head_blocks = (mode == MODE_GQA) ? (G + 7) / 8 : (mode == MODE_GQA2 ? (G + 15) / 16 : 1);
     const float scale = d->scale > 0.f ? d->scale : 1.0f / sqrtf((float)d->head_dim);
     p.scale_log2 = scale * 1.4426950408889634f;
-    p.stages = env_int("HG_ATTN_STAGES", 3, 2, MAX_STAGES);   // 3 x 32 KB of K and V (plus q rows): 2 CTAs per SM
+    p.stages = tune.stages >= 2 ? (tune.stages > MAX_STAGES ? MAX_STAGES : tune.stages) : 3;   // 3 x 32 KB of K and V (plus q rows): 2 CTAs per SM
     // persistent schedule unless the batch or the chunk's page list exceeds what the kernel keeps in shared memory
     p.persistent = (d->batch <= PERSIST_MAX_BATCH && d->chunk_tokens / d->page_size <= PERSIST_CHUNK_PAGES)
-                       ? env_int("HG_ATTN_PERSISTENT", 1, 0, 1) : 0;
+                       ? (tune.off(HG_TUNE_NO_PERSISTENT) ? 0 : 1) : 0;
     p.test_stall = (d->flags & HG_FLAG_TEST_STALL) ? 1 : 0;
     p.sparse_empty = (d->flags & HG_FLAG_SPARSE_EMPTY) ? 1 : 0;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    p.sched = p.persistent && env_int("HG_ATTN_DYNAMIC", 1, 0, 1) ? desc_sched(d) : nullptr;
+    p.sched = p.persistent && !tune.off(HG_TUNE_NO_DYNAMIC) ? desc_sched(d) : nullptr;
     const bool bf16 = d->dtype == HG_DTYPE_BF16;
     switch (mode) {
-        case MODE_MHA: return launch_partial_m<MODE_MHA>(d->head_dim, bf16, tk, tv, p, cs, counter_is_zero);
-        case MODE_GQA: return launch_partial_m<MODE_GQA>(d->head_dim, bf16, tk, tv, p, cs, counter_is_zero);
-        case MODE_GQA2: return launch_partial_m<MODE_GQA2>(d->head_dim, bf16, tk, tv, p, cs, counter_is_zero);
-        default: return launch_partial_m<MODE_PROBE>(d->head_dim, bf16, tk, tv, p, cs, counter_is_zero);
+        case MODE_MHA: return launch_partial_m<MODE_MHA>(d->head_dim, bf16, tk, tv, p, cs, counter_is_zero, tune);
+        case MODE_GQA: return launch_partial_m<MODE_GQA>(d->head_dim, bf16, tk, tv, p, cs, counter_is_zero, tune);
+        case MODE_GQA2: return launch_partial_m<MODE_GQA2>(d->head_dim, bf16, tk, tv, p, cs, counter_is_zero, tune);
+        default: return launch_partial_m<MODE_PROBE>(d->head_dim, bf16, tk, tv, p, cs, counter_is_zero, tune);
     }
 }
 
@@ -254,8 +262,9 @@ static hg_status run_merge(const hg_partial_src* src, int32_t n_src, float* out,
     // long rows and few of them: a cluster of 2, 4 or 8 CTAs splits each row's partials, as long as the grid
     // stays within a few CTAs per SM
     const int rows = d->batch * d->num_q_heads;
+    const Tune tune = desc_tune(d);
     int cluster = 1;
-    if (p.total > 64 && env_int("HG_ATTN_MERGE_CLUSTER", 1, 0, 1)) cluster = rows <= 64 ? 8 : (rows <= 128 ? 4 : (rows <= 256 ? 2 : 1));
+    if (p.total > 64 && !tune.off(HG_TUNE_NO_MERGE_CLUSTER)) cluster = rows <= 64 ? 8 : (rows <= 128 ? 4 : (rows <= 256 ? 2 : 1));
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3((unsigned)(rows * cluster));
@@ -264,7 +273,7 @@ static hg_status run_merge(const hg_partial_src* src, int32_t n_src, float* out,
     cfg.stream = static_cast<cudaStream_t>(stream);
     cudaLaunchAttribute attr[2];
     int na = 0;
-    if (env_int("HG_ATTN_PDL", 1, 0, 1)) {
+    if (!tune.off(HG_TUNE_NO_PDL)) {
         attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[na].val.programmaticStreamSerializationAllowed = 1;     // start while the producer of the partials drains
         ++na;
@@ -280,7 +289,7 @@ static hg_status run_merge(const hg_partial_src* src, int32_t n_src, float* out,
     cudaError_t e;
     // many rows: a warp per row, eight rows per CTA (a warp spends about 0.12 us per non-empty slot, a 1024-thread CTA
     // about 5 us per row whatever it finds: the warp wins from 2048 rows on, and from 1024 when rows are short)
-    if ((rows >= 2048 || (rows >= 1024 && p.total <= 160)) && env_int("HG_ATTN_MERGE_ROWS", 1, 0, 1)) {
+    if ((rows >= 2048 || (rows >= 1024 && p.total <= 160)) && !tune.off(HG_TUNE_NO_MERGE_ROWS)) {
         cfg.gridDim = dim3((unsigned)((rows + 7) / 8));
         cfg.blockDim = dim3(256);
         e = d->head_dim == 128 ? cudaLaunchKernelEx(&cfg, merge_rows_kernel<128>, p, rows)
@@ -493,7 +502,7 @@ hg_status hg_attn_decode_host(const void* q_host, const void* k_cache, const voi
     const int D = desc->head_dim;
     // Fast path when the device can address every host buffer: one kernel stages q and the ranges, the merge
     // reads the host partials and writes the results in place - no copy-engine transfers at all.
-    if (env_int("HG_ATTN_HOST_DIRECT", 1, 0, 1) && rows * D * 2 < (1ull << 32)) {
+    if (!desc_tune(desc).off(HG_TUNE_NO_HOST_DIRECT) && rows * D * 2 < (1ull << 32)) {
         StageParams sp;
         memset(&sp, 0, sizeof sp);
         const void* in[4] = {q_host, seq_lens_host, tok_begin_host, tok_end_host};
@@ -634,7 +643,8 @@ uint32_t hg_version(void) { return HG_VERSION; }
 
 // Scratch for hg_attn_decode_static.  In host code this name is only a handle for the symbol, not a
 // device address: the address is obtained once per device with cudaGetSymbolAddress.
-static __device__ __align__(256) unsigned char hg_static_scratch[HG_STATIC_SCRATCH_BYTES];
+// (the 256 bytes behind the partials hold the partial kernel's work counter)
+static __device__ __align__(256) unsigned char hg_static_scratch[HG_STATIC_SCRATCH_BYTES + 256];
 
 static std::atomic<void*> g_static_scratch_addr[hg::kMaxDevices];
 
@@ -657,9 +667,9 @@ extern "C" hg_status hg_attn_decode_static(const void* q, const void* k_cache, c
     hg_status st = hg::check_desc(desc, true);
     if (st != HG_OK) return st;
     const hg::Workspace w = hg::plan_workspace(desc, 0, 0);
-    if (w.q > HG_STATIC_SCRATCH_BYTES) return HG_ERR_WORKSPACE;     // chunk partials exceed the fixed scratch
+    if (w.sched > HG_STATIC_SCRATCH_BYTES) return HG_ERR_WORKSPACE;     // the three partial arrays exceed the fixed scratch
     void* scratch = static_scratch_ptr();
     if (!scratch) return HG_ERR_CUDA;
     return hg_attn_decode(q, k_cache, v_cache, seq_lens, tok_begin, tok_end, host_partials, n_host_src, out, lse,
-                          scratch, HG_STATIC_SCRATCH_BYTES, stream, desc);
+                          scratch, HG_STATIC_SCRATCH_BYTES + 256, stream, desc);
 }

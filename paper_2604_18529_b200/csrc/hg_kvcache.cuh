@@ -34,7 +34,7 @@ __global__ void kv_append_kernel(KvPoolView pv, const uint16_t* __restrict__ k_n
     const int phys = kv_page_of(pv, b, t);
     __syncthreads();                                   // everybody has read the old length
     if (phys < 0) {
-        if (threadIdx.x == 0 && status) atomicMax(status, HG_DEV_BAD_PAGE);
+        if (threadIdx.x == 0 && status) atomicOr(status, HG_DEV_BAD_PAGE);
         return;
     }
     const int vec_per_row = pv.D / 8;                  // 16-byte vectors
@@ -69,7 +69,7 @@ __global__ void kv_evict_copy_kernel(KvPoolView pv, const int32_t* __restrict__ 
     if ((int)threadIdx.x < i1 - i0) {
         const int phys = kv_page_of(pv, b, tb + i0 + threadIdx.x);
         s_phys[threadIdx.x] = phys;
-        if (phys < 0 && status) atomicMax(status, HG_DEV_BAD_PAGE);
+        if (phys < 0 && status) atomicOr(status, HG_DEV_BAD_PAGE);
     }
     __syncthreads();
     const int n_vec = (i1 - i0) * vec_per_tok;

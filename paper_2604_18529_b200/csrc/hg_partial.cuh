@@ -73,6 +73,8 @@ struct Control {
     uint64_t empty[MAX_STAGES];
     uint64_t cbar;                       // barrier among the consumer warps (one arrival per warp)
     int2 sdesc[MAX_STAGES];              // what a filled stage holds: x = item index (-1: no more work), y = tile in item
+                                         // (low 16 bits) and, above them, one bit per box of the stage's K tiles that
+                                         // was NOT loaded although the item has tokens in it (a bad block-table entry)
     int abort_flag;
     int pages[MAX_CHUNK_PAGES];          // persistent schedule: two buffers, at 0 and at MAX_CHUNK_PAGES / 2
     float red_m[2][64];                  // per-warp running maxima / exp-sums of an item (4 warps x up to 16 heads),
@@ -95,12 +97,23 @@ __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volati
     return __all_sync(0xffffffffu, ok);
 }
 
-// Clamped slice [tb, te) of sequence b and its number of chunk slots in use.
+// Tokens a sequence's row of the block table can address.
+__device__ __forceinline__ int table_reach(const PartialParams& p) {
+    return (int)min((long long)p.max_pages << p.page_shift, (long long)INT32_MAX);
+}
+
+// Clamped slice [tb, te) of sequence b and its number of chunk slots in use.  The slice also ends where the
+// block table's row ends: tokens beyond it have no page to be read from (range_beyond_table() reports them).
 __device__ __forceinline__ int seq_chunks(const PartialParams& p, int b, int& tb, int& te) {
     tb = max(p.tok_begin[b], 0);
-    te = min(p.tok_end[b], p.seq_lens[b]);
+    te = min(min(p.tok_end[b], p.seq_lens[b]), table_reach(p));
     if (te <= tb) return 0;
     return min((te + p.C - 1) / p.C - tb / p.C, p.NC);
+}
+
+// True when sequence b's slice reaches past the last page its block-table row can name.
+__device__ __forceinline__ bool range_beyond_table(const PartialParams& p, int b) {
+    return min(p.tok_end[b], p.seq_lens[b]) > table_reach(p) && max(p.tok_begin[b], 0) < min(p.tok_end[b], p.seq_lens[b]);
 }
 
 __device__ __forceinline__ void set_range(const PartialParams& p, Item& it, int tb, int te) {
@@ -204,7 +217,9 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
         const int per = (p.B + THREADS - 1) / THREADS;
         const int b0 = min(p.B, tid * per), b1 = min(p.B, b0 + per);
         int sum = 0;
-        for (int b = b0; b < b1; ++b) { int tb, te; sum += seq_chunks(p, b, tb, te) * Y; }
+        bool beyond = false;
+        for (int b = b0; b < b1; ++b) { int tb, te; sum += seq_chunks(p, b, tb, te) * Y; beyond |= range_beyond_table(p, b); }
+        if (beyond && p.status && blockIdx.x == 0) atomicOr(p.status, HG_DEV_RANGE);
         int incl = sum;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -232,9 +247,10 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
         // (CTAs beyond the round-robin width, or any CTA when there is no item at all, still help with the empty
         // chunk slots below before they leave)
     } else {
+        if (tid == 0 && blockIdx.x == 0 && blockIdx.y == 0 && p.status && range_beyond_table(p, blockIdx.z)) atomicOr(p.status, HG_DEV_RANGE);
         __syncthreads();
     }
-    if (status_at_entry == HG_DEV_WAIT_TIMEOUT) return;   // checked only now: its load overlapped the scan's loads
+    if (status_at_entry & HG_DEV_WAIT_TIMEOUT) return;   // checked only now: its load overlapped the scan's loads
 
     volatile int* abort_flag = &ctl.abort_flag;
     auto get_item = [&](int i) -> Item {
@@ -302,7 +318,7 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
         auto check_page = [&](int phys) -> int {
             if (phys == -2) return -1;
             if (phys < 0 || phys >= p.num_pages) {
-                if (p.status) atomicMax(p.status, HG_DEV_BAD_PAGE);
+                if (p.status) atomicOr(p.status, HG_DEV_BAD_PAGE);
                 return -1;
             }
             return phys;
@@ -372,10 +388,13 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 int phys = -1;
                 if (sub < SUB && it + sub < cur.ntiles && t0j < cur.hi && t0j + R > cur.lo) phys = pages[(t0j >> p.page_shift) - page0];
                 const uint32_t nvalid = __popc(__ballot_sync(0xffffffffu, phys >= 0));   // K and V boxes
+                // boxes the item has tokens in but whose page id was refused: their rows must not enter the result
+                const bool wanted = sub < SUB && it + sub < cur.ntiles && t0j < cur.hi && t0j + R > cur.lo;
+                const uint32_t missing = __ballot_sync(0xffffffffu, wanted && phys < 0 && !isv) & 0xffffu;
                 // (items of 16 heads fetch their query rows themselves: the stage's q slot holds 8)
                 const uint32_t qbytes = (MODE != MODE_PROBE && NB == 1 && it == 0) ? (uint32_t)q_heads * D * 2u : 0u;
                 if (lane == 0) {
-                    ctl.sdesc[s] = make_int2(i_cur, it);
+                    ctl.sdesc[s] = make_int2(i_cur, it | (int)(missing << 16));
                     if (it == 0) sitem[s] = cur;
                     mbar_arrive_expect_tx(&ctl.full[s], nvalid * box_bytes + qbytes);
                 }
@@ -480,12 +499,19 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
         };
         // Waits for the next filled stage; returns its ring position, or -1 when there is no more work (or the
         // CTA is unwinding).  d receives the stage's descriptor.
+        uint32_t missing = 0u;     // of the stage just received: bit (sub * 2 * boxes per tile + box) = that K/V box is absent
         auto next_stage = [&](int2& d) -> int {
             const int s = cs;
             if (!warp_wait(&ctl.full[s], cph, abort_flag)) return -1;
             if (++cs == p.stages) { cs = 0; cph ^= 1u; }
             d = ctl.sdesc[s];
+            missing = (uint32_t)d.y >> 16;
+            d.y &= 0xffff;
             return d.x < 0 ? -1 : s;
+        };
+        // row r of the stage's tile `sub` sits in a box that was loaded
+        auto row_present = [&](int sub, int r) -> bool {
+            return !((missing >> (sub * (2 * (TILE_T >> rshift)) + (r >> rshift))) & 1u);
         };
 
         Item cur;
@@ -516,7 +542,7 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                     const int idx = u * 32 + lane;
                     const int r = row0 + (idx >> 3) % 16, hh = ((idx >> 3) / 16) % HALVES, kv = (idx >> 3) / (16 * HALVES);
                     const int t = tokbase + r;
-                    if (t >= cur.lo && t < cur.hi) {
+                    if (t >= cur.lo && t < cur.hi && (missing == 0u || row_present(sub, r))) {
                         uint4 v = lds128(base + kv * TILE_BYTES + row_off(r) + hh * half_stride + ((idx & 7) << 4));
                         probe_x ^= v.x ^ v.y ^ v.z ^ v.w;
                     }
@@ -565,7 +591,10 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 const int tokbase = (cur.tile0 + d.y + sub) * TILE_T;
                 bool valid[4];
 #pragma unroll
-                for (int k = 0; k < 4; ++k) { const int t = tokbase + rbase + k; valid[k] = t >= cur.lo && t < cur.hi; }
+                for (int k = 0; k < 4; ++k) {
+                    const int t = tokbase + rbase + k;
+                    valid[k] = t >= cur.lo && t < cur.hi && (missing == 0u || row_present(sub, rbase + k));
+                }
                 const uint32_t kbase = stage0 + s * STAGE_BYTES + sub * PAIR_BYTES, vbase = kbase + TILE_BYTES;
 
                 // ---- K tile: 4 logits per lane group ----
@@ -638,10 +667,11 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                     float M = NEG_INF;
 #pragma unroll
                     for (int sidx = 0; sidx < 16; ++sidx) M = fmaxf(M, ctl.red_m[par][sidx]);
+                    const float Ms = (M == NEG_INF) ? 0.f : M;     // every page of the item refused: an empty partial
                     float accv = 0.f, lsum = 0.f;
 #pragma unroll
                     for (int sidx = 0; sidx < 16; ++sidx) {
-                        const float w = fast_exp2(ctl.red_m[par][sidx] - M);      // -inf states weigh 0; M is finite
+                        const float w = fast_exp2(ctl.red_m[par][sidx] - Ms);     // -inf states weigh 0
                         accv = fmaf(w, *warp_scratch(s, sidx >> 2, (sidx & 3) * D + tid), accv);
                         lsum = fmaf(w, ctl.red_l[par][sidx], lsum);
                     }
@@ -699,8 +729,9 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 for (int sub = 0; sub < SUB && d.y + sub < cur.ntiles; ++sub) {
                 const int tokbase = (cur.tile0 + d.y + sub) * TILE_T;
                 const int tA = tokbase + row0 + quad, tB = tA + 8;
-                const bool vA = tA >= cur.lo && tA < cur.hi, vB = tB >= cur.lo && tB < cur.hi;
-                const bool edge = tokbase < cur.lo || tokbase + TILE_T > cur.hi;
+                const bool vA = tA >= cur.lo && tA < cur.hi && (missing == 0u || row_present(sub, row0 + quad));
+                const bool vB = tB >= cur.lo && tB < cur.hi && (missing == 0u || row_present(sub, row0 + quad + 8));
+                const bool edge = tokbase < cur.lo || tokbase + TILE_T > cur.hi || missing != 0u;
                 wrote |= edge;
                 const uint32_t kbase = stage0 + s * STAGE_BYTES + sub * PAIR_BYTES, vbase = kbase + TILE_BYTES;
 
@@ -758,7 +789,7 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                     for (int u = lane; u < 16 * 8 * HALVES; u += 32) {
                         const int r = row0 + (u / (8 * HALVES)), ch = u % (8 * HALVES);
                         const int t = tokbase + r;
-                        if (t < cur.lo || t >= cur.hi) sts128_zero(vbase + row_off(r) + (ch >> 3) * half_stride + ((ch & 7) << 4));
+                        if (t < cur.lo || t >= cur.hi || !row_present(sub, r)) sts128_zero(vbase + row_off(r) + (ch >> 3) * half_stride + ((ch & 7) << 4));
                     }
                     __syncwarp();
                 }
@@ -811,12 +842,13 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                         float mw[CONSUMER_WARPS], M = NEG_INF, lsum = 0.f;
 #pragma unroll
                         for (int w2 = 0; w2 < CONSUMER_WARPS; ++w2) { mw[w2] = ctl.red_m[par][w2 * HPI + hh]; M = fmaxf(M, mw[w2]); }
+                        const float Ms = (M == NEG_INF) ? 0.f : M;     // every page of the item refused: an empty partial
                         float accv[PER];
 #pragma unroll
                         for (int v = 0; v < PER; ++v) accv[v] = 0.f;
 #pragma unroll
                         for (int w2 = 0; w2 < CONSUMER_WARPS; ++w2) {
-                            const float w = fast_exp2(mw[w2] - M);                 // M is finite: the item has tokens
+                            const float w = fast_exp2(mw[w2] - Ms);
                             lsum = fmaf(w, ctl.red_l[par][w2 * HPI + hh], lsum);
                             const float4* src = reinterpret_cast<const float4*>(warp_scratch(s, w2, hh * D + dbase));
 #pragma unroll
@@ -841,7 +873,7 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
 
     // ---- all roles meet; report a timed-out wait ---------------------------------------------------------
     __syncthreads();
-    if (*abort_flag && p.status && tid == 0) atomicMax(p.status, HG_DEV_WAIT_TIMEOUT);
+    if (*abort_flag && p.status && tid == 0) atomicOr(p.status, HG_DEV_WAIT_TIMEOUT);
 }
 
 }  // namespace hg

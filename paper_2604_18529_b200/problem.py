@@ -34,13 +34,15 @@ class DeviceProblem:
         self.out = torch.empty(B, Hq, D, dtype=torch.float32, device=dev)
         self.lse = torch.empty(B, Hq, dtype=torch.float32, device=dev)
 
-    def make_desc(self, chunk_tokens: int, num_chunks: int, scale: float = 0.0, flags: int = 0):
+    def make_desc(self, chunk_tokens: int, num_chunks: int, scale: float = 0.0, flags: int = 0, tune: int = 0,
+                  tune_stages: int = 0, tune_ctas_per_sm: int = 0):
         w, kv = self.w, self.kv
         return hg.attn_desc(batch=w.B, num_q_heads=w.Hq, num_kv_heads=w.Hkv, head_dim=w.D, dtype=w.dtype,
                             page_size=w.page_size, num_pages=kv["num_pages"], page_stride=kv["page_stride"],
                             head_stride=kv["head_stride"], tok_stride=kv["tok_stride"], block_table=kv["block_table"],
                             max_pages=kv["max_pages"], chunk_tokens=chunk_tokens, num_chunks=num_chunks, scale=scale,
-                            status=self.status, sched_counter=self.sched, flags=flags)
+                            status=self.status, sched_counter=self.sched, flags=flags, tune=tune,
+                            tune_stages=tune_stages, tune_ctas_per_sm=tune_ctas_per_sm)
 
     def partial(self, stream=None):
         hg.hg_attn_partial(self.q, self.kv["k"], self.kv["v"], self.seq_lens, self.tok_begin, self.tok_end,

@@ -51,7 +51,8 @@ def test_desc_struct_matches_the_c_layout():
     f = {n: getattr(hg.HgAttnDesc, n).offset for n, _ in hg.HgAttnDesc._fields_}
     assert f["struct_size"] == 0 and f["num_pages"] == 28 and f["page_stride"] == 32 and f["block_table"] == 56
     assert f["max_pages"] == 64 and f["flags"] == 80 and f["status"] == 88 and f["sched_counter"] == 96
-    assert C.sizeof(hg.HgAttnDesc) == 104
+    assert f["tune"] == 104 and f["tune_stages"] == 108 and f["tune_ctas_per_sm"] == 112
+    assert C.sizeof(hg.HgAttnDesc) == 120
     assert C.sizeof(hg.HgPartialSrc) == 32
 
 
@@ -128,8 +129,11 @@ def test_shorter_struct_without_the_trailing_field_is_accepted(lib):
     d.struct_size = 96                       # a caller compiled before sched_counter existed
     d.sched_counter = 0x3                    # garbage behind the declared size must be ignored
     assert call_partial(lib, d, q=None) == hg.HG_ERR_INVALID_ARG      # gets as far as the pointer checks
-    d.struct_size = 104
+    d.struct_size = 104                      # a caller compiled before the tuning fields existed
     assert call_partial(lib, d) == hg.HG_ERR_INVALID_ARG              # now the misaligned counter is seen
+    d.sched_counter = 0
+    d.tune, d.tune_stages, d.tune_ctas_per_sm = 0xffffffff, 99, -5   # behind the declared size: ignored
+    assert call_partial(lib, d, q=None) == hg.HG_ERR_INVALID_ARG
 
 
 def test_workspace_bytes(lib):

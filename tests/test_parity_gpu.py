@@ -19,10 +19,12 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-def run_and_check(w, poison_tail=False, what=None):
+def run_and_check(w, poison_tail=False, what=None, **tune):
     what = what or w.name
     ref = OracleRef(w)
     prob = DeviceProblem(w, DEV, poison_tail=poison_tail)
+    if tune:
+        prob.desc = prob.make_desc(w.chunk_tokens, prob.NC, **tune)
     prob.partial()
     torch.cuda.synchronize()
     assert int(prob.status.item()) == hg.HG_DEV_OK, what
@@ -212,8 +214,36 @@ def test_decode_and_decode_host_match_partial_plus_merge(G):
     check_output(out_h, lse_h, ref.out, ref.lse)
 
 
+@pytest.mark.parametrize("pinned", [True, False])
+def test_decode_host_with_a_host_source_of_several_partials(pinned):
+    """The workspace is sized by the number of host PARTIALS (the sum of the sources' nc), not of sources: one host
+    source that carries the host-held prefix as three chunk partials needs room for three."""
+    from oracle import hg_oracle as O
+    w = wl(Hq=8, Hkv=2, seq_lens=[900, 411], tok_begin=[300, 130], tok_end=[900, 411])
+    ref = OracleRef(w)
+    prob = DeviceProblem(w, DEV)
+    m, l, o = O.chunked_partials(ref.q, ref.K, ref.V, w.dtype, [0, 0], w.tok_begin, 128, 3)     # prefix in 128-token chunks
+    to = (lambda a: torch.from_numpy(a).float().pin_memory()) if pinned else (lambda a: torch.from_numpy(a).float())
+    host_h = [(to(o), to(m), to(l))]
+    need = pkg.hg_attn_workspace_bytes(prob.desc, 3)
+    assert need > pkg.hg_attn_workspace_bytes(prob.desc, 1)
+    ws = torch.empty(need, dtype=torch.uint8, device=DEV)
+    pin = (lambda t: t.cpu().pin_memory()) if pinned else (lambda t: t.cpu())
+    out_h, lse_h = pin(torch.empty_like(prob.out)), pin(torch.empty_like(prob.lse))
+    pkg.hg_attn_decode_host(pin(prob.q), prob.kv["k"], prob.kv["v"], pin(prob.seq_lens), pin(prob.tok_begin),
+                            pin(prob.tok_end), host_h, out_h, lse_h, ws, prob.desc)
+    torch.cuda.synchronize()
+    check_output(out_h, lse_h, ref.out, ref.lse, "host source with nc = 3")
+    if not pinned:      # the staged form checks the size it was given against what this source needs
+        small = torch.empty(pkg.hg_attn_workspace_bytes(prob.desc, 1), dtype=torch.uint8, device=DEV)
+        with pytest.raises(hg.HgError) as e:
+            pkg.hg_attn_decode_host(pin(prob.q), prob.kv["k"], prob.kv["v"], pin(prob.seq_lens), pin(prob.tok_begin),
+                                    pin(prob.tok_end), host_h, out_h, lse_h, small, prob.desc)
+        assert e.value.status == hg.HG_ERR_WORKSPACE
+
+
 @pytest.mark.parametrize("how", ["pinned", "pageable", "pinned_copies", "mixed", "unaligned"])
-def test_decode_host_paths_agree(how, monkeypatch):
+def test_decode_host_paths_agree(how):
     """Pinned host buffers are read and written by the kernels in place; pageable ones (or a mix, or a
     host partial the merge cannot read with 16-byte loads) go through staged copies.  Same bits either way."""
     w = wl(Hq=8, Hkv=2, seq_lens=[900, 411], tok_begin=[77, 0], tok_end=[900, 300])
@@ -223,7 +253,7 @@ def test_decode_host_paths_agree(how, monkeypatch):
     prob.step(host_dev)
     torch.cuda.synchronize()
     if how == "pinned_copies":
-        monkeypatch.setenv("HG_ATTN_HOST_DIRECT", "0")
+        prob.desc = prob.make_desc(w.chunk_tokens, prob.NC, tune=hg.HG_TUNE_NO_HOST_DIRECT)
     pin = (lambda t: t.cpu()) if how == "pageable" else (lambda t: t.cpu().pin_memory())
     host_h = [tuple(pin(x) for x in src) for src in host_dev]
     if how == "mixed":
@@ -275,34 +305,85 @@ def test_read_probe_checksum_is_the_xor_of_the_slice(layout):
                 assert got[b, g, c] == want, (b, g, c)
 
 
-def test_bad_page_id_is_reported_not_dereferenced():
-    w = wl()
+def partials_over_index_sets(w, prob, keep):
+    """Oracle chunk partials when only the tokens `keep(b, t)` of each slice count."""
+    from oracle import hg_oracle as O
+    q, K, V = bits(w.q()), bits(w.kv_logical("k")), bits(w.kv_logical("v"))
+    NC, D = prob.NC, w.D
+    rm = np.full((w.B, w.Hq, NC), -np.inf); rl = np.zeros((w.B, w.Hq, NC)); ro = np.zeros((w.B, w.Hq, NC, D))
+    for b in range(w.B):
+        for c in range(w.chunk_grid(b)[1]):
+            lo, hi = w.chunk_range(b, c)
+            idx = [t for t in range(lo, hi) if keep(b, t)]
+            for h in range(w.Hq):
+                g = h // w.G
+                rm[b, h, c], rl[b, h, c], ro[b, h, c] = O.partial(q[b, h], np.ascontiguousarray(K[b, :, g]),
+                                                                   np.ascontiguousarray(V[b, :, g]), w.dtype, idx=idx)
+    return rm, rl, ro
+
+
+@pytest.mark.parametrize("G,page", [(1, 16), (4, 16), (1, 64), (8, 32)])
+def test_bad_page_id_is_reported_and_its_tokens_left_out(G, page):
+    """A block-table entry outside the pool is never dereferenced: the call is flagged and the partials are those
+    of the slice without that page's tokens (rows of the box that was not loaded must not leak stale data)."""
+    w = wl(Hq=2 * G, Hkv=2, page_size=page, chunk_tokens=128, seed=90 + G)
     prob = DeviceProblem(w, DEV)
+    # fill the ring with another call first, so that a skipped box would expose stale rows
+    prob.partial()
     table = prob.kv["block_table"].clone()
-    page = w.tok_begin[0] // w.page_size + 3
-    table[0, page] = prob.kv["num_pages"] + 5          # out of range: the kernel must skip it and flag the call
+    bad = w.tok_begin[0] // w.page_size + 3
+    table[0, bad] = prob.kv["num_pages"] + 5
+    whole_chunk = [pg for pg in range(w.max_pages) if pg * page >= 256 and (pg + 1) * page <= 384]   # a chunk with no page left
+    for pg in whole_chunk:
+        table[1, pg] = -7
     prob.kv = dict(prob.kv, block_table=table)
     prob.desc = prob.make_desc(w.chunk_tokens, prob.NC)
     prob.partial()
     torch.cuda.synchronize()
     assert int(prob.status.item()) == hg.HG_DEV_BAD_PAGE
 
+    def keep(b, t):
+        pg = t // page
+        return not ((b == 0 and pg == bad) or (b == 1 and pg in whole_chunk))
+
+    rm, rl, ro = partials_over_index_sets(w, prob, keep)
+    assert np.isinf(rm[1, :, (256 - (w.tok_begin[1] // 128) * 128) // 128]).all()        # that chunk became an empty partial
+    check_partials(prob.o_part.reshape(-1, w.D), prob.m_part.reshape(-1), prob.l_part.reshape(-1),
+                   rm.reshape(-1), rl.reshape(-1), ro.reshape(-1, w.D), "bad page")
+
+
+@pytest.mark.parametrize("G", [1, 4])
+@pytest.mark.parametrize("persistent", [True, False])
+def test_slice_beyond_the_block_table_is_cut_and_reported(G, persistent):
+    """seq_lens and tok_end live on the device, so the host cannot check them against max_pages: a slice that reaches
+    past the table's last page is cut there, the call is flagged, and the partials are those of the cut slice."""
+    w = wl(Hq=2 * G, Hkv=2, seed=95 + G)
+    prob = DeviceProblem(w, DEV)
+    short = 35                                               # pages the table row is cut to: 560 tokens < 700
+    assert short * w.page_size < w.tok_end[0] and short * w.page_size > w.tok_end[1]
+    table = prob.kv["block_table"][:, :short].contiguous()
+    prob.kv = dict(prob.kv, block_table=table, max_pages=short)
+    prob.desc = prob.make_desc(w.chunk_tokens, prob.NC, tune=0 if persistent else hg.HG_TUNE_NO_PERSISTENT)
+    prob.partial()
+    torch.cuda.synchronize()
+    assert int(prob.status.item()) == hg.HG_DEV_RANGE
+    rm, rl, ro = partials_over_index_sets(w, prob, lambda b, t: t < short * w.page_size)
+    check_partials(prob.o_part.reshape(-1, w.D), prob.m_part.reshape(-1), prob.l_part.reshape(-1),
+                   rm.reshape(-1), rl.reshape(-1), ro.reshape(-1, w.D), "beyond table")
+
 
 # ---- schedules: persistent-dynamic, persistent-static and one-CTA-per-item give the same bits --------------------
 
 @pytest.mark.parametrize("G", [1, 4])
-def test_result_does_not_depend_on_the_schedule(G, monkeypatch):
+def test_result_does_not_depend_on_the_schedule(G):
     w = wl(B=3, Hq=2 * G, Hkv=2, seq_lens=[2100, 900, 333], tok_begin=[400, 100, 333], tok_end=[2100, 900, 333],
            chunk_tokens=128)
     ref = OracleRef(w)
     results = []
-    for env in ({}, {"HG_ATTN_DYNAMIC": "0"}, {"HG_ATTN_PERSISTENT": "0"}, {"HG_ATTN_STAGES": "2"},
-                {"HG_ATTN_CTAS_PER_SM": "1", "HG_ATTN_STAGES": "5"}):
-        for k in ("HG_ATTN_DYNAMIC", "HG_ATTN_PERSISTENT", "HG_ATTN_STAGES", "HG_ATTN_CTAS_PER_SM"):
-            monkeypatch.delenv(k, raising=False)
-        for k, v in env.items():
-            monkeypatch.setenv(k, v)
+    for env in ({}, {"tune": hg.HG_TUNE_NO_DYNAMIC}, {"tune": hg.HG_TUNE_NO_PERSISTENT}, {"tune_stages": 2},
+                {"tune_ctas_per_sm": 1, "tune_stages": 5}, {"tune": hg.HG_TUNE_NO_PDL}):
         prob = DeviceProblem(w, DEV)
+        prob.desc = prob.make_desc(w.chunk_tokens, prob.NC, **env)
         prob.step(ref.host_partials_device(DEV))
         torch.cuda.synchronize()
         assert int(prob.status.item()) == hg.HG_DEV_OK
@@ -441,10 +522,9 @@ def test_random_shapes(seed):
 
 @pytest.mark.parametrize("dynamic", ["1", "0"])
 @pytest.mark.parametrize("seed", range(5))
-def test_random_shapes_with_many_items_per_cta(seed, dynamic, monkeypatch):
+def test_random_shapes_with_many_items_per_cta(seed, dynamic):
     """Several hundred to a couple of thousand work items: every resident CTA takes several, so the ring runs
     across item boundaries, the look-ahead of item indices and page ids is in play, and (dynamic) the counter."""
-    monkeypatch.setenv("HG_ATTN_DYNAMIC", dynamic)
     rng = np.random.default_rng(50000 + seed)
     B = int(rng.integers(4, 9))
     Hkv = int(rng.choice([4, 8]))
@@ -459,7 +539,7 @@ def test_random_shapes_with_many_items_per_cta(seed, dynamic, monkeypatch):
     w = W.AttnWorkload(f"many{seed}", B, Hkv * G, Hkv, D, str(rng.choice(["f16", "bf16"])), lens, tb, te, page_size=page,
                        layout=layout, paged=paged, chunk_tokens=chunk, seed=7000 + seed)
     assert sum(w.chunk_grid(b)[1] for b in range(B)) * Hkv > 296
-    run_and_check(w, what=repr(w)[:200])
+    run_and_check(w, what=repr(w)[:200], tune=0 if dynamic == "1" else hg.HG_TUNE_NO_DYNAMIC)
 
 
 # ---- a token set made of several ranges (Section 4.3's position-based choice: sinks + recent window) ----
@@ -545,7 +625,7 @@ def test_prepared_calls_are_the_same_calls():
 
 
 @pytest.mark.parametrize("D,G", [(128, 4), (64, 1)])
-def test_many_short_rows_take_the_warp_per_row_merge(D, G, monkeypatch):
+def test_many_short_rows_take_the_warp_per_row_merge(D, G):
     """A large batch of short sequences: thousands of (sequence, head) rows with a handful of partials each are
     merged a warp per row; same result as the CTA-per-row kernel up to summation order."""
     rng = np.random.default_rng(3)
@@ -558,7 +638,7 @@ def test_many_short_rows_take_the_warp_per_row_merge(D, G, monkeypatch):
     assert w.B * w.Hq >= 2048
     prob, ref, _ = run_and_check(w)
     out_rows, lse_rows = prob.out.clone(), prob.lse.clone()
-    monkeypatch.setenv("HG_ATTN_MERGE_ROWS", "0")
+    prob.desc = prob.make_desc(w.chunk_tokens, prob.NC, tune=hg.HG_TUNE_NO_MERGE_ROWS)
     prob.merge(ref.host_partials_device(DEV))
     torch.cuda.synchronize()
     check_output(prob.out, prob.lse, ref.out, ref.lse, "cta per row")
@@ -567,15 +647,14 @@ def test_many_short_rows_take_the_warp_per_row_merge(D, G, monkeypatch):
 
 
 @pytest.mark.parametrize("G", [9, 12, 16, 24])
-def test_groups_of_more_than_8_heads_either_way(G, monkeypatch):
+def test_groups_of_more_than_8_heads_either_way(G):
     """Groups above 8 query heads run as items of 16 heads (two MMA head blocks sharing every tile read); the
     older form - one item per block of 8 - stays selectable.  Both match the oracle and each other."""
     w = wl(B=2, Hq=G, Hkv=1, D=128, dtype="bf16", seq_lens=[900, 300], tok_begin=[70, 0], tok_end=[900, 217],
            chunk_tokens=256, seed=300 + G, outlier_frac=0.01)
     prob, ref, _ = run_and_check(w)
     a_out, a_o = prob.out.clone(), prob.o_part.clone()
-    monkeypatch.setenv("HG_ATTN_GQA16", "0")
-    prob2, _, _ = run_and_check(w)
+    prob2, _, _ = run_and_check(w, tune=hg.HG_TUNE_NO_GQA16)
     assert (prob2.out - a_out).abs().max().item() <= 1e-5 * max(1.0, a_out.abs().max().item())
     assert (prob2.o_part - a_o).abs().max().item() <= 1e-4 * max(1.0, a_o.abs().max().item())
 
