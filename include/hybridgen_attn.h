@@ -327,6 +327,13 @@ hg_status hg_kv_append(const void* k_new, const void* v_new, void* k_cache, void
  * freed_pages (dev int32 [B][max_freed], -1 padded; n_freed dev int32 [B]; both may be NULL).  The pools are
  * not modified.  desc->block_table is updated in place (it must be writable); with identity paging (NULL)
  * only tok_begin moves.
+ * No page is un-mapped whose id cannot be reported: when freed_pages is given and a sequence would free more
+ * than max_freed pages, its eviction stops at the first page that does not fit the list - tok_begin[b] moves
+ * only to that page's first token and n_freed[b] = max_freed - so read tok_begin back (new minus old) to learn
+ * how many rows of k_out / v_out are valid; max_freed >= max_evict / page_size + 1 never truncates.  With
+ * freed_pages == NULL every emptied page is un-mapped (the caller keeps its own record).  A sequence whose
+ * evicted range meets an unmapped or out-of-pool block-table entry keeps its tok_begin and its block-table
+ * row (its rows of k_out / v_out are unspecified) and *desc->status gets HG_DEV_BAD_PAGE.
  */
 hg_status hg_kv_evict(const void* k_cache, const void* v_cache, int32_t* tok_begin, const int32_t* tok_end,
                       const int32_t* n_evict, int32_t max_evict, void* k_out, void* v_out, int32_t* freed_pages,

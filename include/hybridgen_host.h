@@ -10,6 +10,7 @@
  *   hg_host_gather_logits     the selected tokens' logits out of the full rows
  *   hg_host_select_positions  a Pre-QK^T, position-based selection (Section 4.5): the first `sinks` and the
  *                             last `window` tokens
+ *   hg_host_select_ranked     a Pre-QK^T selection from ranked candidate lists: the first K of each list
  *   hg_host_gather_rows       gathers the selected tokens' V rows into a staging buffer for the transfer
  *   hg_sched_init / _update   the Feedback Scheduler policy (Algorithm 1)
  *   hg_host_tier_*            host memory bound to one NUMA node, the mechanism under the semantic-aware
@@ -37,7 +38,8 @@ typedef struct hg_host_desc {
     int32_t head_dim;       /* D, a multiple of 8 */
     int32_t dtype;          /* hg_dtype */
     int32_t max_selected;   /* K: slots per row in idx / logits */
-    int32_t reserved;
+    int32_t num_rows;       /* token rows per sequence behind k_rows / rows; 0 = not stated (gathers then only
+                               refuse negative indices) */
     int64_t seq_stride;
     int64_t tok_stride;
     int64_t head_stride;
@@ -88,8 +90,21 @@ hg_status hg_host_gather_logits(const float* full, int64_t full_stride, const in
 int32_t hg_host_select_positions(int32_t n_tokens, int32_t sinks, int32_t window, int32_t k, int32_t* idx_out);
 
 /*
+ * Pre-QK^T selection from ranked candidate lists (Section 4.5: any predictor - positions, accumulated scores,
+ * head importance - reduces to a list of host token indices, most important first).  ranking: host int32
+ * [B][Hkv][R], -1 padded at the end.  Every KV head of sequence b takes the first n_out[b] entries of its list,
+ * where n_out[b] = min(k, n_host[b], shortest valid prefix among the sequence's heads) - one count per sequence,
+ * because the hand-off carries one slot count per sequence.  idx_out: host int32 [B][Hkv][k], the entries taken,
+ * then -1.  An entry that is negative or not below n_host[b] ends its list.
+ */
+hg_status hg_host_select_ranked(const int32_t* ranking, int32_t batch, int32_t num_kv_heads, int32_t r,
+                                const int32_t* n_host, int32_t k, int32_t* idx_out, int32_t* n_out);
+
+/*
  * dst[b][g][i][:] = rows[b][idx[b][g][i]][g][:] for i < n_sel[b] (layout of `rows` as in desc); slots beyond
- * n_sel[b] are zero-filled.  dst: host 16-bit [B][Hkv][K][D].
+ * n_sel[b] are zero-filled, and so is a slot whose index is negative (the -1 padding of a selection) or, when
+ * desc->num_rows is stated, not below it: no row outside the caller's buffer is read.
+ * dst: host 16-bit [B][Hkv][K][D].
  */
 hg_status hg_host_gather_rows(const void* rows, const int32_t* idx, const int32_t* n_sel, void* dst,
                               const hg_host_desc* desc);
@@ -126,10 +141,13 @@ typedef struct hg_sched_state {
 void hg_sched_init(hg_sched_state* st, int32_t k_min);
 
 /*
- * One step of the policy on the measured stage latencies (any common unit).  If the CPU stage plus the
- * transfer hides behind the GPU stage (t_cpu + t_tx <= t_gpu) K grows by `step` (up to k_max) - coming
- * from Pre-QK^T the strategy first returns to Post-QK^T; otherwise K shrinks by `step` down to k_min, and at
- * k_min the strategy becomes Pre-QK^T.
+ * One step of the policy on the measured stage latencies (any common unit), branch for branch as
+ * Algorithm 1 lists them.  If the CPU stage plus the transfer hides behind the GPU stage
+ * (t_cpu + t_tx <= t_gpu) K grows by `step` (up to k_max), whichever strategy is in force; otherwise K
+ * shrinks by `step` down to k_min, and at k_min the strategy becomes Pre-QK^T.  No branch sets the
+ * strategy back to Post-QK^T: within a run the switch is one-way (call hg_sched_init to start over), so
+ * latencies that hover around the balance point move K up and down by one step and never flip the
+ * strategy back and forth.
  */
 void hg_sched_update(hg_sched_state* st, double t_gpu, double t_cpu, double t_tx, int32_t k_min, int32_t k_max,
                      int32_t step);

@@ -619,7 +619,7 @@ hg_status hg_kv_evict(const void* k_cache, const void* v_cache, int32_t* tok_beg
                                                 static_cast<uint16_t*>(v_out), max_evict, desc->status);
     if (cudaGetLastError() != cudaSuccess) return HG_ERR_CUDA;
     kv_evict_commit_kernel<<<(desc->batch + 127) / 128, 128, 0, cs>>>(
-        desc->batch, pv.page_shift, desc->max_pages, tok_begin, tok_end, n_evict, max_evict,
+        desc->batch, pv.page_shift, desc->max_pages, desc->num_pages, tok_begin, tok_end, n_evict, max_evict,
         const_cast<int32_t*>(desc->block_table), freed_pages, n_freed, max_freed);
     return cudaGetLastError() == cudaSuccess ? HG_OK : HG_ERR_CUDA;
 }

@@ -435,6 +435,27 @@ int32_t hg_host_select_positions(int32_t n_tokens, int32_t sinks, int32_t window
     return w;
 }
 
+hg_status hg_host_select_ranked(const int32_t* ranking, int32_t batch, int32_t num_kv_heads, int32_t r,
+                                const int32_t* n_host, int32_t k, int32_t* idx_out, int32_t* n_out) {
+    if (!ranking || !n_host || !idx_out || !n_out || batch < 1 || num_kv_heads < 1 || r < 0 || k < 1) return HG_ERR_INVALID_ARG;
+    for (int b = 0; b < batch; ++b) {
+        int n = std::max(0, std::min(k, n_host[b]));
+        for (int g = 0; g < num_kv_heads; ++g) {                // the shortest valid prefix among the heads
+            const int32_t* row = ranking + ((int64_t)b * num_kv_heads + g) * r;
+            int valid = 0;
+            while (valid < r && valid < n && row[valid] >= 0 && row[valid] < n_host[b]) ++valid;
+            n = std::min(n, valid);
+        }
+        for (int g = 0; g < num_kv_heads; ++g) {
+            const int32_t* row = ranking + ((int64_t)b * num_kv_heads + g) * r;
+            int32_t* o = idx_out + ((int64_t)b * num_kv_heads + g) * k;
+            for (int i = 0; i < k; ++i) o[i] = i < n ? row[i] : -1;
+        }
+        n_out[b] = n;
+    }
+    return HG_OK;
+}
+
 hg_status hg_host_gather_rows(const void* rows, const int32_t* idx, const int32_t* n_sel, void* dst, const hg_host_desc* d) {
     if (!desc_ok(d) || !rows || !idx || !n_sel || !dst) return HG_ERR_INVALID_ARG;
     const int D = d->head_dim, K = d->max_selected;
@@ -446,7 +467,10 @@ hg_status hg_host_gather_rows(const void* rows, const int32_t* idx, const int32_
         const int32_t* ix = idx + bg * K;
         uint16_t* o = out + bg * (int64_t)K * D;
         const uint16_t* base = src + (int64_t)b * d->seq_stride + (int64_t)g * d->head_stride;
-        for (int i = 0; i < n; ++i) copy_row(o + (int64_t)i * D, base + (int64_t)ix[i] * d->tok_stride, (size_t)D * 2);
+        for (int i = 0; i < n; ++i) {
+            if (ix[i] >= 0 && (d->num_rows <= 0 || ix[i] < d->num_rows)) copy_row(o + (int64_t)i * D, base + (int64_t)ix[i] * d->tok_stride, (size_t)D * 2);
+            else memset(o + (int64_t)i * D, 0, (size_t)D * 2);       // padding or out of range: nothing is read
+        }
         if (n < K) memset(o + (int64_t)n * D, 0, (size_t)(K - n) * D * 2);
         rows_written();
     });
@@ -539,9 +563,8 @@ void hg_sched_update(hg_sched_state* st, double t_gpu, double t_cpu, double t_tx
     if (!st) return;
     if (step < 1) step = 1;
     if (k_max < k_min) k_max = k_min;
-    if (t_cpu + t_tx <= t_gpu) {                       // the CPU stage is hidden behind the GPU stage
-        if (st->strategy == HG_SCHED_PRE_QK) st->strategy = HG_SCHED_POST_QK;
-        else st->k = std::min(k_max, st->k + step);
+    if (t_cpu + t_tx <= t_gpu) {                       // the CPU stage is hidden behind the GPU stage:
+        st->k = std::min(k_max, st->k + step);         // more tokens, in either selection mode
     } else if (st->k > k_min) {
         st->k = std::max(k_min, st->k - step);
     } else {

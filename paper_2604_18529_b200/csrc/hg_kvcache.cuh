@@ -104,26 +104,36 @@ __global__ void kv_evict_copy_kernel(KvPoolView pv, const int32_t* __restrict__ 
 
 // After the copy: advances tok_begin, un-maps the pages that no longer hold a token of the slice and lists
 // their physical ids in freed [B][max_freed] (-1 padded), n_freed [B].  One thread per sequence.
-__global__ void kv_evict_commit_kernel(int B, int page_shift, int max_pages, int32_t* tok_begin, const int32_t* tok_end,
-                                       const int32_t* n_evict, int max_evict, int32_t* block_table, int32_t* freed,
-                                       int32_t* n_freed, int max_freed) {
+// A page is only un-mapped if its id can be reported: when a freed list is given and fills up, the eviction of
+// that sequence stops at the first page it cannot list (tok_begin goes to that page's first token, which stays
+// resident).  A sequence whose evicted range touches an unmapped or out-of-pool page (the copy kernel flagged
+// it and skipped those rows) keeps its beginning and its table row: no token is lost from both tiers.
+__global__ void kv_evict_commit_kernel(int B, int page_shift, int max_pages, int num_pages, int32_t* tok_begin,
+                                       const int32_t* tok_end, const int32_t* n_evict, int max_evict, int32_t* block_table,
+                                       int32_t* freed, int32_t* n_freed, int max_freed) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
     const int tb = tok_begin[b], te = tok_end[b];
     const int ne = max(0, min(min(n_evict[b], max_evict), te - tb));
-    const int nb = tb + ne;
+    int nb = tb + ne;
     // pages wholly below the new beginning leave; a partly used page stays mapped (it may still take appended rows)
     const int first_pg = tb >> page_shift;
-    const int last_pg = nb >> page_shift;
     int cnt = 0;
+    bool bad = false;
+    if (block_table && ne > 0)
+        for (int pg = first_pg; pg <= ((nb - 1) >> page_shift); ++pg) {
+            const int phys = pg < max_pages ? block_table[(size_t)b * max_pages + pg] : -1;
+            bad |= phys < 0 || phys >= num_pages;
+        }
+    if (bad) nb = tb;
+    const int last_pg = nb >> page_shift;
     for (int pg = first_pg; pg < last_pg && pg < max_pages; ++pg) {
         if (block_table) {
             const int phys = block_table[(size_t)b * max_pages + pg];
-            if (phys >= 0) {
-                if (freed && cnt < max_freed) freed[(size_t)b * max_freed + cnt] = phys;
-                ++cnt;
-                block_table[(size_t)b * max_pages + pg] = -1;
-            }
+            if (freed && cnt == max_freed) { nb = pg << page_shift; break; }     // cannot report it: it stays
+            if (freed) freed[(size_t)b * max_freed + cnt] = phys;
+            ++cnt;
+            block_table[(size_t)b * max_pages + pg] = -1;
         }
     }
     if (freed) for (int i = cnt; i < max_freed; ++i) freed[(size_t)b * max_freed + i] = -1;

@@ -16,7 +16,7 @@ HG_SCHED_POST_QK, HG_SCHED_PRE_QK = 0, 1
 class HgHostDesc(C.Structure):
     _fields_ = [
         ("struct_size", C.c_uint32), ("batch", C.c_int32), ("num_q_heads", C.c_int32), ("num_kv_heads", C.c_int32),
-        ("head_dim", C.c_int32), ("dtype", C.c_int32), ("max_selected", C.c_int32), ("reserved", C.c_int32),
+        ("head_dim", C.c_int32), ("dtype", C.c_int32), ("max_selected", C.c_int32), ("num_rows", C.c_int32),
         ("seq_stride", C.c_int64), ("tok_stride", C.c_int64), ("head_stride", C.c_int64), ("scale", C.c_float),
         ("threads", C.c_int32),
     ]
@@ -44,6 +44,8 @@ def _lib():
         L.hg_host_gather_logits.restype = C.c_int
         L.hg_host_select_positions.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, vp]
         L.hg_host_select_positions.restype = C.c_int32
+        L.hg_host_select_ranked.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, vp, C.c_int32, vp, vp]
+        L.hg_host_select_ranked.restype = C.c_int
         L.hg_host_gather_rows.argtypes = [vp, vp, vp, vp, C.POINTER(HgHostDesc)]
         L.hg_host_gather_rows.restype = C.c_int
         L.hg_host_tier_alloc.argtypes = [C.c_size_t, C.c_int32, C.POINTER(vp)]
@@ -64,13 +66,14 @@ def _lib():
 
 def host_desc(rows: torch.Tensor, num_q_heads: int, max_selected: int, scale: float = 0.0, threads: int = 0) -> HgHostDesc:
     """Describe host rows laid out [B][T][Hkv][D] (any strides with D contiguous)."""
-    B, _, Hkv, D = rows.shape
+    B, T, Hkv, D = rows.shape
     assert rows.stride(3) == 1
     d = HgHostDesc()
     d.struct_size = C.sizeof(HgHostDesc)
     d.batch, d.num_q_heads, d.num_kv_heads, d.head_dim = B, num_q_heads, Hkv, D
     d.dtype = _DTYPES[rows.dtype]
     d.max_selected = max_selected
+    d.num_rows = T
     d.seq_stride, d.tok_stride, d.head_stride = rows.stride(0), rows.stride(1), rows.stride(2)
     d.scale, d.threads = scale, threads
     return d
@@ -119,6 +122,16 @@ def hg_host_select_positions(n_tokens: int, sinks: int, window: int, k: int) -> 
     idx = torch.empty(max(k, 1), dtype=torch.int32)
     n = _lib().hg_host_select_positions(n_tokens, sinks, window, k, idx.data_ptr())
     return idx[:n]
+
+
+def hg_host_select_ranked(ranking: torch.Tensor, n_host: torch.Tensor, k: int):
+    """The first K candidates of each (sequence, KV head) list -> (idx [B][Hkv][k] int32, -1 padded; n [B] int32)."""
+    B, Hkv, R = ranking.shape
+    idx = torch.empty(B, Hkv, k, dtype=torch.int32)
+    n = torch.empty(B, dtype=torch.int32)
+    _check(_lib().hg_host_select_ranked(_host(ranking, "ranking", torch.int32), B, Hkv, R, _host(n_host, "n_host", torch.int32),
+                                        k, idx.data_ptr(), n.data_ptr()), "hg_host_select_ranked")
+    return idx, n
 
 
 def hg_host_gather_rows(rows: torch.Tensor, idx: torch.Tensor, n_sel: torch.Tensor, dst: torch.Tensor, desc: HgHostDesc) -> None:

@@ -125,10 +125,7 @@ class HybridAttentionStep:
             n_pre = n_post.clone()
             pos = torch.full((B, Hkv, k), -1, dtype=torch.int32)
             if self._ranking is not None:
-                # the first K candidates of the caller's list; a sequence offers as many as every one of its heads has
-                take = self._ranking[:, :, :k]
-                pos[:, :, : take.shape[2]] = take
-                n_pre = torch.minimum(n_pre, (take >= 0).sum(dim=2).min(dim=1).values.to(torch.int32))
+                pos, n_pre = H.hg_host_select_ranked(self._ranking, self.n_host, k)      # the first K of the caller's lists
             else:
                 for b in range(B):
                     sel = H.hg_host_select_positions(int(self.n_host[b]), self.sinks, max(k - self.sinks, 0), k)

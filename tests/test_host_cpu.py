@@ -174,6 +174,18 @@ def test_gather_rows():
             assert (dst[b, g, n:] == 0).all()
 
 
+def test_gather_rows_never_reads_outside_the_buffer():
+    """Selections are -1 padded, and a caller may pass a count that reaches into the padding: such slots (and
+    indices at or beyond the stated number of rows) come back as zero rows instead of an out-of-bounds read."""
+    w = W.AttnWorkload("g2", 1, 2, 1, 64, "f16", [40], [0], [40], seed=10)
+    V = w.kv_logical("v")
+    idx = torch.tensor([[[3, -1, 39, 40, 7, 1 << 20]]], dtype=torch.int32)
+    dst = torch.full((1, 1, 6, 64), 1.0, dtype=torch.float16)
+    H.hg_host_gather_rows(V, idx, torch.tensor([6], dtype=torch.int32), dst, H.host_desc(V, 2, 6))
+    assert torch.equal(dst[0, 0, 0], V[0, 3, 0]) and torch.equal(dst[0, 0, 2], V[0, 39, 0]) and torch.equal(dst[0, 0, 4], V[0, 7, 0])
+    assert (dst[0, 0, [1, 3, 5]] == 0).all()
+
+
 def test_feedback_scheduler_follows_algorithm_1():
     rng = np.random.default_rng(11)
     k_min, k_max, step = 128, 1024, 96
@@ -190,10 +202,10 @@ def test_feedback_scheduler_follows_algorithm_1():
     assert s.update(1.0, 0.5, 0.2) == (228, H.HG_SCHED_POST_QK)          # hidden: K grows
     assert s.update(1.0, 0.9, 0.2) == (128, H.HG_SCHED_POST_QK)          # not hidden, K > K_min: shrink, clamped
     assert s.update(1.0, 0.9, 0.2) == (128, H.HG_SCHED_PRE_QK)           # at K_min: switch strategy
-    assert s.update(1.0, 0.5, 0.5) == (128, H.HG_SCHED_POST_QK)          # boundary t_cpu + t_tx == t_gpu counts as hidden
-    for _ in range(20):
+    assert s.update(1.0, 0.5, 0.5) == (228, H.HG_SCHED_PRE_QK)           # boundary t_cpu + t_tx == t_gpu counts as hidden:
+    for _ in range(20):                                                  # K grows, the strategy is not set back
         s.update(1.0, 0.1, 0.1)
-    assert s.state.k == 1024
+    assert (s.state.k, s.state.strategy) == (1024, H.HG_SCHED_PRE_QK)
 
 
 def test_tier_memory_is_bound_to_its_node():
@@ -208,3 +220,22 @@ def test_tier_memory_is_bound_to_its_node():
         H.TierBuffer((16,), torch.float32, node=H.hg_host_tier_nodes() + 500)   # no such node
     with pytest.raises(H.HgError):
         H.TierBuffer((16,), torch.float32, node=-1)
+
+
+def test_ranked_selection_against_the_policy_oracle():
+    rng = np.random.default_rng(21)
+    for _ in range(60):
+        B, Hkv, R = int(rng.integers(1, 4)), int(rng.integers(1, 4)), int(rng.integers(1, 12))
+        n_host = [int(rng.integers(0, 15)) for _ in range(B)]
+        k = int(rng.integers(1, 14))
+        ranking = torch.full((B, Hkv, R), -1, dtype=torch.int32)
+        for b in range(B):
+            for g in range(Hkv):
+                n = int(rng.integers(0, R + 1))
+                ranking[b, g, :n] = torch.from_numpy(rng.integers(0, 16, size=n).astype(np.int32))   # now and then >= n_host
+        idx, n = H.hg_host_select_ranked(ranking, torch.tensor(n_host, dtype=torch.int32), k)
+        for b in range(B):
+            want = P.ranked([ranking[b, g].tolist() for g in range(Hkv)], k, n_host[b])
+            assert int(n[b]) == len(want[0])
+            for g in range(Hkv):
+                assert idx[b, g].tolist() == want[g] + [-1] * (k - len(want[g]))

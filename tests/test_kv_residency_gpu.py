@@ -124,3 +124,51 @@ def test_evicting_more_than_the_slice_empties_it_and_append_needs_a_mapped_page(
     pkg.hg_kv_append(new, new, prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_end, prob.desc)
     torch.cuda.synchronize()
     assert prob.seq_lens.tolist() == [112] and int(prob.status.item()) == hg.HG_DEV_BAD_PAGE
+
+
+def test_a_full_freed_list_stops_the_eviction_instead_of_losing_pages():
+    """Two pages fit the freed list, the request would empty five: the sequence keeps the pages that cannot be
+    reported, its slice then begins at the first of them, and a later call finishes the job."""
+    w = W.AttnWorkload("freed", 2, 2, 2, 64, "f16", [400, 300], [37, 10], [400, 300], page_size=16, chunk_tokens=64, seed=7)
+    prob = DeviceProblem(w, DEV)
+    table0 = prob.kv["block_table"].clone()
+    max_evict, max_freed = 128, 2
+    k_out = torch.zeros(2, max_evict, 2, 64, dtype=torch.float16, device=DEV); v_out = torch.zeros_like(k_out)
+    freed = torch.full((2, max_freed), 77, dtype=torch.int32, device=DEV)
+    n_freed = torch.zeros(2, dtype=torch.int32, device=DEV)
+    ne = torch.tensor([90, 20], dtype=torch.int32, device=DEV)
+    pkg.hg_kv_evict(prob.kv["k"], prob.kv["v"], prob.tok_begin, prob.tok_end, ne, k_out, v_out, freed, n_freed, prob.desc)
+    torch.cuda.synchronize()
+    # sequence 0: [37, 127) would empty pages 2..6 (five); pages 2 and 3 are listed, page 4 cannot be: begin = 64
+    # sequence 1: [10, 30) empties page 0 only (page 1 still holds tokens 30, 31)
+    assert prob.tok_begin.tolist() == [64, 30] and n_freed.tolist() == [2, 1]
+    assert freed[0].tolist() == table0[0, 2:4].tolist() and freed[1].tolist() == [int(table0[1, 0]), -1]
+    assert (prob.kv["block_table"][0, 2:4] == -1).all() and torch.equal(prob.kv["block_table"][0, 4:], table0[0, 4:])
+    assert torch.equal(k_out[0, :27, 1].cpu(), w.kv_rows("k", 0, 1, 37, 64))        # the rows that did leave
+    assert int(prob.status.item()) == hg.HG_DEV_OK
+    # the rest of the request in a second call
+    pkg.hg_kv_evict(prob.kv["k"], prob.kv["v"], prob.tok_begin, prob.tok_end, torch.tensor([63, 0], dtype=torch.int32, device=DEV),
+                    k_out, v_out, freed, n_freed, prob.desc)
+    torch.cuda.synchronize()
+    assert prob.tok_begin.tolist() == [96, 30] and n_freed.tolist() == [2, 0]      # pages 4, 5 listed; page 6 still cannot be
+    after = dataclasses.replace(w, tok_begin=[96, 30])
+    ref = OracleRef(after)
+    prob.step(ref.host_partials_device(DEV))
+    torch.cuda.synchronize()
+    check_output(prob.out, prob.lse, ref.out, ref.lse, "after two truncated evictions")
+
+
+def test_eviction_over_an_unmapped_page_leaves_the_sequence_alone():
+    w = W.AttnWorkload("hole", 2, 2, 2, 64, "f16", [400, 300], [32, 16], [400, 300], page_size=16, chunk_tokens=64, seed=8)
+    prob = DeviceProblem(w, DEV)
+    prob.kv["block_table"][0, 3] = -1                      # a hole inside sequence 0's oldest tokens
+    table0 = prob.kv["block_table"].clone()
+    k_out = torch.zeros(2, 64, 2, 64, dtype=torch.float16, device=DEV); v_out = torch.zeros_like(k_out)
+    freed = torch.full((2, 8), 77, dtype=torch.int32, device=DEV); n_freed = torch.zeros(2, dtype=torch.int32, device=DEV)
+    pkg.hg_kv_evict(prob.kv["k"], prob.kv["v"], prob.tok_begin, prob.tok_end, torch.tensor([48, 48], dtype=torch.int32, device=DEV),
+                    k_out, v_out, freed, n_freed, prob.desc)
+    torch.cuda.synchronize()
+    assert int(prob.status.item()) == hg.HG_DEV_BAD_PAGE
+    assert prob.tok_begin.tolist() == [32, 64] and n_freed.tolist() == [0, 3]
+    assert torch.equal(prob.kv["block_table"][0], table0[0]) and (freed[0] == -1).all()
+    assert torch.equal(k_out[1, :48, 0].cpu(), w.kv_rows("k", 1, 0, 16, 64))
