@@ -367,7 +367,11 @@ def measure_workload(name, args, R, sampler):
     w = W.make_workload(name)
     if args.batch:
         w = W.first_sequences(w, args.batch)
-    prob = DeviceProblem(w, dev)
+    if args.chunk:
+        import dataclasses
+        w = dataclasses.replace(w, chunk_tokens=args.chunk)
+    # (empty chunk slots - a ragged batch has many - get m = -inf and l = 0 only: the merge never reads their o rows)
+    prob = DeviceProblem(w, dev, flags=pkg.binding.HG_FLAG_SPARSE_EMPTY)
     # partials of the host-held slice: produced by the host in the real system; here synthetic values with
     # the statistics of a real partial (they are inputs of the merge, not results of this library)
     gen = torch.Generator(device=dev).manual_seed(w.seed)
@@ -566,6 +570,7 @@ def main():
     ap.add_argument("--repeats", type=int, default=5, help="times the K-step pass is repeated per workload")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=0, help="keep only the first BATCH sequences (small profiling captures)")
+    ap.add_argument("--chunk", type=int, default=0, help="override the workload's chunk_tokens (sweeps)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sharded", action="store_true", help="add the token-sharded record even on one rank")
     ap.add_argument("--probe", action="store_true", help="also time the read-probe kernel")

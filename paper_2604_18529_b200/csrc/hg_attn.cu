@@ -8,6 +8,9 @@
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stddef.h>
+#ifdef HG_TRACE
+#include <stdlib.h>
+#endif
 #include <string.h>
 
 #include <atomic>
@@ -235,6 +238,9 @@ static hg_status run_partial(int mode, const void* q, const void* k, const void*
     p.sparse_empty = (d->flags & HG_FLAG_SPARSE_EMPTY) ? 1 : 0;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     p.sched = p.persistent && !tune.off(HG_TUNE_NO_DYNAMIC) ? desc_sched(d) : nullptr;
+#ifdef HG_TRACE
+    { const char* e = getenv("HG_TRACE_PTR"); p.trace = e ? reinterpret_cast<long long*>(strtoull(e, nullptr, 16)) : nullptr; }
+#endif
     const bool bf16 = d->dtype == HG_DTYPE_BF16;
     switch (mode) {
         case MODE_MHA: return launch_partial_m<MODE_MHA>(d->head_dim, bf16, tk, tv, p, cs, counter_is_zero, tune);

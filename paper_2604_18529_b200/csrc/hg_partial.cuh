@@ -66,7 +66,18 @@ struct PartialParams {
     int pdl_wait;             // launched as a programmatic dependent: wait for the preceding kernel before reading any input
     int32_t* sched;           // zeroed work counter: items are handed out dynamically (NULL: round-robin)
     float scale_log2;         // logit scale * log2(e)
+#ifdef HG_TRACE
+    long long* trace;         // development builds only: 8 timestamps / counters per CTA
+#endif
 };
+
+#ifdef HG_TRACE
+#define HG_TRACE_AT(slot) do { if (p.trace) p.trace[(size_t)blockIdx.x * 8 + (slot)] = (long long)global_timer_ns(); } while (0)
+#define HG_TRACE_SET(slot, v) do { if (p.trace) p.trace[(size_t)blockIdx.x * 8 + (slot)] = (long long)(v); } while (0)
+#else
+#define HG_TRACE_AT(slot) do { } while (0)
+#define HG_TRACE_SET(slot, v) do { } while (0)
+#endif
 
 struct Control {
     uint64_t full[MAX_STAGES];
@@ -124,7 +135,8 @@ __device__ __forceinline__ void set_range(const PartialParams& p, Item& it, int 
     it.ntiles = it.hi > it.lo ? (it.hi + TILE_T - 1) / TILE_T - it.tile0 : 0;
 }
 
-// Item i of the persistent schedule: items are ordered by (b, y, c).  Only the producer decodes (it looks ahead, so the
+// Item i of the persistent schedule: items are ordered by (b, c, y) - within a sequence the KV heads vary fastest - or,
+// for groups of more than 8 query heads, by (b, KV head, c, head block).  Only the producer decodes (it looks ahead, so the
 // three range loads are off the critical path); consumers get the decoded item with the item's first stage.
 __device__ __forceinline__ Item decode_item(const PartialParams& p, const Control& ctl, int i) {
     int lo = 0, hi = p.B;                 // largest b with cum[b] <= i
@@ -138,8 +150,9 @@ __device__ __forceinline__ Item decode_item(const PartialParams& p, const Contro
     const int nc = max(seq_chunks(p, lo, tb, te), 1);
     const int r = i - ctl.cum[lo];
     if (p.head_blocks == 1) {
-        it.y = r / nc;
-        it.c = r - it.y * nc;
+        const int Y = p.Hkv;
+        it.c = r / Y;                     // KV heads vary fastest: CTAs that run side by side read the same pages
+        it.y = r - it.c * Y;
     } else {
         // groups of more than 8 query heads: the head blocks of one (KV head, chunk) sit next to each other in the
         // order, so they are taken at about the same time and the second reader finds part of the tiles in L2
@@ -153,7 +166,7 @@ __device__ __forceinline__ Item decode_item(const PartialParams& p, const Contro
 }
 
 template <int D, bool BF16, int MODE>
-__global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant__ CUtensorMap tmK,
+__global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_constant__ CUtensorMap tmK,
                                                           const __grid_constant__ CUtensorMap tmV,
                                                           const PartialParams p) {
     constexpr int HALVES = D / 64;
@@ -181,6 +194,7 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
 #endif
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int Y = p.Hkv * p.head_blocks;
+    if (tid == 0) HG_TRACE_AT(0);
 
     // ---- set-up that touches no input: barriers, tensor-map prefetch ------------------------------------
     if (tid == CONSUMER_THREADS) {
@@ -251,6 +265,7 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
         __syncthreads();
     }
     if (status_at_entry & HG_DEV_WAIT_TIMEOUT) return;   // checked only now: its load overlapped the scan's loads
+    if (tid == 0) HG_TRACE_AT(1);
 
     volatile int* abort_flag = &ctl.abort_flag;
     auto get_item = [&](int i) -> Item {
@@ -338,6 +353,10 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
         };
         auto settle = [&](int raw) -> int { return dynamic ? __shfl_sync(0xffffffffu, raw, 0) : raw; };
 
+#ifdef HG_TRACE
+        long long trace_wait = 0, trace_look = 0;
+        const long long trace_c0 = clock64();
+#endif
         int s = 0, issued = 0, k = 0;                // ring position, stages armed so far, items taken so far
         uint32_t ph = 0;
         bool alive = true;
@@ -351,6 +370,12 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
             __syncwarp();
         }
         while (i_cur < n_items && alive) {
+#ifdef HG_TRACE
+            if (p.trace && lane == 0 && k < 64) {
+                long long* tl = p.trace + (size_t)gridDim.x * 8 + ((size_t)blockIdx.x * 64 + k) * 2;
+                tl[0] = (long long)global_timer_ns(); tl[1] = issued;
+            }
+#endif
             const int page0 = first_page(cur);
             const int* const pages = &ctl.pages[(k & 1) * (MAX_CHUNK_PAGES / 2)];
             // the next item (its index was requested one item ago) is looked at right after this item's first
@@ -362,6 +387,9 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
             int nxt_ids[PER_LANE];
             int nxt_npages = 0;
             auto look_ahead = [&]() {
+#ifdef HG_TRACE
+                const long long tl0 = clock64();
+#endif
                 i_nxt = settle(raw_nxt);
                 raw_nxt = request(k + 2);
                 has_next = i_nxt < n_items;
@@ -375,13 +403,22 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                         nxt_ids[u] = idx < nxt_npages ? lookup(nxt, np0 + idx) : -2;
                     }
                 }
+#ifdef HG_TRACE
+                trace_look += clock64() - tl0;
+#endif
             };
             const int g = cur.y / p.head_blocks;
             const int q_heads = GQA ? min(HPI, p.G - (cur.y % p.head_blocks) * HPI) : 1;
             const int q_head0 = GQA ? g * p.G + (cur.y % p.head_blocks) * HPI : g;
             for (int it = 0; it < cur.ntiles; it += SUB) {         // one stage = SUB x (K tile + V tile of 64 tokens)
                 int okw = 1;
+#ifdef HG_TRACE
+                const long long tw0 = clock64();
+#endif
                 if (lane == 0) okw = mbar_wait(&ctl.empty[s], ph ^ 1u, abort_flag) ? 1 : 0;
+#ifdef HG_TRACE
+                trace_wait += clock64() - tw0;
+#endif
                 okw = __shfl_sync(0xffffffffu, okw, 0);
                 if (!okw) { alive = false; break; }
                 const int t0j = (cur.tile0 + it + sub) * TILE_T + j * R;
@@ -406,6 +443,7 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                     uint8_t* dst = stage0_ptr + (size_t)s * STAGE_BYTES + sub * PAIR_BYTES + isv * TILE_BYTES + j * box_bytes;
                     tma_load_5d(dst, isv ? &tmV : &tmK, &ctl.full[s], 0, t0j & (p.page_size - 1), 0, g, phys, policy);
                 }
+                if (issued == 0 && lane == 0) HG_TRACE_AT(2);
                 ++issued;
                 if (++s == p.stages) { s = 0; ph ^= 1u; }
                 if (it == 0) look_ahead();
@@ -424,6 +462,13 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
             i_cur = i_nxt;
             ++k;
         }
+#ifdef HG_TRACE
+        if (lane == 0 && p.trace) {
+            HG_TRACE_AT(5); HG_TRACE_SET(6, k + 1); HG_TRACE_SET(7, issued);
+            long long* ex = p.trace + (size_t)gridDim.x * 8 + (size_t)gridDim.x * 128 + (size_t)blockIdx.x * 8;
+            ex[0] = trace_wait; ex[1] = clock64() - trace_c0; ex[7] = trace_look;
+        }
+#endif
         if (alive && !p.test_stall) {
             // no more work: one last, empty stage tells the consumers
             int okw = 1;
@@ -444,28 +489,24 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
     } else {
         // =============================== consumer warps ===============================
         if (p.persistent) {
-            // empty chunk slots (c >= nc_b): neutral elements, spread over all CTAs; the consumer warps write them
-            // while the first stage is on its way
-            for (int sl = blockIdx.x; sl < p.B * Y; sl += gridDim.x) {
-                const int b = sl / Y, y = sl - b * Y;
+            // Empty chunk slots (c >= nc_b) get neutral elements while the first stage is on its way.  The empty
+            // slots of one (sequence, head) row are contiguous in all three arrays, so a row is one warp's job: rows
+            // are dealt round-robin to the consumer warps of the whole grid and written with full-width stores.
+            const int NW = (int)gridDim.x * CONSUMER_WARPS, wg = (int)blockIdx.x * CONSUMER_WARPS + warp;
+            const int rows_per_seq = MODE == MODE_PROBE ? p.Hkv : p.Hq;
+            for (int r = wg; r < p.B * rows_per_seq; r += NW) {
+                const int b = r / rows_per_seq;
                 const int nc = (ctl.cum[b + 1] - ctl.cum[b]) / Y;
-                const int ne = p.NC - nc;                 // empty slots per head
+                const int ne = p.NC - nc;                 // empty slots of this row
                 if (ne <= 0) continue;
+                const size_t first = (size_t)r * p.NC + nc;
                 if constexpr (MODE == MODE_PROBE) {
-                    for (int i = tid; i < ne; i += CONSUMER_THREADS) p.sink[((size_t)b * p.Hkv + y) * p.NC + nc + i] = 0u;
+                    for (int i = lane; i < ne; i += 32) p.sink[first + i] = 0u;
                 } else {
-                    const int hb = y % p.head_blocks, g = y / p.head_blocks;
-                    const int nh = GQA ? min(HPI, p.G - hb * HPI) : 1;
-                    const int hq0 = GQA ? g * p.G + hb * HPI : g;
-                    if (!p.sparse_empty)
-                        for (int i = tid; i < nh * ne * D; i += CONSUMER_THREADS) {
-                            const int e = i / D, hh = e / ne, cc = nc + e % ne;
-                            p.o_part[(((size_t)b * p.Hq + hq0 + hh) * p.NC + cc) * D + i % D] = 0.f;
-                        }
-                    for (int i = tid; i < nh * ne; i += CONSUMER_THREADS) {
-                        const int hh = i / ne, cc = nc + i % ne;
-                        p.m_part[((size_t)b * p.Hq + hq0 + hh) * p.NC + cc] = NEG_INF;
-                        p.l_part[((size_t)b * p.Hq + hq0 + hh) * p.NC + cc] = 0.f;
+                    for (int i = lane; i < ne; i += 32) { p.m_part[first + i] = NEG_INF; p.l_part[first + i] = 0.f; }
+                    if (!p.sparse_empty) {
+                        float4* o4 = reinterpret_cast<float4*>(p.o_part + first * D);
+                        for (int i = lane; i < ne * (D / 4); i += 32) o4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
                     }
                 }
             }
@@ -499,10 +540,22 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
         };
         // Waits for the next filled stage; returns its ring position, or -1 when there is no more work (or the
         // CTA is unwinding).  d receives the stage's descriptor.
+#ifdef HG_TRACE
+        bool traced_first = false;
+        long long ctrace_wait = 0, ctrace_c0 = 0, ctrace_epi = 0, ctrace_sync = 0, ctrace_begin = 0;
+#endif
         uint32_t missing = 0u;     // of the stage just received: bit (sub * 2 * boxes per tile + box) = that K/V box is absent
         auto next_stage = [&](int2& d) -> int {
             const int s = cs;
+#ifdef HG_TRACE
+            const long long tw0 = clock64();
+#endif
             if (!warp_wait(&ctl.full[s], cph, abort_flag)) return -1;
+#ifdef HG_TRACE
+            if (traced_first) ctrace_wait += clock64() - tw0;
+            if (tid == 0 && !traced_first) { HG_TRACE_AT(3); }
+            if (!traced_first) { traced_first = true; ctrace_c0 = clock64(); }
+#endif
             if (++cs == p.stages) { cs = 0; cph ^= 1u; }
             d = ctl.sdesc[s];
             missing = (uint32_t)d.y >> 16;
@@ -697,6 +750,9 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 int2 d;
                 const int s = next_stage(d);
                 if (s < 0) break;
+#ifdef HG_TRACE
+                const long long tb0 = clock64();
+#endif
                 if (d.y == 0) {
                     begin_item(s);
                     // b0 = q[head quad][16 ks + 2 tq + {0,1}], b1 = the same + 8; heads past the group read as zero
@@ -725,6 +781,9 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                         for (int u = 0; u < KSTEPS; ++u) { oacc[nb][u][0] = oacc[nb][u][1] = oacc[nb][u][2] = oacc[nb][u][3] = 0.f; }
                     }
                 }
+#ifdef HG_TRACE
+                ctrace_begin += clock64() - tb0;
+#endif
                 bool wrote = false;
                 for (int sub = 0; sub < SUB && d.y + sub < cur.ntiles; ++sub) {
                 const int tokbase = (cur.tile0 + d.y + sub) * TILE_T;
@@ -735,20 +794,58 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 wrote |= edge;
                 const uint32_t kbase = stage0 + s * STAGE_BYTES + sub * PAIR_BYTES, vbase = kbase + TILE_BYTES;
 
+                if (edge) {
+                    // rows outside the slice may hold anything (even NaN patterns): clear this warp's copies in the V tile
+                    for (int u = lane; u < 16 * 8 * HALVES; u += 32) {
+                        const int r = row0 + (u / (8 * HALVES)), ch = u % (8 * HALVES);
+                        const int t = tokbase + r;
+                        if (t < cur.lo || t >= cur.hi || !row_present(sub, r)) sts128_zero(vbase + row_off(r) + (ch >> 3) * half_stride + ((ch & 7) << 4));
+                    }
+                    __syncwarp();
+                }
+
                 // ---- S^T (16 tokens x 8 heads per block) ----
+                // One head block: all fragment loads are issued before the first MMA, the products accumulate in two
+                // independent chains, and the V fragments are requested before the softmax arithmetic, so that the
+                // warp (the only one of its CTA on its scheduler) is not held up by one dependent instruction after
+                // the other.  Two head blocks already give two independent chains and have no registers to spare.
                 float sc[NB][4];
+                uint32_t va[NB == 1 ? KSTEPS : 1][4];
+                if constexpr (NB == 1) {
+                    uint32_t ka[KSTEPS][4];
 #pragma unroll
-                for (int nb = 0; nb < NB; ++nb) sc[nb][0] = sc[nb][1] = sc[nb][2] = sc[nb][3] = 0.f;
+                    for (int ks = 0; ks < KSTEPS; ++ks) {
+                        const int ch = 2 * ks + a_kc;   // 16-byte chunk index along d
+                        ldmatrix_x4(ka[ks], kbase + a_off + (ch >> 3) * half_stride + (((ch & 7) ^ (a_row & 7)) << 4));
+                    }
+                    float se[4] = {0.f, 0.f, 0.f, 0.f}, so[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int ks = 0; ks < KSTEPS; ++ks) {
-                    const int ch = 2 * ks + a_kc;   // 16-byte chunk index along d
-                    uint32_t a[4];
-                    ldmatrix_x4(a, kbase + a_off + (ch >> 3) * half_stride + (((ch & 7) ^ (a_row & 7)) << 4));
+                    for (int ks = 0; ks < KSTEPS; ks += 2) {
+                        mma_16816<BF16>(se, ka[ks], qb[0][ks][0], qb[0][ks][1]);
+                        mma_16816<BF16>(so, ka[ks + 1], qb[0][ks + 1][0], qb[0][ks + 1][1]);
+                    }
 #pragma unroll
-                    for (int nb = 0; nb < NB; ++nb) mma_16816<BF16>(sc[nb], a, qb[nb][ks][0], qb[nb][ks][1]);
+                    for (int mt = 0; mt < KSTEPS; ++mt) {
+                        const int ch = 2 * mt + v_dc;
+                        ldmatrix_x4_trans(va[mt], vbase + v_off + (ch >> 3) * half_stride + (((ch & 7) ^ (v_row & 7)) << 4));
+                    }
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) sc[0][i] = se[i] + so[i];
+                } else {
+#pragma unroll
+                    for (int nb = 0; nb < NB; ++nb) sc[nb][0] = sc[nb][1] = sc[nb][2] = sc[nb][3] = 0.f;
+#pragma unroll
+                    for (int ks = 0; ks < KSTEPS; ++ks) {
+                        const int ch = 2 * ks + a_kc;
+                        uint32_t a[4];
+                        ldmatrix_x4(a, kbase + a_off + (ch >> 3) * half_stride + (((ch & 7) ^ (a_row & 7)) << 4));
+#pragma unroll
+                        for (int nb = 0; nb < NB; ++nb) mma_16816<BF16>(sc[nb], a, qb[nb][ks][0], qb[nb][ks][1]);
+                    }
                 }
                 float corr[NB][2];
                 uint32_t bh0[NB], bh1[NB], bl0[NB], bl1[NB];
+                bool moved = false;              // some running maximum of this lane grew: the accumulators need rescaling
 #pragma unroll
                 for (int nb = 0; nb < NB; ++nb) {
                     // sc[0], sc[1]: token tA, heads 2tq, 2tq+1 of the block; sc[2], sc[3]: token tB
@@ -766,7 +863,9 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                     for (int hc = 0; hc < 2; ++hc) {
                         const float m_new = fmaxf(m_run[nb][hc], mx[hc]);
                         msafe[hc] = (m_new == NEG_INF) ? 0.f : m_new;
-                        corr[nb][hc] = fast_exp2(m_run[nb][hc] - msafe[hc]);
+                        const bool same = m_new == m_run[nb][hc];
+                        corr[nb][hc] = same ? 1.f : fast_exp2(m_run[nb][hc] - msafe[hc]);
+                        moved |= !same;
                         m_run[nb][hc] = m_new;
                     }
                     float pr[4];
@@ -784,32 +883,39 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                 }
 
                 // ---- O^T ----
-                if (edge) {
-                    // rows outside the slice may hold anything (even NaN patterns): clear this warp's copies
-                    for (int u = lane; u < 16 * 8 * HALVES; u += 32) {
-                        const int r = row0 + (u / (8 * HALVES)), ch = u % (8 * HALVES);
-                        const int t = tokbase + r;
-                        if (t < cur.lo || t >= cur.hi || !row_present(sub, r)) sts128_zero(vbase + row_off(r) + (ch >> 3) * half_stride + ((ch & 7) << 4));
-                    }
-                    __syncwarp();
+                // the running maxima settle after an item's first tiles: most tiles need no rescaling at all
+                if (__any_sync(0xffffffffu, moved)) {
+#pragma unroll
+                    for (int nb = 0; nb < NB; ++nb)
+#pragma unroll
+                        for (int mt = 0; mt < KSTEPS; ++mt) {
+                            oacc[nb][mt][0] *= corr[nb][0]; oacc[nb][mt][1] *= corr[nb][1];
+                            oacc[nb][mt][2] *= corr[nb][0]; oacc[nb][mt][3] *= corr[nb][1];
+                        }
                 }
+                if constexpr (NB == 1) {
 #pragma unroll
-                for (int mt = 0; mt < KSTEPS; ++mt) {
-                    const int ch = 2 * mt + v_dc;
-                    uint32_t a[4];
-                    ldmatrix_x4_trans(a, vbase + v_off + (ch >> 3) * half_stride + (((ch & 7) ^ (v_row & 7)) << 4));
+                    for (int mt = 0; mt < KSTEPS; ++mt) mma_16816<BF16>(oacc[0][mt], va[mt], bh0[0], bh1[0]);
 #pragma unroll
-                    for (int nb = 0; nb < NB; ++nb) {
-                        oacc[nb][mt][0] *= corr[nb][0]; oacc[nb][mt][1] *= corr[nb][1];
-                        oacc[nb][mt][2] *= corr[nb][0]; oacc[nb][mt][3] *= corr[nb][1];
-                        mma_16816<BF16>(oacc[nb][mt], a, bh0[nb], bh1[nb]);
-                        mma_16816<BF16>(oacc[nb][mt], a, bl0[nb], bl1[nb]);
+                    for (int mt = 0; mt < KSTEPS; ++mt) mma_16816<BF16>(oacc[0][mt], va[mt], bl0[0], bl1[0]);
+                } else {
+#pragma unroll
+                    for (int mt = 0; mt < KSTEPS; ++mt) {
+                        const int ch = 2 * mt + v_dc;
+                        ldmatrix_x4_trans(va[0], vbase + v_off + (ch >> 3) * half_stride + (((ch & 7) ^ (v_row & 7)) << 4));
+#pragma unroll
+                        for (int nb = 0; nb < NB; ++nb) mma_16816<BF16>(oacc[nb][mt], va[0], bh0[nb], bh1[nb]);
+#pragma unroll
+                        for (int nb = 0; nb < NB; ++nb) mma_16816<BF16>(oacc[nb][mt], va[0], bl0[nb], bl1[nb]);
                     }
                 }
                 }
                 if (d.y + SUB < cur.ntiles) { release(s, wrote); continue; }
 
                 // ---- item epilogue: merge the 4 warp states (the item's last stage is the scratch) ----
+#ifdef HG_TRACE
+                const long long te0 = clock64();
+#endif
 #pragma unroll
                 for (int nb = 0; nb < NB; ++nb) {
 #pragma unroll
@@ -832,7 +938,13 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                         lane_base[D + mt * 16 + 8] = oacc[nb][mt][3];
                     }
                 }
+#ifdef HG_TRACE
+                const long long ts0 = clock64();
+#endif
                 if (!consumer_sync()) break;
+#ifdef HG_TRACE
+                ctrace_sync += clock64() - ts0;
+#endif
                 // thread -> (head, D/16 consecutive components): the four warp states of one head, weighted
 #pragma unroll
                 for (int nb = 0; nb < NB; ++nb) {
@@ -867,12 +979,22 @@ __global__ void __launch_bounds__(THREADS) partial_kernel(const __grid_constant_
                     }
                 }
                 release(s, true);
+#ifdef HG_TRACE
+                ctrace_epi += clock64() - te0;
+#endif
             }
         }
+#ifdef HG_TRACE
+        if (tid == 0 && p.trace) {
+            long long* ex = p.trace + (size_t)gridDim.x * 8 + (size_t)gridDim.x * 128 + (size_t)blockIdx.x * 8;
+            ex[2] = ctrace_wait; ex[3] = clock64() - ctrace_c0; ex[4] = ctrace_epi; ex[5] = ctrace_sync; ex[6] = ctrace_begin;
+        }
+#endif
     }
 
     // ---- all roles meet; report a timed-out wait ---------------------------------------------------------
     __syncthreads();
+    if (tid == 0) HG_TRACE_AT(4);
     if (*abort_flag && p.status && tid == 0) atomicOr(p.status, HG_DEV_WAIT_TIMEOUT);
 }
 

@@ -14,7 +14,8 @@ from .workload import AttnWorkload
 
 
 class DeviceProblem:
-    def __init__(self, w: AttnWorkload, device="cuda:0", poison_tail: bool = False, kv: Optional[dict] = None):
+    def __init__(self, w: AttnWorkload, device="cuda:0", poison_tail: bool = False, kv: Optional[dict] = None,
+                 flags: int = 0):
         self.w = w
         self.device = torch.device(device)
         dev = self.device
@@ -26,7 +27,7 @@ class DeviceProblem:
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         self.sched = torch.zeros(1, dtype=torch.int32, device=dev)
         self.NC = w.num_chunks
-        self.desc = self.make_desc(w.chunk_tokens, self.NC)
+        self.desc = self.make_desc(w.chunk_tokens, self.NC, flags=flags)
         B, Hq, D, NC = w.B, w.Hq, w.D, self.NC
         self.o_part = torch.empty(B, Hq, NC, D, dtype=torch.float32, device=dev)
         self.m_part = torch.empty(B, Hq, NC, dtype=torch.float32, device=dev)
