@@ -307,6 +307,38 @@ def time_extras(w, prob, dev, steps):
     restore_only()
     moved = 2 * 2 * w.B * max_evict * w.Hkv * w.D * 2                 # K and V, read + written
     out["kv_evict"] = {"tokens_per_seq": max_evict, "us": us, "gbs": moved / us / 1e3}
+    # ---- the same eviction with the step's attention: in front of it on one stream, and beside it (three-step form:
+    #      begin on the attention's stream, row copy + device -> host copies + un-mapping on a second stream)
+    kh = torch.empty(k_out.shape, dtype=dt).pin_memory(); vh = torch.empty_like(kh).pin_memory()
+    src_begin = torch.empty(w.B, dtype=torch.int32, device=dev); n_moved = torch.empty_like(src_begin)
+    side = torch.cuda.Stream(device=dev)
+    main = torch.cuda.current_stream(dev)
+    step = prob.prepare_step([prob.empty_host_partial()])
+
+    def serial():
+        restore_only()
+        pkg.hg_kv_evict(prob.kv["k"], prob.kv["v"], prob.tok_begin, prob.tok_end, ne, k_out, v_out, None, None, prob.desc)
+        kh.copy_(k_out, non_blocking=True); vh.copy_(v_out, non_blocking=True)
+        step()
+
+    def beside():
+        restore_only()
+        pkg.hg_kv_evict_begin(prob.tok_begin, prob.tok_end, ne, max_evict, 0, src_begin, n_moved, prob.desc)
+        ev = torch.cuda.Event(); ev.record(main)
+        with torch.cuda.stream(side):
+            side.wait_event(ev)
+            pkg.hg_kv_evict_copy(prob.kv["k"], prob.kv["v"], src_begin, n_moved, k_out, v_out, prob.desc, side)
+            kh.copy_(k_out, non_blocking=True); vh.copy_(v_out, non_blocking=True)
+            pkg.hg_kv_evict_finish(src_begin, n_moved, None, None, prob.desc, side)
+            fin = torch.cuda.Event(); fin.record(side)
+        step()
+        main.wait_event(fin)                  # the timed region ends when both the attention and the eviction are done
+
+    base = dev_us(restore_only, steps)
+    out["evict_with_attention"] = {"tokens_per_seq": max_evict, "d2h_bytes": 2 * kh.numel() * 2,
+                                   "in_front_us": dev_us(serial, steps) - base, "beside_us": dev_us(beside, steps) - base,
+                                   "attention_alone_us": dev_us(step, steps)}
+    restore_only()
     return out
 
 

@@ -340,6 +340,39 @@ hg_status hg_kv_evict(const void* k_cache, const void* v_cache, int32_t* tok_beg
                       int32_t* n_freed, int32_t max_freed, void* stream, const hg_attn_desc* desc);
 
 /*
+ * hg_kv_evict in three steps, for an eviction that drains BESIDE the attention of the same decode step instead
+ * of in front of it (Section 4.2, device-side support: the Eviction Engine works under memory pressure while
+ * decoding goes on; the Token Mapper's ranges are what keeps both sides consistent).
+ *
+ *   hg_kv_evict_begin   on the attention's stream, before it: decides for every sequence the rows that leave
+ *                       (the rule of hg_kv_evict, including its two cut-backs; pass the max_freed that
+ *                       hg_kv_evict_finish will be given, 0 if no list is wanted), records them in
+ *                       src_begin[b] (the old beginning) and n_moved[b] (dev int32 [B] each) and advances
+ *                       tok_begin.  The block table is not touched.  Everything enqueued on this stream afterwards -
+ *                       hg_attn_partial, hg_attn_decode - works on the shrunk slice [tok_begin, tok_end).
+ *   hg_kv_evict_copy    on a second stream, after an event recorded behind step 1: copies the recorded rows to
+ *                       k_out / v_out (layout as in hg_kv_evict; rows beyond n_moved[b] are left alone).  It only
+ *                       reads the pools and block-table entries of the rows that leave.
+ *   hg_kv_evict_finish  behind the copy (same second stream, or any stream ordered after it): un-maps the pages
+ *                       that lie wholly below the new beginning and lists them, as hg_kv_evict does.
+ *
+ * Why nothing races: attention over the shrunk slice looks up block-table entries only from tok_begin's page on,
+ * and step 3 writes only entries of pages wholly below it - the two never touch the same entry, so step 3 needs
+ * no ordering against the attention that runs beside it; the page that holds the new beginning stays mapped and
+ * is only read by both.  Attention launched BEFORE step 1 (the previous decode step, over the old range) does read
+ * the entries step 3 clears: step 1 sits behind it in stream order and steps 2 and 3 wait for step 1's event, which
+ * orders them.  A freed page may be handed out again only once step 3 has completed (wait for its stream or an
+ * event behind it); until then the rows are still being read.  Results are those of hg_kv_evict, bit for bit.
+ */
+hg_status hg_kv_evict_begin(int32_t* tok_begin, const int32_t* tok_end, const int32_t* n_evict, int32_t max_evict,
+                            int32_t max_freed, int32_t* src_begin, int32_t* n_moved, void* stream,
+                            const hg_attn_desc* desc);
+hg_status hg_kv_evict_copy(const void* k_cache, const void* v_cache, const int32_t* src_begin, const int32_t* n_moved,
+                           int32_t max_evict, void* k_out, void* v_out, void* stream, const hg_attn_desc* desc);
+hg_status hg_kv_evict_finish(const int32_t* src_begin, const int32_t* n_moved, int32_t* freed_pages, int32_t* n_freed,
+                             int32_t max_freed, void* stream, const hg_attn_desc* desc);
+
+/*
  * Evidence kernel, not part of the attention path: streams the same K and V tiles through the
  * same TMA pipeline as hg_attn_partial and folds them into one 32-bit checksum per work item
  * (sink: dev uint32 [B][Hkv][NC]).  Used to measure the read ceiling of the paged access pattern.

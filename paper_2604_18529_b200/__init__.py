@@ -27,5 +27,8 @@ from .binding import (  # noqa: F401
     hg_kv_read_probe,
     hg_kv_append,
     hg_kv_evict,
+    hg_kv_evict_begin,
+    hg_kv_evict_copy,
+    hg_kv_evict_finish,
     hg_version,
 )

@@ -111,6 +111,12 @@ def lib():
         L.hg_kv_append.restype = C.c_int
         L.hg_kv_evict.argtypes = [vp] * 5 + [i32, vp, vp, vp, vp, i32, vp, C.POINTER(HgAttnDesc)]
         L.hg_kv_evict.restype = C.c_int
+        L.hg_kv_evict_begin.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, C.POINTER(HgAttnDesc)]
+        L.hg_kv_evict_begin.restype = C.c_int
+        L.hg_kv_evict_copy.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, C.POINTER(HgAttnDesc)]
+        L.hg_kv_evict_copy.restype = C.c_int
+        L.hg_kv_evict_finish.argtypes = [vp, vp, vp, vp, i32, vp, C.POINTER(HgAttnDesc)]
+        L.hg_kv_evict_finish.restype = C.c_int
         L.hg_kv_read_probe.argtypes = [vp] * 7 + [C.POINTER(HgAttnDesc)]
         L.hg_kv_read_probe.restype = C.c_int
         L.hg_status_string.argtypes = [C.c_int]
@@ -367,6 +373,32 @@ def hg_kv_evict(k_cache, v_cache, tok_begin, tok_end, n_evict, k_out, v_out, fre
                            _dev(n_freed, "n_freed", torch.int32), 0 if freed_pages is None else freed_pages.shape[1],
                            _stream(stream), C.byref(desc))
     _check(st, "hg_kv_evict")
+
+
+def hg_kv_evict_begin(tok_begin, tok_end, n_evict, max_evict: int, max_freed: int, src_begin, n_moved, desc: HgAttnDesc,
+                      stream=None) -> None:
+    """Step 1 of an eviction that drains beside the attention: decide and record the rows that leave, advance tok_begin."""
+    st = lib().hg_kv_evict_begin(_dev(tok_begin, "tok_begin", torch.int32), _dev(tok_end, "tok_end", torch.int32),
+                                 _dev(n_evict, "n_evict", torch.int32), max_evict, max_freed,
+                                 _dev(src_begin, "src_begin", torch.int32), _dev(n_moved, "n_moved", torch.int32),
+                                 _stream(stream), C.byref(desc))
+    _check(st, "hg_kv_evict_begin")
+
+
+def hg_kv_evict_copy(k_cache, v_cache, src_begin, n_moved, k_out, v_out, desc: HgAttnDesc, stream=None) -> None:
+    """Step 2: copy the recorded rows to k_out / v_out [B][max_evict][Hkv][D] (reads only)."""
+    st = lib().hg_kv_evict_copy(_dev(k_cache, "k_cache"), _dev(v_cache, "v_cache"), _dev(src_begin, "src_begin", torch.int32),
+                                _dev(n_moved, "n_moved", torch.int32), k_out.shape[1], _dev(k_out, "k_out"),
+                                _dev(v_out, "v_out"), _stream(stream), C.byref(desc))
+    _check(st, "hg_kv_evict_copy")
+
+
+def hg_kv_evict_finish(src_begin, n_moved, freed_pages, n_freed, desc: HgAttnDesc, stream=None) -> None:
+    """Step 3: un-map and list the pages that lie wholly below the new beginning."""
+    st = lib().hg_kv_evict_finish(_dev(src_begin, "src_begin", torch.int32), _dev(n_moved, "n_moved", torch.int32),
+                                  _dev(freed_pages, "freed_pages", torch.int32), _dev(n_freed, "n_freed", torch.int32),
+                                  0 if freed_pages is None else freed_pages.shape[1], _stream(stream), C.byref(desc))
+    _check(st, "hg_kv_evict_finish")
 
 
 def hg_kv_read_probe(k_cache, v_cache, seq_lens, tok_begin, tok_end, sink, desc: HgAttnDesc, stream=None) -> None:

@@ -630,6 +630,42 @@ hg_status hg_kv_evict(const void* k_cache, const void* v_cache, int32_t* tok_beg
     return cudaGetLastError() == cudaSuccess ? HG_OK : HG_ERR_CUDA;
 }
 
+hg_status hg_kv_evict_begin(int32_t* tok_begin, const int32_t* tok_end, const int32_t* n_evict, int32_t max_evict,
+                            int32_t max_freed, int32_t* src_begin, int32_t* n_moved, void* stream, const hg_attn_desc* desc) {
+    hg_status st = check_pool(desc);
+    if (st != HG_OK) return st;
+    if (!tok_begin || !tok_end || !n_evict || !src_begin || !n_moved || max_evict < 1 || max_freed < 0) return HG_ERR_INVALID_ARG;
+    kv_evict_begin_kernel<<<(desc->batch + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        desc->batch, ilog2_exact(desc->page_size), desc->max_pages, desc->num_pages, tok_begin, tok_end, n_evict, max_evict,
+        desc->block_table, max_freed > 0 ? 1 : 0, max_freed, src_begin, n_moved, desc->status);
+    return cudaGetLastError() == cudaSuccess ? HG_OK : HG_ERR_CUDA;
+}
+
+hg_status hg_kv_evict_copy(const void* k_cache, const void* v_cache, const int32_t* src_begin, const int32_t* n_moved,
+                           int32_t max_evict, void* k_out, void* v_out, void* stream, const hg_attn_desc* desc) {
+    hg_status st = check_pool(desc);
+    if (st != HG_OK) return st;
+    if (!k_cache || !v_cache || !src_begin || !n_moved || !k_out || !v_out || max_evict < 1) return HG_ERR_INVALID_ARG;
+    if (!aligned16(k_cache) || !aligned16(v_cache) || !aligned16(k_out) || !aligned16(v_out)) return HG_ERR_INVALID_ARG;
+    const KvPoolView pv = pool_view(desc, k_cache, v_cache);
+    dim3 grid((unsigned)((max_evict + EVICT_TOK_PER_CTA - 1) / EVICT_TOK_PER_CTA), (unsigned)desc->batch);
+    kv_evict_copy_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(pv, src_begin, nullptr, n_moved,
+                                                                               static_cast<uint16_t*>(k_out),
+                                                                               static_cast<uint16_t*>(v_out), max_evict, desc->status);
+    return cudaGetLastError() == cudaSuccess ? HG_OK : HG_ERR_CUDA;
+}
+
+hg_status hg_kv_evict_finish(const int32_t* src_begin, const int32_t* n_moved, int32_t* freed_pages, int32_t* n_freed,
+                             int32_t max_freed, void* stream, const hg_attn_desc* desc) {
+    hg_status st = check_pool(desc);
+    if (st != HG_OK) return st;
+    if (!src_begin || !n_moved || max_freed < 0 || (freed_pages && max_freed < 1)) return HG_ERR_INVALID_ARG;
+    kv_evict_finish_kernel<<<(desc->batch + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        desc->batch, ilog2_exact(desc->page_size), desc->max_pages, src_begin, n_moved, const_cast<int32_t*>(desc->block_table),
+        freed_pages, n_freed, max_freed);
+    return cudaGetLastError() == cudaSuccess ? HG_OK : HG_ERR_CUDA;
+}
+
 const char* hg_status_string(hg_status s) {
     switch (s) {
         case HG_OK: return "ok";

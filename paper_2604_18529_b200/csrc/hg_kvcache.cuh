@@ -62,7 +62,8 @@ __global__ void kv_evict_copy_kernel(KvPoolView pv, const int32_t* __restrict__ 
                                      int32_t* status) {
     const int b = blockIdx.y;
     const int tb = tok_begin[b];
-    const int ne = max(0, min(min(n_evict[b], max_evict), tok_end[b] - tb));
+    // (three-step form: tok_begin / n_evict are the recorded range, tok_end is absent)
+    const int ne = max(0, min(min(n_evict[b], max_evict), tok_end ? tok_end[b] - tb : max_evict));
     const int vec_per_row = pv.D / 8, vec_per_tok = pv.Hkv * vec_per_row;
     const int i0 = blockIdx.x * EVICT_TOK_PER_CTA, i1 = min(ne, i0 + EVICT_TOK_PER_CTA);
     __shared__ int s_phys[EVICT_TOK_PER_CTA];          // one block-table look-up per token, not per vector
@@ -102,43 +103,86 @@ __global__ void kv_evict_copy_kernel(KvPoolView pv, const int32_t* __restrict__ 
     }
 }
 
-// After the copy: advances tok_begin, un-maps the pages that no longer hold a token of the slice and lists
-// their physical ids in freed [B][max_freed] (-1 padded), n_freed [B].  One thread per sequence.
-// A page is only un-mapped if its id can be reported: when a freed list is given and fills up, the eviction of
-// that sequence stops at the first page it cannot list (tok_begin goes to that page's first token, which stays
-// resident).  A sequence whose evicted range touches an unmapped or out-of-pool page (the copy kernel flagged
-// it and skipped those rows) keeps its beginning and its table row: no token is lost from both tiers.
+// Which rows leave sequence b: [tb, nb).  ne = min(n_evict, max_evict, slice length) rows are asked for; the range is
+// cut back to nothing when it meets an unmapped or out-of-pool block-table entry (no token may be lost from both
+// tiers), and, when the emptied pages are to be listed, to the first page that does not fit a list of max_freed
+// entries (no page is un-mapped whose id cannot be reported).
+struct EvictRange { int tb, nb; };
+
+__device__ __forceinline__ EvictRange evict_range(int b, int page_shift, int max_pages, int num_pages, const int32_t* tok_begin,
+                                                  const int32_t* tok_end, const int32_t* n_evict, int max_evict,
+                                                  const int32_t* block_table, bool listed, int max_freed) {
+    EvictRange r;
+    r.tb = tok_begin[b];
+    const int ne = max(0, min(min(n_evict[b], max_evict), tok_end[b] - r.tb));
+    r.nb = r.tb + ne;
+    if (!block_table || ne == 0) return r;
+    const int first_pg = r.tb >> page_shift;
+    for (int pg = first_pg; pg <= ((r.nb - 1) >> page_shift); ++pg) {
+        const int phys = pg < max_pages ? block_table[(size_t)b * max_pages + pg] : -1;
+        if (phys < 0 || phys >= num_pages) { r.nb = r.tb; return r; }
+    }
+    // pages wholly below the new beginning leave; a partly used page stays mapped (it may still take appended rows)
+    if (listed && (r.nb >> page_shift) - first_pg > max_freed) r.nb = (first_pg + max_freed) << page_shift;
+    return r;
+}
+
+// Un-maps the pages wholly below nb (starting at tb's page) and lists them.  One thread's work for one sequence.
+__device__ __forceinline__ void evict_unmap(int b, int page_shift, int max_pages, EvictRange r, int32_t* block_table,
+                                            int32_t* freed, int32_t* n_freed, int max_freed) {
+    int cnt = 0;
+    if (block_table)
+        for (int pg = r.tb >> page_shift; pg < (r.nb >> page_shift) && pg < max_pages; ++pg) {
+            if (freed && cnt < max_freed) freed[(size_t)b * max_freed + cnt] = block_table[(size_t)b * max_pages + pg];
+            ++cnt;
+            block_table[(size_t)b * max_pages + pg] = -1;
+        }
+    if (freed) for (int i = cnt; i < max_freed; ++i) freed[(size_t)b * max_freed + i] = -1;
+    if (n_freed) n_freed[b] = cnt;
+}
+
+// After the copy (one-call form): advances tok_begin, un-maps the pages that no longer hold a token of the slice and
+// lists their physical ids in freed [B][max_freed] (-1 padded), n_freed [B].  One thread per sequence.
 __global__ void kv_evict_commit_kernel(int B, int page_shift, int max_pages, int num_pages, int32_t* tok_begin,
                                        const int32_t* tok_end, const int32_t* n_evict, int max_evict, int32_t* block_table,
                                        int32_t* freed, int32_t* n_freed, int max_freed) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
-    const int tb = tok_begin[b], te = tok_end[b];
-    const int ne = max(0, min(min(n_evict[b], max_evict), te - tb));
-    int nb = tb + ne;
-    // pages wholly below the new beginning leave; a partly used page stays mapped (it may still take appended rows)
-    const int first_pg = tb >> page_shift;
-    int cnt = 0;
-    bool bad = false;
-    if (block_table && ne > 0)
-        for (int pg = first_pg; pg <= ((nb - 1) >> page_shift); ++pg) {
-            const int phys = pg < max_pages ? block_table[(size_t)b * max_pages + pg] : -1;
-            bad |= phys < 0 || phys >= num_pages;
-        }
-    if (bad) nb = tb;
-    const int last_pg = nb >> page_shift;
-    for (int pg = first_pg; pg < last_pg && pg < max_pages; ++pg) {
-        if (block_table) {
-            const int phys = block_table[(size_t)b * max_pages + pg];
-            if (freed && cnt == max_freed) { nb = pg << page_shift; break; }     // cannot report it: it stays
-            if (freed) freed[(size_t)b * max_freed + cnt] = phys;
-            ++cnt;
-            block_table[(size_t)b * max_pages + pg] = -1;
-        }
-    }
-    if (freed) for (int i = cnt; i < max_freed; ++i) freed[(size_t)b * max_freed + i] = -1;
-    if (n_freed) n_freed[b] = cnt;
-    tok_begin[b] = nb;
+    const EvictRange r = evict_range(b, page_shift, max_pages, num_pages, tok_begin, tok_end, n_evict, max_evict, block_table,
+                                     freed != nullptr, max_freed);
+    evict_unmap(b, page_shift, max_pages, r, block_table, freed, n_freed, max_freed);
+    tok_begin[b] = r.nb;
+}
+
+// Three-step form, for an eviction that drains beside the attention of the same step.
+// Step 1 (on the attention's stream, before it): decides the range, records it in src_begin / n_moved and moves
+// tok_begin, so that whatever follows on this stream already works on the shrunk slice.  The block table is left
+// alone: the rows are still where the table says.
+__global__ void kv_evict_begin_kernel(int B, int page_shift, int max_pages, int num_pages, int32_t* tok_begin,
+                                      const int32_t* tok_end, const int32_t* n_evict, int max_evict,
+                                      const int32_t* block_table, int listed, int max_freed, int32_t* src_begin,
+                                      int32_t* n_moved, int32_t* status) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const EvictRange r = evict_range(b, page_shift, max_pages, num_pages, tok_begin, tok_end, n_evict, max_evict, block_table,
+                                     listed != 0, max_freed);
+    const int asked = max(0, min(min(n_evict[b], max_evict), tok_end[b] - r.tb));
+    if (r.nb == r.tb && asked > 0 && status) atomicOr(status, HG_DEV_BAD_PAGE);
+    src_begin[b] = r.tb;
+    n_moved[b] = r.nb - r.tb;
+    tok_begin[b] = r.nb;
+}
+
+// Step 3 (any stream, after step 2's copy kernel): un-maps and lists the pages below the new beginning.  These
+// block-table entries belong to pages no attention over the shrunk slice looks up.
+__global__ void kv_evict_finish_kernel(int B, int page_shift, int max_pages, const int32_t* src_begin, const int32_t* n_moved,
+                                       int32_t* block_table, int32_t* freed, int32_t* n_freed, int max_freed) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    EvictRange r;
+    r.tb = src_begin[b];
+    r.nb = r.tb + n_moved[b];
+    evict_unmap(b, page_shift, max_pages, r, block_table, freed, n_freed, max_freed);
 }
 
 }  // namespace hg

@@ -305,3 +305,62 @@ class HostKvStore:
                 self.v[b, n0:n0 + ne].copy_(v_out[b, :ne], non_blocking=True)
             self.n[b] = n0 + ne
         torch.cuda.current_stream(dev).synchronize()
+
+    def begin_evict(self, k_cache, v_cache, tok_begin, tok_end, n_evict: List[int], desc: hg.HgAttnDesc,
+                    freed: Optional[torch.Tensor] = None, n_freed: Optional[torch.Tensor] = None) -> "PendingEviction":
+        """The same move, draining beside the attention of this decode step instead of in front of it.
+
+        On the current stream only ``hg_kv_evict_begin`` is enqueued: it advances ``tok_begin``, so the attention the
+        caller enqueues next already covers the shrunk slice.  The row copy, the device -> host copies and the
+        un-mapping of the emptied pages (``hg_kv_evict_copy``, ``hg_kv_evict_finish``) go to this store's own stream
+        behind an event.  Call ``wait()`` on the returned object before using the host rows or the freed pages."""
+        B, dev = len(n_evict), k_cache.device
+        max_evict = max(max(n_evict), 1)
+        if any(int(self.n[b]) + n_evict[b] > self.capacity for b in range(B)):
+            raise ValueError("host rows full")
+        Hkv, D = self.k.shape[2], self.k.shape[3]
+        if getattr(self, "_stream", None) is None:
+            self._stream = torch.cuda.Stream(device=dev)
+        main, side = torch.cuda.current_stream(dev), self._stream
+        k_out = torch.empty(B, max_evict, Hkv, D, dtype=self.k.dtype, device=dev)
+        v_out = torch.empty_like(k_out)
+        src_begin = torch.empty(B, dtype=torch.int32, device=dev)
+        n_moved = torch.empty(B, dtype=torch.int32, device=dev)
+        n_dev = torch.tensor(n_evict, dtype=torch.int32, device=dev)
+        hg.hg_kv_evict_begin(tok_begin, tok_end, n_dev, max_evict, 0 if freed is None else freed.shape[1], src_begin, n_moved,
+                             desc, main)
+        started = torch.cuda.Event()
+        started.record(main)
+        moved_host = torch.empty(B, dtype=torch.int32).pin_memory()
+        with torch.cuda.stream(side):
+            side.wait_event(started)
+            hg.hg_kv_evict_copy(k_cache, v_cache, src_begin, n_moved, k_out, v_out, desc, side)
+            for b in range(B):
+                n0, ne = int(self.n[b]), n_evict[b]
+                if ne:
+                    self.k[b, n0:n0 + ne].copy_(k_out[b, :ne], non_blocking=True)
+                    self.v[b, n0:n0 + ne].copy_(v_out[b, :ne], non_blocking=True)
+            hg.hg_kv_evict_finish(src_begin, n_moved, freed, n_freed, desc, side)
+            moved_host.copy_(n_moved, non_blocking=True)
+            done = torch.cuda.Event()
+            done.record(side)
+        for t in (k_out, v_out, src_begin, n_moved, n_dev):
+            t.record_stream(side)
+        return PendingEviction(self, done, moved_host, list(n_evict))
+
+
+class PendingEviction:
+    """An eviction whose copies are still draining on the store's stream."""
+
+    def __init__(self, store: HostKvStore, done: torch.cuda.Event, moved_host: torch.Tensor, asked: List[int]):
+        self.store, self.done, self.moved_host, self.asked = store, done, moved_host, asked
+
+    def wait(self) -> List[int]:
+        """Blocks until the rows are in the host tier; returns how many rows of every sequence arrived (fewer than
+        asked for only when the library cut a range back) and counts them in."""
+        self.done.synchronize()
+        moved = self.moved_host.tolist()
+        for b, m in enumerate(moved):
+            self.store.n[b] = int(self.store.n[b]) + m
+        return moved
+

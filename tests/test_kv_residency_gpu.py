@@ -3,6 +3,8 @@ oldest tokens to the host and attending over the shrunk slice.  Data movement is
 the logical rows of the workload generator, attention against the oracle."""
 import dataclasses
 
+import numpy as np
+
 import pytest
 import torch
 
@@ -172,3 +174,64 @@ def test_eviction_over_an_unmapped_page_leaves_the_sequence_alone():
     assert prob.tok_begin.tolist() == [32, 64] and n_freed.tolist() == [0, 3]
     assert torch.equal(prob.kv["block_table"][0], table0[0]) and (freed[0] == -1).all()
     assert torch.equal(k_out[1, :48, 0].cpu(), w.kv_rows("k", 1, 0, 16, 64))
+
+
+@pytest.mark.parametrize("G", [1, 4])
+def test_eviction_beside_attention_gives_the_bits_of_the_serial_order(G):
+    """The three-step eviction (begin on the attention's stream; row copy, device -> host copies and un-mapping on a
+    second stream) with the attention of the same step running meanwhile over the shrunk slice: block table, freed
+    list, host rows and attention output are bit for bit those of evicting first and attending afterwards, and the
+    attention - merged with a host partial recomputed from the rows that arrived on the host - equals monolithic
+    attention over the whole sequence."""
+    from oracle import hg_oracle as O
+    from paper_2604_18529_b200.hybrid import HostKvStore
+    from parity_util import bits
+    w = W.AttnWorkload("beside", 3, 2 * G, 2, 128, "f16", [3000, 1500, 900], [700, 100, 333], [3000, 1500, 900], page_size=16,
+                       chunk_tokens=256, seed=60 + G)
+    n_evict = [640, 333, 0]
+    new_begin = [tb + ne for tb, ne in zip(w.tok_begin, n_evict)]
+    after = dataclasses.replace(w, tok_begin=new_begin)
+    q, K, V = bits(w.q()), bits(w.kv_logical("k")), bits(w.kv_logical("v"))
+    ref_out, ref_lse = O.full_batch(q, K, V, w.dtype, [0] * w.B, w.seq_lens)
+
+    results = []
+    for beside in (False, True):
+        prob = DeviceProblem(w, DEV)
+        # the host tier already holds the tokens below the old beginning
+        store = HostKvStore(w.B, 2048, w.Hkv, w.D, torch.float16)
+        for b in range(w.B):
+            for g in range(w.Hkv):
+                store.k[b, : w.tok_begin[b], g] = w.kv_rows("k", b, g, 0, w.tok_begin[b])
+                store.v[b, : w.tok_begin[b], g] = w.kv_rows("v", b, g, 0, w.tok_begin[b])
+            store.n[b] = w.tok_begin[b]
+        freed = torch.full((w.B, 64), 77, dtype=torch.int32, device=DEV)
+        n_freed = torch.zeros(w.B, dtype=torch.int32, device=DEV)
+        # attention of the shrunk slice, with no host source: its partials must not depend on the order either
+        if beside:
+            pending = store.begin_evict(prob.kv["k"], prob.kv["v"], prob.tok_begin, prob.tok_end, n_evict, prob.desc, freed, n_freed)
+            prob.step([])                                  # enqueued right behind step 1, runs while the rows drain
+            assert pending.wait() == n_evict
+        else:
+            store.evict_from_gpu(prob.kv["k"], prob.kv["v"], prob.tok_begin, prob.tok_end, n_evict, prob.desc, freed, n_freed)
+            prob.step([])
+        torch.cuda.synchronize()
+        assert int(prob.status.item()) == hg.HG_DEV_OK and prob.tok_begin.tolist() == new_begin
+        assert store.n.tolist() == new_begin
+        results.append((prob.out.clone(), prob.lse.clone(), prob.o_part.clone(), prob.kv["block_table"].clone(), freed.clone(),
+                        n_freed.clone(), store.k.clone(), store.v.clone()))
+        # the host rows are the sequence's prefix, bit for bit; the host partial comes from them
+        hm = np.empty((w.B, w.Hq, 1)); hl = np.empty((w.B, w.Hq, 1)); ho = np.empty((w.B, w.Hq, 1, w.D))
+        for b in range(w.B):
+            for g in range(w.Hkv):
+                assert torch.equal(store.k[b, : new_begin[b], g], w.kv_rows("k", b, g, 0, new_begin[b]))
+                assert torch.equal(store.v[b, : new_begin[b], g], w.kv_rows("v", b, g, 0, new_begin[b]))
+            for h in range(w.Hq):
+                g = h // w.G
+                hm[b, h, 0], hl[b, h, 0], ho[b, h, 0] = O.partial(q[b, h], bits(store.k[b, :, g]), bits(store.v[b, :, g]),
+                                                                   w.dtype, t0=0, n=new_begin[b])
+        prob.merge([tuple(torch.from_numpy(x).float().to(DEV) for x in (ho, hm, hl))])
+        torch.cuda.synchronize()
+        check_output(prob.out, prob.lse, ref_out, ref_lse, "beside" if beside else "serial")
+    for a, b in zip(*results):
+        assert torch.equal(a, b)
+    assert (results[0][5] > 0).any()                       # pages did get freed and listed
