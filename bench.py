@@ -402,8 +402,9 @@ def measure_workload(name, args, R, sampler):
     if args.chunk:
         import dataclasses
         w = dataclasses.replace(w, chunk_tokens=args.chunk)
-    # (empty chunk slots - a ragged batch has many - get m = -inf and l = 0 only: the merge never reads their o rows)
-    prob = DeviceProblem(w, dev, flags=pkg.binding.HG_FLAG_SPARSE_EMPTY)
+    # (empty chunk slots - a ragged batch has many - get m = -inf and l = 0 only: the merge never reads their o rows;
+    # the work counter starts at zero and every call leaves it so: no clearing between the steps of the loop)
+    prob = DeviceProblem(w, dev, flags=pkg.binding.HG_FLAG_SPARSE_EMPTY | pkg.binding.HG_FLAG_COUNTER_CLEAN)
     # partials of the host-held slice: produced by the host in the real system; here synthetic values with
     # the statistics of a real partial (they are inputs of the merge, not results of this library)
     gen = torch.Generator(device=dev).manual_seed(w.seed)

@@ -66,6 +66,13 @@ typedef enum hg_dtype { HG_DTYPE_F16 = 0, HG_DTYPE_BF16 = 1 } hg_dtype;
                                    attention itself.  hg_attn_decode and its variants always work this way on
                                    their own workspace. */
 
+#define HG_FLAG_COUNTER_CLEAN 4u /* both words of sched_counter are zero when the call's kernel starts (for instance
+                                   because the last thing that used them was an earlier call of this library that
+                                   ended normally: every call leaves them at zero).  The call then enqueues no
+                                   clearing in front of its kernel, which lets the kernel start as a programmatic
+                                   dependent of whatever precedes it in the stream.  After a call that reported
+                                   HG_DEV_WAIT_TIMEOUT clear the words yourself before using the flag again. */
+
 /* bits the kernels may set in *hg_attn_desc.status (device word, optional; several may be set at once) */
 #define HG_DEV_OK 0
 #define HG_DEV_WAIT_TIMEOUT 1 /* a bounded on-chip barrier wait ran out; the call's results are invalid.
@@ -116,11 +123,13 @@ typedef struct hg_attn_desc {
     float scale;               /* logit scale; 0 means 1/sqrt(D) */
     uint32_t flags;            /* HG_FLAG_* */
     int32_t* status;           /* dev, optional: receives HG_DEV_* if a kernel detects a problem */
-    int32_t* sched_counter;    /* dev, optional, 4 bytes: when given, hg_attn_partial zeroes it on the stream and
-                                  its CTAs draw work items from it dynamically (better balance on ragged
-                                  batches); NULL: items are dealt round-robin.  Left alone when the problem has no
-                                  more items than the device has resident CTAs.  Must not be shared by calls
-                                  that may overlap on the GPU.  Present when struct_size covers it. */
+    int32_t* sched_counter;    /* dev, optional, 8 bytes (two int32, 8-byte aligned): when given, the CTAs of
+                                  hg_attn_partial draw work items from it dynamically (better balance on ragged
+                                  batches); NULL: items are dealt round-robin.  The call clears both words on the
+                                  stream in front of its kernel unless HG_FLAG_COUNTER_CLEAN says they are zero
+                                  already; the kernel leaves them at zero when it ends normally.  Left alone when
+                                  the problem has no more items than the device has resident CTAs.  Must not be
+                                  shared by calls that may overlap on the GPU.  Present when struct_size covers it. */
     uint32_t tune;             /* HG_TUNE_* bits; 0 = the library's defaults.  Each bit switches one choice of the
                                   schedule off; results do not depend on them (the tests show equal bits), speed
                                   does.  Present when struct_size covers it, like the two fields below. */

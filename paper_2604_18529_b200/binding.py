@@ -23,6 +23,7 @@ HG_DEV_OK, HG_DEV_WAIT_TIMEOUT, HG_DEV_BAD_PAGE, HG_DEV_RANGE = 0, 1, 2, 4
 HG_MAX_MERGE_SRC = 8
 HG_FLAG_TEST_STALL = 1
 HG_FLAG_SPARSE_EMPTY = 2
+HG_FLAG_COUNTER_CLEAN = 4
 HG_STATIC_SCRATCH_BYTES = 8 << 20
 (HG_TUNE_NO_PERSISTENT, HG_TUNE_NO_DYNAMIC, HG_TUNE_NO_PDL, HG_TUNE_NO_MERGE_CLUSTER, HG_TUNE_NO_MERGE_ROWS,
  HG_TUNE_NO_GQA16, HG_TUNE_NO_HOST_DIRECT) = 1, 2, 4, 8, 16, 32, 64

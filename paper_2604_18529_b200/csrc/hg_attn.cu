@@ -60,7 +60,7 @@ static hg_status check_desc(const hg_attn_desc* d, bool need_kv) {
     if (d->chunk_tokens % TILE_T || d->chunk_tokens % d->page_size || d->chunk_tokens > 65536)
         return HG_ERR_UNSUPPORTED;
     if (d->chunk_tokens / d->page_size > MAX_CHUNK_PAGES) return HG_ERR_UNSUPPORTED;
-    if (desc_sched(d) && (reinterpret_cast<uintptr_t>(desc_sched(d)) & 3u)) return HG_ERR_INVALID_ARG;
+    if (desc_sched(d) && (reinterpret_cast<uintptr_t>(desc_sched(d)) & 7u)) return HG_ERR_INVALID_ARG;
     if ((int64_t)d->num_kv_heads * ((d->num_q_heads / d->num_kv_heads + 7) / 8) > 65535) return HG_ERR_UNSUPPORTED;
     if (!d->block_table && (int64_t)d->batch * d->max_pages > d->num_pages) return HG_ERR_INVALID_ARG;
     return HG_OK;
@@ -168,7 +168,7 @@ static hg_status launch_partial_t(const CUtensorMap& tk, const CUtensorMap& tv, 
         grid = dim3((unsigned)(slots < resident ? slots : resident), 1, 1);
         if (slots <= resident) p.sched = nullptr;     // at most one item per CTA: nothing to hand out, no counter to clear
     }
-    if (p.sched && !counter_is_zero && cudaMemsetAsync(p.sched, 0, sizeof(int32_t), st) != cudaSuccess) {
+    if (p.sched && !counter_is_zero && cudaMemsetAsync(p.sched, 0, 2 * sizeof(int32_t), st) != cudaSuccess) {
         cudaGetLastError();
         return HG_ERR_CUDA;
     }
@@ -206,6 +206,7 @@ static hg_status run_partial(int mode, const void* q, const void* k, const void*
     hg_status st = check_desc(d, true);
     if (st != HG_OK) return st;
     if (!k || !v || !seq_lens || !tok_begin || !tok_end) return HG_ERR_INVALID_ARG;
+    if (d->flags & HG_FLAG_COUNTER_CLEAN) counter_is_zero = true;      // the caller vouches for it
     if (mode == MODE_PROBE) {
         if (!sink) return HG_ERR_INVALID_ARG;
     } else if (!q || !o_part || !m_part || !l_part) {

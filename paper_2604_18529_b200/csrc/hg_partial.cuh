@@ -64,7 +64,8 @@ struct PartialParams {
     int test_stall;           // HG_FLAG_TEST_STALL: the producer never fills a stage
     int sparse_empty;         // HG_FLAG_SPARSE_EMPTY: empty chunk slots get m and l only, their o rows stay untouched
     int pdl_wait;             // launched as a programmatic dependent: wait for the preceding kernel before reading any input
-    int32_t* sched;           // zeroed work counter: items are handed out dynamically (NULL: round-robin)
+    int32_t* sched;           // two zeroed words: [0] hands out items dynamically, [1] counts the CTAs that are done
+                              // drawing (NULL: round-robin)
     float scale_log2;         // logit scale * log2(e)
 #ifdef HG_TRACE
     long long* trace;         // development builds only: 8 timestamps / counters per CTA
@@ -477,6 +478,16 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
             if (okw && lane == 0) {
                 ctl.sdesc[s] = make_int2(-1, 0);
                 mbar_arrive_expect_tx(&ctl.full[s], 0u);
+            }
+        }
+        if (dynamic && lane == 0) {
+            // This CTA draws no further index.  The last CTA to get here leaves both words of the counter at zero
+            // for the next call, which then needs no clearing in front of it.
+            __threadfence();
+            if (atomicAdd(p.sched + 1, 1) == (int)gridDim.x - 1) {
+                p.sched[0] = 0;
+                p.sched[1] = 0;
+                __threadfence();
             }
         }
         if (*abort_flag && lane == 0) {

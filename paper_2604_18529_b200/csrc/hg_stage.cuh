@@ -18,7 +18,7 @@ struct StageParams {
     void* dst[STAGE_MAX_SEG];           // device memory
     uint32_t bytes[STAGE_MAX_SEG];
     int n;
-    int32_t* zero;                      // a device word to clear on the way (the work counter of the launch that follows), or NULL
+    int32_t* zero;                      // two device words to clear on the way (the work counter of the launch that follows), or NULL
 };
 
 // Any number of CTAs; segment s is copied by all of them together, 16 bytes per thread and trip where
@@ -26,7 +26,7 @@ struct StageParams {
 __global__ void __launch_bounds__(STAGE_THREADS) stage_kernel(const StageParams p) {
     const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
     const uint32_t nt = gridDim.x * blockDim.x;
-    if (t == 0 && p.zero) *p.zero = 0;
+    if (t == 0 && p.zero) { p.zero[0] = 0; p.zero[1] = 0; }
     for (int s = 0; s < p.n; ++s) {
         const uintptr_t a = reinterpret_cast<uintptr_t>(p.src[s]) | reinterpret_cast<uintptr_t>(p.dst[s]) | p.bytes[s];
         if ((a & 15u) == 0) {

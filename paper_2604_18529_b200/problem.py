@@ -25,7 +25,7 @@ class DeviceProblem:
         self.tok_begin = torch.tensor(w.tok_begin, dtype=torch.int32, device=dev)
         self.tok_end = torch.tensor(w.tok_end, dtype=torch.int32, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
-        self.sched = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.sched = torch.zeros(2, dtype=torch.int32, device=dev)
         self.NC = w.num_chunks
         self.desc = self.make_desc(w.chunk_tokens, self.NC, flags=flags)
         B, Hq, D, NC = w.B, w.Hq, w.D, self.NC

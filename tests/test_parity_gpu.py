@@ -394,6 +394,31 @@ def test_result_does_not_depend_on_the_schedule(G):
             assert torch.equal(a, b)
 
 
+@pytest.mark.parametrize("G", [1, 8])
+def test_every_call_leaves_the_work_counter_at_zero(G):
+    """More items than resident CTAs, so the counter hands them out.  The last CTA to stop drawing clears both
+    words: with HG_FLAG_COUNTER_CLEAN the next call runs without any clearing in front of it (and may start as a
+    programmatic dependent) and gives the same bits as a call that cleared the counter itself."""
+    w = wl(B=6, Hq=4 * G, Hkv=4, seq_lens=[6000] * 6, tok_begin=[100] * 6, tok_end=[6000] * 6, chunk_tokens=64, seed=70 + G)
+    assert sum(w.chunk_grid(b)[1] for b in range(w.B)) * w.Hkv > 2 * 296
+    ref = OracleRef(w)
+    prob = DeviceProblem(w, DEV)
+    prob.step(ref.host_partials_device(DEV))
+    torch.cuda.synchronize()
+    assert prob.sched.tolist() == [0, 0]
+    want = (prob.o_part.clone(), prob.m_part.clone(), prob.l_part.clone(), prob.out.clone(), prob.lse.clone())
+    prob.desc = prob.make_desc(w.chunk_tokens, prob.NC, flags=hg.HG_FLAG_COUNTER_CLEAN)
+    for _ in range(3):
+        for t in (prob.o_part, prob.m_part, prob.l_part, prob.out, prob.lse):
+            t.fill_(float("nan"))
+        prob.step(ref.host_partials_device(DEV))        # back to back: partial, merge, partial, ...
+    torch.cuda.synchronize()
+    assert prob.sched.tolist() == [0, 0] and int(prob.status.item()) == hg.HG_DEV_OK
+    for a, b in zip(want, (prob.o_part, prob.m_part, prob.l_part, prob.out, prob.lse)):
+        assert torch.equal(a, b)
+    check_output(prob.out, prob.lse, ref.out, ref.lse)
+
+
 def test_without_a_work_counter_items_are_dealt_round_robin():
     w = wl(Hq=8, Hkv=2)
     ref = OracleRef(w)
