@@ -342,6 +342,40 @@ def time_extras(w, prob, dev, steps):
     return out
 
 
+def time_handoff(dev, steps):
+    """The device side of the paper's literal hand-off on HBM-resident inputs larger than L2: partials from host-computed
+    logits [B][Hq][K] and V rows [B][Hkv][K][D] (hg_attn_partial_from_logits), one head per KV head and groups of 8."""
+    import torch
+    import paper_2604_18529_b200 as pkg
+    peak, peak_kind = measured_peak()
+    out = []
+    for name, B, Hq, Hkv, K in (("mha", 8, 40, 40, 8192), ("gqa8", 1, 64, 8, 262144)):
+        gen = torch.Generator(device=dev).manual_seed(11)
+        logits = torch.randn(B, Hq, K, device=dev, generator=gen)
+        vrows = torch.randn(B, Hkv, K, 128, device=dev, generator=gen).half()
+        n_sel = torch.full((B,), K, dtype=torch.int32, device=dev)
+        ld = pkg.logits_desc(batch=B, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=128, dtype="f16", max_selected=K, chunk_tokens=256)
+        o = torch.empty(B, Hq, ld.num_chunks, 128, device=dev); m = torch.empty(B, Hq, ld.num_chunks, device=dev); l = torch.empty_like(m)
+        call = lambda: pkg.hg_attn_partial_from_logits(logits, vrows, n_sel, o, m, l, ld)
+        for _ in range(3):
+            call()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            call()
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / steps
+        nbytes = logits.numel() * 4 + vrows.numel() * 2 + o.numel() * 4 + 2 * m.numel() * 4
+        out.append({"shape": name, "batch": B, "q_heads": Hq, "kv_heads": Hkv, "head_dim": 128, "selected_per_seq": K,
+                    "chunk_tokens": 256, "us": us, "alg_bytes": nbytes, "gbs": nbytes / us / 1e3,
+                    "frac": nbytes / us / 1e3 / peak, "peak_kind": f"{peak_kind} copy bandwidth",
+                    "frac_of_8000": nbytes / us / 1e3 / 8000.0})
+        del logits, vrows, o, m, l
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_reference(args, rank, world):
     """--impl reference: the fp64 oracle on the host cores, each step a bounded sample of the workload."""
     if rank != 0:
@@ -659,6 +693,7 @@ def main():
         time.sleep(0.3)
     recs = {n: measure_workload(n, args, R, sampler) for n in names}
     shard_rec = measure_sharded(args, R) if (world > 1 or args.sharded) and args.workload == "all" else None
+    handoff = time_handoff(R.dev, args.steps) if args.workload == "all" and rank == 0 else None
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
@@ -679,6 +714,7 @@ def main():
     if args.workload == "all":
         config["workloads"] = [recs[n] for n in names]
         config["min_step_frac_of_8000"] = min(recs[n]["step_frac_of_8000"] for n in LARGE)
+        config["handoff"] = handoff
     line = {
         "metric": METRIC, "value": head["kv_tokens_per_s"], "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": hl["ms_step"], "higher_is_better": True,

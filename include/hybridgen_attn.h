@@ -288,6 +288,8 @@ typedef struct hg_logits_desc {
     int32_t max_selected;  /* K: row length of logits / v_rows (selected-token slots per sequence) */
     int32_t chunk_tokens;  /* slots per partial, a multiple of 32, at most 1024 */
     int32_t num_chunks;    /* NC >= ceil(K / chunk_tokens): partials per (sequence, head) */
+    int32_t* status;       /* dev, optional (present when struct_size covers it): receives HG_DEV_WAIT_TIMEOUT if a
+                              bounded on-chip wait of the kernel ran out */
 } hg_logits_desc;
 
 /*
@@ -298,14 +300,19 @@ typedef struct hg_logits_desc {
  * device logits and V rows and taking one softmax over them.
  *
  *   logits   dev float [B][Hq][K]      scaled logits s = q.k / sqrt(D) of the selected tokens, natural units;
- *                                      a slot holding -inf is ignored (its V row is never used)
+ *                                      a slot holding -inf weighs nothing for that head
  *   v_rows   dev 16-bit [B][Hkv][K][D] V rows of those tokens, slot for slot; the query heads of a group share
- *                                      their KV head's rows; 16-byte aligned
+ *                                      their KV head's rows; 16-byte aligned.  Rows of slots at or beyond n_sel[b]
+ *                                      are never used, whatever they hold; rows below n_sel[b] must hold finite
+ *                                      numbers even where every head's logit is -inf (their weight is zero, and
+ *                                      zero times a NaN is not zero)
  *   n_sel    dev int32 [B]             slots in use per sequence (clamped to [0, K])
  *   o_part, m_part, l_part             dev float [B][Hq][NC][D] / [B][Hq][NC]: chunk c covers slots
  *                                      [c * chunk_tokens, (c+1) * chunk_tokens) below n_sel; empty chunks are
  *                                      (m, l, o) = (-inf, 0, 0)
  * Token order and token indices do not matter for the result and are not passed.
+ * Every group size runs the P.V product on tensor cores with P as a two-term (hi + lo) 16-bit expansion, fp32
+ * accumulation; m is the exact maximum of the chunk's logits, l the fp32 sum of the unrounded weights.
  */
 hg_status hg_attn_partial_from_logits(const float* logits, const void* v_rows, const int32_t* n_sel, float* o_part,
                                       float* m_part, float* l_part, void* stream, const hg_logits_desc* desc);

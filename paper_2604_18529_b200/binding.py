@@ -73,6 +73,7 @@ class HgLogitsDesc(C.Structure):
         ("max_selected", C.c_int32),
         ("chunk_tokens", C.c_int32),
         ("num_chunks", C.c_int32),
+        ("status", C.c_void_p),
     ]
 
 
@@ -223,13 +224,15 @@ def hg_attn_partial(q, k_cache, v_cache, seq_lens, tok_begin, tok_end, o_part, m
 
 
 def logits_desc(*, batch: int, num_q_heads: int, num_kv_heads: int, head_dim: int, dtype, max_selected: int,
-                chunk_tokens: int = 256, num_chunks: int = 0) -> HgLogitsDesc:
+                chunk_tokens: int = 256, num_chunks: int = 0, status: Optional[torch.Tensor] = None) -> HgLogitsDesc:
     d = HgLogitsDesc()
     d.struct_size = C.sizeof(HgLogitsDesc)
     d.batch, d.num_q_heads, d.num_kv_heads, d.head_dim = batch, num_q_heads, num_kv_heads, head_dim
     d.dtype = _DTYPES[dtype]
     d.max_selected, d.chunk_tokens = max_selected, chunk_tokens
     d.num_chunks = num_chunks or -(-max_selected // chunk_tokens)
+    d.status = _dev(status, "status", torch.int32)
+    d._keep = (status,)
     return d
 
 

@@ -14,7 +14,6 @@
 #include <string.h>
 
 #include <atomic>
-#include <type_traits>
 
 #include "hg_kvcache.cuh"
 #include "hg_logits.cuh"
@@ -383,7 +382,7 @@ hg_status hg_attn_merge(const hg_partial_src* partials, int32_t n_src, float* ou
 
 hg_status hg_attn_partial_from_logits(const float* logits, const void* v_rows, const int32_t* n_sel, float* o_part,
                                       float* m_part, float* l_part, void* stream, const hg_logits_desc* d) {
-    if (!d || d->struct_size < sizeof(hg_logits_desc)) return HG_ERR_INVALID_ARG;
+    if (!d || d->struct_size < offsetof(hg_logits_desc, status)) return HG_ERR_INVALID_ARG;
     if (d->batch < 1 || d->batch > 65535 || d->num_kv_heads < 1 || d->num_kv_heads > 65535 || d->num_q_heads < 1 ||
         d->num_q_heads % d->num_kv_heads)
         return HG_ERR_INVALID_ARG;
@@ -393,39 +392,45 @@ hg_status hg_attn_partial_from_logits(const float* logits, const void* v_rows, c
     if (d->max_selected < 1 || d->chunk_tokens < 32 || d->chunk_tokens % 32 || d->num_chunks < 1) return HG_ERR_INVALID_ARG;
     if (d->chunk_tokens > LG_MAX_CHUNK) return HG_ERR_UNSUPPORTED;
     if ((int64_t)d->num_chunks * d->chunk_tokens < d->max_selected) return HG_ERR_INVALID_ARG;
+    if ((int64_t)d->batch * d->num_kv_heads * d->max_selected > 0x7fffffffll) return HG_ERR_UNSUPPORTED;   // row coordinate
     if (!logits || !v_rows || !n_sel || !o_part || !m_part || !l_part) return HG_ERR_INVALID_ARG;
     if (!aligned16(v_rows) || !aligned16(o_part)) return HG_ERR_INVALID_ARG;
     LogitsParams p;
-    p.logits = logits; p.v_rows = v_rows; p.n_sel = n_sel; p.o_part = o_part; p.m_part = m_part; p.l_part = l_part;
+    memset(&p, 0, sizeof p);
+    p.logits = logits; p.n_sel = n_sel; p.o_part = o_part; p.m_part = m_part; p.l_part = l_part;
+    p.status = d->struct_size >= sizeof(hg_logits_desc) ? d->status : nullptr;
     p.B = d->batch; p.Hq = d->num_q_heads; p.Hkv = d->num_kv_heads; p.G = p.Hq / p.Hkv; p.K = d->max_selected;
     p.chunk = d->chunk_tokens; p.NC = d->num_chunks;
-    // heads per pass over the V rows: the smallest of 1, 2, 4, 8 that covers the group (8 for larger groups)
-    const int nh = p.G >= 8 ? 8 : (p.G > 2 ? 4 : p.G);
-    const size_t smem = ((size_t)nh * p.chunk + (size_t)LG_WARPS * nh * d->head_dim) * sizeof(float);
+    // the V rows as a 3-D tensor {component within a 64-element half, row, half}; one box is 64 rows of all halves,
+    // 128-byte swizzled: the tile layout of hg_attn_partial
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return HG_ERR_CUDA;
+    const int halves = d->head_dim / 64;
+    CUtensorMap tv;
+    cuuint64_t dims[3] = {64, (cuuint64_t)d->batch * d->num_kv_heads * d->max_selected, (cuuint64_t)halves};
+    cuuint64_t strides[2] = {(cuuint64_t)d->head_dim * 2u, 128u};
+    cuuint32_t box[3] = {64, (cuuint32_t)LG_TILE, (cuuint32_t)halves};
+    cuuint32_t estr[3] = {1, 1, 1};
+    if (enc(&tv, d->dtype == HG_DTYPE_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3,
+            const_cast<void*>(v_rows), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return HG_ERR_UNSUPPORTED;
     dim3 grid((unsigned)p.NC, (unsigned)p.Hkv, (unsigned)p.B);
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     const bool bf16 = d->dtype == HG_DTYPE_BF16;
-    auto launch = [&](auto kern) -> hg_status {
+    auto launch = [&](auto kern, size_t smem) -> hg_status {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
             cudaGetLastError();
             return HG_ERR_CUDA;
         }
-        kern<<<grid, LG_THREADS, smem, cs>>>(p);
+        kern<<<grid, LG_THREADS, smem, cs>>>(tv, p);
         return cudaGetLastError() == cudaSuccess ? HG_OK : HG_ERR_CUDA;
     };
-    auto pick = [&](auto dtag, auto btag) -> hg_status {
-        constexpr int DD = decltype(dtag)::value;
-        constexpr bool BB = decltype(btag)::value;
-        switch (nh) {
-            case 1: return launch(logits_partial_kernel<DD, BB, 1>);
-            case 2: return launch(logits_partial_kernel<DD, BB, 2>);
-            case 4: return launch(logits_partial_kernel<DD, BB, 4>);
-            default: return launch(logits_partial_kernel<DD, BB, 8>);
-        }
-    };
     if (d->head_dim == 128)
-        return bf16 ? pick(std::integral_constant<int, 128>{}, std::true_type{}) : pick(std::integral_constant<int, 128>{}, std::false_type{});
-    return bf16 ? pick(std::integral_constant<int, 64>{}, std::true_type{}) : pick(std::integral_constant<int, 64>{}, std::false_type{});
+        return bf16 ? launch(logits_partial_kernel<128, true>, logits_smem_bytes<128>(p.chunk))
+                    : launch(logits_partial_kernel<128, false>, logits_smem_bytes<128>(p.chunk));
+    return bf16 ? launch(logits_partial_kernel<64, true>, logits_smem_bytes<64>(p.chunk))
+                : launch(logits_partial_kernel<64, false>, logits_smem_bytes<64>(p.chunk));
 }
 
 int32_t hg_attn_suggest_chunk(int64_t total_tokens, int32_t num_q_heads, int32_t num_kv_heads, int32_t page_size) {

@@ -103,12 +103,6 @@ struct Item {
     int tile0, ntiles;  // 64-token tiles covering it
 };
 
-// All lanes wait; the verdict is made warp-uniform so that no lane leaves a loop alone.
-__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    const bool ok = mbar_wait(bar, parity, abort_flag);
-    return __all_sync(0xffffffffu, ok);
-}
-
 // Tokens a sequence's row of the block table can address.
 __device__ __forceinline__ int table_reach(const PartialParams& p) {
     return (int)min((long long)p.max_pages << p.page_shift, (long long)INT32_MAX);
