@@ -34,6 +34,17 @@ static int32_t* desc_sched(const hg_attn_desc* d) {
     return d->struct_size >= offsetof(hg_attn_desc, sched_counter) + sizeof(int32_t*) ? d->sched_counter : nullptr;
 }
 
+// Multiplier and shift that divide a number below 2^31 by d (see FastDiv).
+static FastDiv make_fast_div(uint32_t d) {
+    FastDiv f = {0u, 0u};
+    if (d <= 1) return f;
+    uint32_t s = 0;
+    while ((1ull << s) < d) ++s;                                   // ceil(log2 d) >= 1
+    f.mul = (uint32_t)(((1ull << (31 + s)) + d - 1) / d);          // < 2^32 because d > 2^(s-1)
+    f.shift = s - 1;
+    return f;
+}
+
 static int ilog2_exact(int v) {
     for (int s = 0; s < 31; ++s)
         if ((1 << s) == v) return s;
@@ -228,6 +239,8 @@ static hg_status run_partial(int mode, const void* q, const void* k, const void*
     p.page_size = d->page_size; p.page_shift = ilog2_exact(d->page_size); p.max_pages = d->max_pages;
     p.num_pages = d->num_pages; p.C = d->chunk_tokens; p.NC = d->num_chunks;
     p.head_blocks = (mode == MODE_GQA) ? (G + 7) / 8 : (mode == MODE_GQA2 ? (G + 15) / 16 : 1);
+    p.div_C = make_fast_div((uint32_t)p.C);
+    p.div_Hkv = make_fast_div((uint32_t)p.Hkv);
     const float scale = d->scale > 0.f ? d->scale : 1.0f / sqrtf((float)d->head_dim);
     p.scale_log2 = scale * 1.4426950408889634f;
     p.stages = tune.stages >= 2 ? (tune.stages > MAX_STAGES ? MAX_STAGES : tune.stages) : 3;   // 3 x 32 KB of K and V (plus q rows): 2 CTAs per SM
@@ -274,7 +287,7 @@ static hg_status run_merge(const hg_partial_src* src, int32_t n_src, float* out,
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3((unsigned)(rows * cluster));
-    const bool big_cta = cluster == 1 && p.total > 64;             // many long rows: 32 warps per row instead
+    const bool big_cta = cluster == 1 && p.total > 256;            // many very long rows: 32 warps per row instead
     cfg.blockDim = dim3(big_cta ? 1024 : 256);
     cfg.stream = static_cast<cudaStream_t>(stream);
     cudaLaunchAttribute attr[2];

@@ -44,7 +44,19 @@ constexpr int PERSIST_CHUNK_PAGES = 256;   // ... for the persistent schedule (p
 constexpr int PERSIST_MAX_BATCH = 1024;    // sequences the in-kernel item scan handles (its table is 4 bytes each; two CTAs
                                            // of three 34 KB stages leave an SM about 2 KB of shared memory to spare)
 
+constexpr int RANGE_CACHE = 128;           // sequences whose slice bounds are kept in shared memory
+
 enum { MODE_MHA = 0, MODE_GQA = 1, MODE_PROBE = 2, MODE_GQA2 = 3 };   // GQA2: items of 16 query heads (two MMA head blocks)
+
+// Division of a non-negative 31-bit number by a launch constant: n / d = umulhi(n, mul) >> shift with
+// mul = ceil(2^(31 + s) / d), s = ceil(log2 d), shift = s - 1 (exact for n < 2^31); d = 1 is flagged by mul = 0.
+// The producer warp divides several times per work item; a hardware-less 32-bit division costs it ~100 cycles each.
+struct FastDiv {
+    uint32_t mul, shift;
+};
+__device__ __forceinline__ int fast_div(int n, FastDiv f) {
+    return f.mul ? (int)(__umulhi((uint32_t)n, f.mul) >> f.shift) : n;
+}
 
 struct PartialParams {
     const void* q;
@@ -67,6 +79,7 @@ struct PartialParams {
     int32_t* sched;           // two zeroed words: [0] hands out items dynamically, [1] counts the CTAs that are done
                               // drawing (NULL: round-robin)
     float scale_log2;         // logit scale * log2(e)
+    FastDiv div_C, div_Hkv;   // division by chunk_tokens and by the number of KV heads
 #ifdef HG_TRACE
     long long* trace;         // development builds only: 8 timestamps / counters per CTA
 #endif
@@ -93,6 +106,8 @@ struct Control {
     float red_l[2][64];                  // double-buffered by item parity
     int scan[8];                         // per-warp totals of the set-up scan
     int cum[PERSIST_MAX_BATCH + 1];      // cum[b] = number of items of sequences < b
+    int2 rng[RANGE_CACHE];               // clamped slices [tb, te) of the first sequences (all of them in a usual batch):
+                                         // the producer decodes an item without going back to global memory
 };
 static_assert(PERSIST_CHUNK_PAGES <= MAX_CHUNK_PAGES / 2, "page-id double buffer");
 
@@ -114,7 +129,12 @@ __device__ __forceinline__ int seq_chunks(const PartialParams& p, int b, int& tb
     tb = max(p.tok_begin[b], 0);
     te = min(min(p.tok_end[b], p.seq_lens[b]), table_reach(p));
     if (te <= tb) return 0;
-    return min((te + p.C - 1) / p.C - tb / p.C, p.NC);
+    return min(fast_div(te + p.C - 1, p.div_C) - fast_div(tb, p.div_C), p.NC);
+}
+
+// Chunk slots in use by a clamped slice [tb, te).
+__device__ __forceinline__ int chunks_of(const PartialParams& p, int tb, int te) {
+    return te <= tb ? 0 : min(fast_div(te + p.C - 1, p.div_C) - fast_div(tb, p.div_C), p.NC);
 }
 
 // True when sequence b's slice reaches past the last page its block-table row can name.
@@ -123,7 +143,7 @@ __device__ __forceinline__ bool range_beyond_table(const PartialParams& p, int b
 }
 
 __device__ __forceinline__ void set_range(const PartialParams& p, Item& it, int tb, int te) {
-    const int first = tb / p.C;
+    const int first = fast_div(tb, p.div_C);
     it.lo = max((first + it.c) * p.C, tb);
     it.hi = min((first + it.c + 1) * p.C, te);
     it.tile0 = it.lo / TILE_T;
@@ -141,13 +161,13 @@ __device__ __forceinline__ Item decode_item(const PartialParams& p, const Contro
     }
     Item it;
     it.b = lo;
-    int tb, te;
-    const int nc = max(seq_chunks(p, lo, tb, te), 1);
+    int tb, te, nc;
+    if (lo < RANGE_CACHE) { tb = ctl.rng[lo].x; te = ctl.rng[lo].y; nc = max(chunks_of(p, tb, te), 1); }
+    else nc = max(seq_chunks(p, lo, tb, te), 1);
     const int r = i - ctl.cum[lo];
     if (p.head_blocks == 1) {
-        const int Y = p.Hkv;
-        it.c = r / Y;                     // KV heads vary fastest: CTAs that run side by side read the same pages
-        it.y = r - it.c * Y;
+        it.c = fast_div(r, p.div_Hkv);    // KV heads vary fastest: CTAs that run side by side read the same pages
+        it.y = r - it.c * p.Hkv;
     } else {
         // groups of more than 8 query heads: the head blocks of one (KV head, chunk) sit next to each other in the
         // order, so they are taken at about the same time and the second reader finds part of the tiles in L2
@@ -216,7 +236,7 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
     // means: do not queue behind it), and this CTA's second work item (its first is its own block index).
     const int32_t status_at_entry = p.status ? *reinterpret_cast<volatile int32_t*>(p.status) : HG_DEV_OK;
     int early_request = 0;
-    if (tid == CONSUMER_THREADS && p.persistent && p.sched && !p.test_stall) early_request = (int)gridDim.x + atomicAdd(p.sched, 1);
+    if (tid == CONSUMER_THREADS && p.persistent && p.sched && !p.test_stall) early_request = atomicAdd(p.sched, 1);   // (raw ticket)
 
     // ---- for the persistent schedule the item counts per sequence -------------------------------------------
     int n_items = 1, item_step = 1, item_first = 0;
@@ -227,7 +247,12 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
         const int b0 = min(p.B, tid * per), b1 = min(p.B, b0 + per);
         int sum = 0;
         bool beyond = false;
-        for (int b = b0; b < b1; ++b) { int tb, te; sum += seq_chunks(p, b, tb, te) * Y; beyond |= range_beyond_table(p, b); }
+        for (int b = b0; b < b1; ++b) {
+            int tb, te;
+            sum += seq_chunks(p, b, tb, te) * Y;
+            beyond |= range_beyond_table(p, b);
+            if (b < RANGE_CACHE) ctl.rng[b] = make_int2(tb, te);
+        }
         if (beyond && p.status && blockIdx.x == 0) atomicOr(p.status, HG_DEV_RANGE);
         int incl = sum;
 #pragma unroll
@@ -321,7 +346,7 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
         // block-table entry of logical page pg of the item's sequence if the page overlaps [lo, hi), else -2
         // (the value is only loaded here; check_page() validates it once it is needed)
         auto lookup = [&](const Item& it, int pg) -> int {
-            if (pg * p.page_size < it.hi && (pg + 1) * p.page_size > it.lo && pg < p.max_pages)
+            if ((pg << p.page_shift) < it.hi && ((pg + 1) << p.page_shift) > it.lo && pg < p.max_pages)
                 return p.block_table ? __ldg(p.block_table + (size_t)it.b * p.max_pages + pg) : it.b * p.max_pages + pg;
             return -2;                                   // no token of the item on this page
         };
@@ -341,12 +366,21 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
         // in `raw` until it is needed, so that the atomic's round trip overlaps the current item's loads.
         // (dynamic schedule: every CTA starts with the item of its own block index, the counter hands out
         // the items from gridDim.x on)
+        // (With the dynamic schedule request() hands back the counter's raw ticket and nothing is computed from it
+        // until settle(): an instruction that depends on the atomic's answer would stall the warp, which issues in
+        // order, for the whole round trip to the L2 - a couple of thousand cycles under load.)
         auto request = [&](int k) -> int {
             if (!p.persistent) return k == 0 ? 0 : n_items;
-            if (dynamic) return k == 0 ? (int)blockIdx.x : (k == 1 ? early_request : (lane == 0 ? (int)gridDim.x + atomicAdd(p.sched, 1) : 0));
+            if (dynamic) {
+                if (k == 0) return (int)blockIdx.x;
+                if (k == 1) return early_request;
+                int raw = 0;
+                if (lane == 0) raw = atomicAdd(p.sched, 1);
+                return raw;
+            }
             return (int)blockIdx.x < item_step ? (int)blockIdx.x + k * item_step : n_items;   // round-robin over item_step CTAs
         };
-        auto settle = [&](int raw) -> int { return dynamic ? __shfl_sync(0xffffffffu, raw, 0) : raw; };
+        auto settle = [&](int raw) -> int { return dynamic ? (int)gridDim.x + __shfl_sync(0xffffffffu, raw, 0) : raw; };
 
 #ifdef HG_TRACE
         long long trace_wait = 0, trace_look = 0;
@@ -395,7 +429,8 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
 #pragma unroll
                     for (int u = 0; u < PER_LANE; ++u) {
                         const int idx = u * 32 + lane;
-                        nxt_ids[u] = idx < nxt_npages ? lookup(nxt, np0 + idx) : -2;
+                        nxt_ids[u] = -2;
+                        if (u * 32 < nxt_npages && idx < nxt_npages) nxt_ids[u] = lookup(nxt, np0 + idx);   // (the first test is warp-uniform)
                     }
                 }
 #ifdef HG_TRACE
@@ -547,7 +582,7 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
         // CTA is unwinding).  d receives the stage's descriptor.
 #ifdef HG_TRACE
         bool traced_first = false;
-        long long ctrace_wait = 0, ctrace_c0 = 0, ctrace_epi = 0, ctrace_sync = 0, ctrace_begin = 0;
+        long long ctrace_wait = 0, ctrace_c0 = 0, ctrace_epi = 0, ctrace_sync = 0, ctrace_begin = 0, ctrace_park = 0;
 #endif
         uint32_t missing = 0u;     // of the stage just received: bit (sub * 2 * boxes per tile + box) = that K/V box is absent
         auto next_stage = [&](int2& d) -> int {
@@ -760,6 +795,9 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
 #endif
                 if (d.y == 0) {
                     begin_item(s);
+#ifdef HG_TRACE
+                    ctrace_sync += clock64() - tb0;      // (development: the begin_item() part of an item's start)
+#endif
                     // b0 = q[head quad][16 ks + 2 tq + {0,1}], b1 = the same + 8; heads past the group read as zero
 #pragma unroll
                     for (int nb = 0; nb < NB; ++nb) {
@@ -787,7 +825,7 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
                     }
                 }
 #ifdef HG_TRACE
-                ctrace_begin += clock64() - tb0;
+                if (d.y == 0) ctrace_begin += clock64() - tb0;
 #endif
                 bool wrote = false;
                 for (int sub = 0; sub < SUB && d.y + sub < cur.ntiles; ++sub) {
@@ -944,12 +982,9 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
                     }
                 }
 #ifdef HG_TRACE
-                const long long ts0 = clock64();
+                ctrace_park += clock64() - te0;
 #endif
                 if (!consumer_sync()) break;
-#ifdef HG_TRACE
-                ctrace_sync += clock64() - ts0;
-#endif
                 // thread -> (head, D/16 consecutive components): the four warp states of one head, weighted
 #pragma unroll
                 for (int nb = 0; nb < NB; ++nb) {
@@ -992,7 +1027,7 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
 #ifdef HG_TRACE
         if (tid == 0 && p.trace) {
             long long* ex = p.trace + (size_t)gridDim.x * 8 + (size_t)gridDim.x * 128 + (size_t)blockIdx.x * 8;
-            ex[2] = ctrace_wait; ex[3] = clock64() - ctrace_c0; ex[4] = ctrace_epi; ex[5] = ctrace_sync; ex[6] = ctrace_begin;
+            ex[2] = ctrace_wait; ex[3] = clock64() - ctrace_c0; ex[4] = ctrace_epi; ex[5] = ctrace_sync; ex[6] = ctrace_begin; ex[0] = ctrace_park;
         }
 #endif
     }
