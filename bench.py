@@ -40,10 +40,10 @@ LARGE = ("opt13b", "opt30b", "llama70b", "ragged")
 # (absent until a capture of that workload exists).  Traffic grows in proportion to the tokens processed, so a
 # capture of the first sequences is scaled to the full launch.
 NCU_TRAFFIC_BYTES = {
-    "opt13b": 4 * (805_546_496 + 5_009_664),          # two of the eight sequences captured, x 4
-    "llama70b": 1_718_226_000 + 7_822_080,            # the full launch captured
-    "opt30b": 4 * (1_879_144_000 + 3_870_464),        # one of the four sequences captured, x 4
-    "ragged": 951_494_144 + 8_356_864,                # the full launch captured
+    "opt13b": 4 * (805_556_224 + 4_392_704),          # two of the eight sequences captured, x 4
+    "llama70b": 1_718_274_000 + 7_049_984,            # the full launch captured
+    "opt30b": 4 * (1_879_137_000 + 3_563_520),        # one of the four sequences captured, x 4
+    "ragged": 951_496_448 + 6_386_432,                # the full launch captured
 }
 
 
@@ -633,7 +633,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", default="all", help="one of tiny, opt13b, opt30b, llama70b, ragged; or all (default)")
+    ap.add_argument("--workload", default="all", help="one of tiny, opt13b, opt30b, llama70b, ragged; all (default); or handoff (the hand-off kernel alone)")
     ap.add_argument("--repeats", type=int, default=5, help="times the K-step pass is repeated per workload")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=0, help="keep only the first BATCH sequences (small profiling captures)")
@@ -685,6 +685,9 @@ def main():
 
     # the group-query configurations first: their consumer warps are the most clock-sensitive, and the 7.5 GB
     # configuration leaves the board at its power cap for the measurements that follow it
+    if args.workload == "handoff":              # only the hand-off kernel (profiling captures); not a bench line
+        print(json.dumps({"handoff": time_handoff(R.dev, args.steps)}), flush=True)
+        return
     names = ["tiny", "ragged", "llama70b", "opt13b", "opt30b"] if args.workload == "all" else [args.workload]
     head_name = HEADLINE if args.workload == "all" else args.workload
     sampler = ClockSampler(local_rank) if rank == 0 else None
