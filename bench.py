@@ -483,6 +483,17 @@ def measure_workload(name, args, R, sampler):
     part_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
     merge_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
 
+    # ---- one step at a time: nothing of a step overlaps its neighbours (in the loop above the merge and the next
+    #      partial kernel start inside their predecessors' tails and the next step's first tiles are requested early)
+    iso = []
+    for _ in range(min(K, 20)):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record(stream); step(); b.record(stream)
+        torch.cuda.synchronize()
+        iso.append(a.elapsed_time(b))
+    (iso_ms,) = max_over_ranks([statistics.median(iso)], dev)
+
     # ---- end to end: per-step data in pinned host memory, results read back every step -----------------------
     pin = lambda t: t.cpu().pin_memory()
     q_h, sl_h, tb_h, te_h = pin(prob.q), pin(prob.seq_lens), pin(prob.tok_begin), pin(prob.tok_end)
@@ -548,7 +559,7 @@ def measure_workload(name, args, R, sampler):
                                 "sm_mhz": [sampler.window(r[1], r[2], fallback_all=False)["sm_mhz"] if sampler else None
                                            for r in reps]},
         "kv_tokens_per_s": whole_job_value(tokens, R.world, ms_step),
-        "partial_us": part_ms * 1e3, "merge_us": merge_ms * 1e3,
+        "partial_us": part_ms * 1e3, "merge_us": merge_ms * 1e3, "isolated_step_us": iso_ms * 1e3,
         "kernel_timing": "a second pass of K steps with CUDA events around each kernel; those events keep the merge "
                          "from starting as a programmatic dependent inside the partial kernel's tail, so partial_us + "
                          "merge_us can exceed the step time of the first pass",

@@ -145,6 +145,8 @@ typedef struct hg_attn_desc {
 #define HG_TUNE_NO_MERGE_ROWS 16u    /* hg_attn_merge: never use the warp-per-row kernel */
 #define HG_TUNE_NO_GQA16 32u         /* groups of more than 8 query heads as items of 8 heads, not 16 */
 #define HG_TUNE_NO_HOST_DIRECT 64u   /* hg_attn_decode_host: always stage through the workspace with copies */
+#define HG_TUNE_NO_SPEC_PREFETCH 128u /* a partial kernel launched as a programmatic dependent does not request its
+                                        guessed first tiles into the L2 while it waits for its predecessor */
 
 /* One source of partials for hg_attn_merge (host struct, dev pointers). */
 typedef struct hg_partial_src {

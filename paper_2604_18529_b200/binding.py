@@ -26,7 +26,7 @@ HG_FLAG_SPARSE_EMPTY = 2
 HG_FLAG_COUNTER_CLEAN = 4
 HG_STATIC_SCRATCH_BYTES = 8 << 20
 (HG_TUNE_NO_PERSISTENT, HG_TUNE_NO_DYNAMIC, HG_TUNE_NO_PDL, HG_TUNE_NO_MERGE_CLUSTER, HG_TUNE_NO_MERGE_ROWS,
- HG_TUNE_NO_GQA16, HG_TUNE_NO_HOST_DIRECT) = 1, 2, 4, 8, 16, 32, 64
+ HG_TUNE_NO_GQA16, HG_TUNE_NO_HOST_DIRECT, HG_TUNE_NO_SPEC_PREFETCH) = 1, 2, 4, 8, 16, 32, 64, 128
 
 
 class HgError(RuntimeError):

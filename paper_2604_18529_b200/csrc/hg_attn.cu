@@ -186,6 +186,7 @@ static hg_status launch_partial_t(const CUtensorMap& tk, const CUtensorMap& tv, 
         // no memset sits between this launch and the kernel before it in the stream: launch as a programmatic
         // dependent, so that block scheduling and the input-free part of the set-up overlap that kernel's tail
         p.pdl_wait = 1;
+        p.spec_prefetch = tune.off(HG_TUNE_NO_SPEC_PREFETCH) ? 0 : 6;
         cudaLaunchConfig_t cfg;
         memset(&cfg, 0, sizeof cfg);
         cfg.gridDim = grid; cfg.blockDim = dim3(THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = st;

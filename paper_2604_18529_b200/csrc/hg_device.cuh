@@ -100,6 +100,13 @@ __device__ __forceinline__ void tma_load_5d(void* dst, const CUtensorMap* tm, ui
         : "memory");
 }
 
+// Hint: bring one box of a 5-D tensor into the L2 (nothing lands in shared memory, nothing is waited for).
+__device__ __forceinline__ void tma_prefetch_5d(const CUtensorMap* tm, int c0, int c1, int c2, int c3, int c4) {
+    asm volatile("cp.async.bulk.prefetch.tensor.5d.L2.global.tile [%0, {%1, %2, %3, %4, %5}];"
+                 ::"l"(reinterpret_cast<uint64_t>(tm)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+                 : "memory");
+}
+
 // One tiled 3-D tensor load (c0, the innermost coordinate, must be a multiple of 8 elements: call sites pass 0).
 __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* tm, uint64_t* bar, int c0, int c1, int c2) {
     asm volatile(

@@ -75,7 +75,8 @@ struct PartialParams {
     int persistent;
     int test_stall;           // HG_FLAG_TEST_STALL: the producer never fills a stage
     int sparse_empty;         // HG_FLAG_SPARSE_EMPTY: empty chunk slots get m and l only, their o rows stay untouched
-    int pdl_wait;             // launched as a programmatic dependent: wait for the preceding kernel before reading any input
+    int pdl_wait;             // launched as a programmatic dependent: wait for the preceding kernel before using any input
+    int spec_prefetch;        // stages of the CTA's guessed first item to request into the L2 while waiting (0: none)
     int32_t* sched;           // two zeroed words: [0] hands out items dynamically, [1] counts the CTAs that are done
                               // drawing (NULL: round-robin)
     float scale_log2;         // logit scale * log2(e)
@@ -225,24 +226,10 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
         ctl.abort_flag = 0;
         fence_barrier_init();
     }
-#if __CUDA_ARCH__ >= 900
-    // launched while the kernel before it in the stream was still running: everything above overlapped that
-    // kernel's tail; nothing it may have written is read before this returns
-    if (p.pdl_wait) cudaGridDependencySynchronize();
-#endif
-
-    // Loads whose answers are needed a little later are issued first, so that their round trips overlap the
-    // scan below: the status word (a wait that timed out earlier in this call, or a word the caller left set,
-    // means: do not queue behind it), and this CTA's second work item (its first is its own block index).
-    const int32_t status_at_entry = p.status ? *reinterpret_cast<volatile int32_t*>(p.status) : HG_DEV_OK;
-    int early_request = 0;
-    if (tid == CONSUMER_THREADS && p.persistent && p.sched && !p.test_stall) early_request = atomicAdd(p.sched, 1);   // (raw ticket)
-
-    // ---- for the persistent schedule the item counts per sequence -------------------------------------------
-    int n_items = 1, item_step = 1, item_first = 0;
-    if (p.persistent) {
-        // cum[b+1] = sum_{b' <= b} nc_b' * Y : every thread a contiguous block of sequences, warp scan, then the
-        // warps' totals through shared memory
+    // Item counts per sequence for the persistent schedule: cum[b+1] = sum_{b' <= b} nc_b' * Y.  Every thread takes a
+    // contiguous block of sequences, a warp scan, then the warps' totals through shared memory.  `report`: flag
+    // slices that reach past their block-table row.
+    auto scan_items = [&](bool report) {
         const int per = (p.B + THREADS - 1) / THREADS;
         const int b0 = min(p.B, tid * per), b1 = min(p.B, b0 + per);
         int sum = 0;
@@ -253,7 +240,7 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
             beyond |= range_beyond_table(p, b);
             if (b < RANGE_CACHE) ctl.rng[b] = make_int2(tb, te);
         }
-        if (beyond && p.status && blockIdx.x == 0) atomicOr(p.status, HG_DEV_RANGE);
+        if (report && beyond && p.status && blockIdx.x == 0) atomicOr(p.status, HG_DEV_RANGE);
         int incl = sum;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -271,6 +258,52 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
             ctl.cum[b + 1] = run;
         }
         __syncthreads();
+    };
+
+#if __CUDA_ARCH__ >= 900
+    if (p.pdl_wait) {
+        // Launched while the kernel before it in the stream is still running (its last CTAs, or a merge, are finishing).
+        // Nothing that kernel may have written is USED before the wait below returns; but the time is not wasted:
+        // on a guess at this CTA's first work item - the ranges and the block table as they look right now, which is
+        // what they will be unless that kernel is the one changing them - the item's first K and V boxes are requested
+        // into the L2.  These are hints: every index is bounds-checked, nothing is written, no result depends on what
+        // was read here, and everything is read again, for real, after the wait.
+        if (p.spec_prefetch && p.persistent) {
+            scan_items(false);
+            if (warp == CONSUMER_WARPS && (int)blockIdx.x < ctl.cum[p.B]) {
+                const Item it = decode_item(p, ctl, (int)blockIdx.x);
+                const int rsh = min(p.page_shift, 6), Rr = 1 << rsh, nb = TILE_T >> rsh;
+                const int j = lane & (nb - 1), isv = (lane >> (6 - rsh)) & 1, sub = lane >> (7 - rsh);
+                const int g = it.y / p.head_blocks;
+                for (int t = 0; t < it.ntiles && t < p.spec_prefetch * SUB; t += SUB) {
+                    const int t0j = (it.tile0 + t + sub) * TILE_T + j * Rr;
+                    if (sub < SUB && t + sub < it.ntiles && t0j < it.hi && t0j + Rr > it.lo) {
+                        const int pg = t0j >> p.page_shift;
+                        int phys = -1;
+                        if (pg >= 0 && pg < p.max_pages)
+                            phys = p.block_table ? __ldg(p.block_table + (size_t)it.b * p.max_pages + pg) : it.b * p.max_pages + pg;
+                        if (phys >= 0 && phys < p.num_pages && g >= 0 && g < p.Hkv)
+                            tma_prefetch_5d(isv ? &tmV : &tmK, 0, t0j & (p.page_size - 1), 0, g, phys);
+                    }
+                }
+            }
+            __syncthreads();                 // the guess is done with the tables the real scan is about to rewrite
+        }
+        cudaGridDependencySynchronize();
+    }
+#endif
+
+    // Loads whose answers are needed a little later are issued first, so that their round trips overlap the
+    // scan below: the status word (a wait that timed out earlier in this call, or a word the caller left set,
+    // means: do not queue behind it), and this CTA's second work item (its first is its own block index).
+    const int32_t status_at_entry = p.status ? *reinterpret_cast<volatile int32_t*>(p.status) : HG_DEV_OK;
+    int early_request = 0;
+    if (tid == CONSUMER_THREADS && p.persistent && p.sched && !p.test_stall) early_request = atomicAdd(p.sched, 1);   // (raw ticket)
+
+    // ---- for the persistent schedule the item counts per sequence -------------------------------------------
+    int n_items = 1, item_step = 1, item_first = 0;
+    if (p.persistent) {
+        scan_items(true);
         n_items = ctl.cum[p.B];
         // use only as many CTAs as keeps every CTA's item count equal (+-1); the others only help with the
         // empty slots below

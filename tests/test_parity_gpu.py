@@ -381,7 +381,7 @@ def test_result_does_not_depend_on_the_schedule(G):
     ref = OracleRef(w)
     results = []
     for env in ({}, {"tune": hg.HG_TUNE_NO_DYNAMIC}, {"tune": hg.HG_TUNE_NO_PERSISTENT}, {"tune_stages": 2},
-                {"tune_ctas_per_sm": 1, "tune_stages": 5}, {"tune": hg.HG_TUNE_NO_PDL}):
+                {"tune_ctas_per_sm": 1, "tune_stages": 5}, {"tune": hg.HG_TUNE_NO_PDL}, {"tune": hg.HG_TUNE_NO_SPEC_PREFETCH}):
         prob = DeviceProblem(w, DEV)
         prob.desc = prob.make_desc(w.chunk_tokens, prob.NC, **env)
         prob.step(ref.host_partials_device(DEV))
