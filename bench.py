@@ -500,7 +500,7 @@ def measure_workload(name, args, R, sampler):
     host_h = [tuple(pin(x) for x in src) for src in host]
     out_h = torch.empty(prob.out.shape, dtype=torch.float32).pin_memory()
     lse_h = torch.empty(prob.lse.shape, dtype=torch.float32).pin_memory()
-    ws = torch.empty(pkg.hg_attn_workspace_bytes(prob.desc, 1), dtype=torch.uint8, device=dev)
+    ws = torch.zeros(pkg.hg_attn_workspace_bytes(prob.desc, 1), dtype=torch.uint8, device=dev)   # (zero-filled: see HG_FLAG_COUNTER_CLEAN)
     decode_host = pkg.prepare_decode_host(q_h, prob.kv["k"], prob.kv["v"], sl_h, tb_h, te_h, host_h, out_h, lse_h, ws,
                                           prob.desc)     # arguments marshalled once, as a decode loop would
 

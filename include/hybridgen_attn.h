@@ -71,7 +71,12 @@ typedef enum hg_dtype { HG_DTYPE_F16 = 0, HG_DTYPE_BF16 = 1 } hg_dtype;
                                    ended normally: every call leaves them at zero).  The call then enqueues no
                                    clearing in front of its kernel, which lets the kernel start as a programmatic
                                    dependent of whatever precedes it in the stream.  After a call that reported
-                                   HG_DEV_WAIT_TIMEOUT clear the words yourself before using the flag again. */
+                                   HG_DEV_WAIT_TIMEOUT clear the words yourself before using the flag again.
+                                   hg_attn_decode and hg_attn_decode_static keep their work counter in the workspace
+                                   (the static scratch): there the flag speaks about that counter - pass it only for a
+                                   workspace that was zero-filled before its first use and has been used by this
+                                   library alone since.  hg_attn_decode_host clears the counter on its way in any
+                                   case. */
 
 /* bits the kernels may set in *hg_attn_desc.status (device word, optional; several may be set at once) */
 #define HG_DEV_OK 0

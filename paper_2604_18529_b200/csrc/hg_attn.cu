@@ -486,7 +486,8 @@ static hg_status decode_impl(const void* q, const void* k_cache, const void* v_c
     memset(&dd, 0, sizeof dd);
     memcpy(&dd, desc, desc->struct_size < sizeof dd ? desc->struct_size : sizeof dd);
     dd.struct_size = sizeof dd;
-    dd.sched_counter = reinterpret_cast<int32_t*>(ws + w.sched);       // the workspace provides the work counter
+    dd.sched_counter = reinterpret_cast<int32_t*>(ws + w.sched);       // the workspace provides the work counter, and
+    // HG_FLAG_COUNTER_CLEAN, if given, speaks about that one (a workspace zero-filled before its first use)
     dd.flags |= HG_FLAG_SPARSE_EMPTY;                                  // the chunk partials are private to this call and its merge
     st = run_partial(MODE_MHA, q, k_cache, v_cache, seq_lens, tok_begin, tok_end, o_part, m_part, l_part, nullptr, stream, &dd,
                      counter_is_zero);

@@ -417,6 +417,14 @@ def test_every_call_leaves_the_work_counter_at_zero(G):
     for a, b in zip(want, (prob.o_part, prob.m_part, prob.l_part, prob.out, prob.lse)):
         assert torch.equal(a, b)
     check_output(prob.out, prob.lse, ref.out, ref.lse)
+    # the fused entry point keeps its counter in the workspace: with the flag, a zero-filled workspace serves call after call
+    ws = torch.zeros(pkg.hg_attn_workspace_bytes(prob.desc, 2), dtype=torch.uint8, device=DEV)
+    for _ in range(3):
+        out, lse = torch.full_like(prob.out, float("nan")), torch.full_like(prob.lse, float("nan"))
+        pkg.hg_attn_decode(prob.q, prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end,
+                           ref.host_partials_device(DEV), out, lse, ws, prob.desc)
+        torch.cuda.synchronize()
+        assert torch.equal(out, want[3]) and torch.equal(lse, want[4])
 
 
 def test_without_a_work_counter_items_are_dealt_round_robin():
