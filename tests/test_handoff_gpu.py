@@ -102,6 +102,43 @@ def test_handoff_partials_and_merged_result(G, D, dtype, keep, chunk):
     assert np.abs(lse - ref_lse).max() <= LSE_ABS
 
 
+@pytest.mark.parametrize("G,D,dtype,K,chunk", [(1, 64, "f16", 77, 96), (16, 64, "bf16", 333, 96), (3, 128, "f16", 1025, 1024),
+                                               (8, 128, "bf16", 2049, 160), (5, 128, "f16", 64, 64)])
+def test_handoff_odd_sizes(G, D, dtype, K, chunk):
+    """Row lengths that are not a multiple of anything (logit rows at odd offsets take the scalar load path, V tiles
+    straddle the end of a chunk and of the whole array), chunk sizes that are not a multiple of the 64-row tile, groups
+    that fill one and a half or two head blocks, empty sequences and sequences that use every slot."""
+    rng = np.random.default_rng(K + G)
+    B, Hkv = 3, 2
+    Hq = Hkv * G
+    n_sel = np.array([K, 0, max(1, K // 3)], dtype=np.int32)
+    logits = (rng.standard_normal((B, Hq, K)) * 3.0).astype(np.float32)
+    logits[0, 0, ::5] = -np.inf                                     # a head that drops slots
+    v = (rng.standard_normal((B, Hkv, K, D)) * 2.0).astype(np.float32)
+    vt = torch.from_numpy(v).to(torch.float16 if dtype == "f16" else torch.bfloat16)
+    vbits = bits(vt)
+    for b in range(B):                                              # rows past n_sel: NaN patterns that must never matter
+        vbits[b, :, n_sel[b]:] = 0x7E00 if dtype == "f16" else 0x7FC0
+    NCs = -(-K // chunk)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    desc = pkg.logits_desc(batch=B, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, dtype=dtype, max_selected=K,
+                           chunk_tokens=chunk, num_chunks=NCs, status=status)
+    lg = torch.from_numpy(logits).to(DEV)
+    vr = torch.from_numpy(vbits.view(np.int16)).to(DEV)
+    ho = torch.full((B, Hq, NCs, D), 5.0, device=DEV); hm = torch.full((B, Hq, NCs), 5.0, device=DEV); hl = torch.full_like(hm, 5.0)
+    pkg.hg_attn_partial_from_logits(lg, vr, torch.from_numpy(n_sel).to(DEV), ho, hm, hl, desc)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    rm = np.full((B, Hq, NCs), -np.inf); rl = np.zeros((B, Hq, NCs)); ro = np.zeros((B, Hq, NCs, D))
+    for b in range(B):
+        for h in range(Hq):
+            for c in range(NCs):
+                a, e = c * chunk, min((c + 1) * chunk, int(n_sel[b]))
+                if e > a:
+                    rm[b, h, c], rl[b, h, c], ro[b, h, c] = O.partial_from_logits(logits[b, h, a:e].astype(np.float64), vbits[b, h // G, a:e], dtype)
+    check_partials(ho.reshape(-1, D), hm.reshape(-1), hl.reshape(-1), rm.reshape(-1), rl.reshape(-1), ro.reshape(-1, D))
+
+
 def test_handoff_rejects_bad_descriptions():
     from paper_2604_18529_b200 import binding as hg
     t = torch.zeros(8, device=DEV)
