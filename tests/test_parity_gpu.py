@@ -372,6 +372,49 @@ def test_slice_beyond_the_block_table_is_cut_and_reported(G, persistent):
                    rm.reshape(-1), rl.reshape(-1), ro.reshape(-1, w.D), "beyond table")
 
 
+# ---- bit patterns the seeded generator never produces -----------------------------------------------------------
+
+@pytest.mark.parametrize("G,dtype", [(1, "f16"), (1, "bf16"), (4, "f16"), (8, "bf16")])
+def test_subnormals_zeros_and_large_values_in_the_cache(G, dtype):
+    """The generator draws from a table of normal quantiles: no subnormal, no signed zero, nothing beyond 4.4 sigma.  Here a
+    tenth of the resident K and V elements and a few q elements are overwritten with such patterns (subnormals of either
+    sign, -0, the smallest normals, values up to +-48); the oracle decodes the same bits exactly, and the GPU path - the
+    fp32 unpacking of the one-head kernel as well as the tensor-core operands of the group-query one - must agree."""
+    from oracle import hg_oracle as O
+    w = wl(B=2, Hq=2 * G, Hkv=2, D=128, dtype=dtype, seq_lens=[700, 333], tok_begin=[130, 5], tok_end=[700, 290], seed=120 + G)
+    prob = DeviceProblem(w, DEV)
+    gen = torch.Generator(device=DEV).manual_seed(5)
+    if dtype == "f16":
+        special = [0x0001, 0x8001, 0x03FF, 0x83FF, 0x8000, 0x0400, 0x8400, 0x5200, 0xD200, 0x4E00]   # subnormals, -0, 2^-14, +-48, 24
+    else:
+        special = [0x0001, 0x8001, 0x007F, 0x807F, 0x8000, 0x0080, 0x8080, 0x4240, 0xC240, 0x41C0]   # the same for bf16
+    pat = torch.tensor(special, dtype=torch.int32, device=DEV)
+    for pool in (prob.kv["k"], prob.kv["v"], prob.q):
+        flat = pool.view(torch.int16).view(-1)
+        hit = torch.rand(flat.numel(), device=DEV, generator=gen) < (0.1 if pool is not prob.q else 0.02)
+        pick = pat[torch.randint(0, len(special), (flat.numel(),), device=DEV, generator=gen)]
+        flat[hit] = pick[hit].to(torch.int16)
+    # the logical cache as the block table maps it (pages of the slice only; the rest is never read)
+    ps, table = w.page_size, prob.kv["block_table"].cpu()
+    K = np.zeros((w.B, w.max_len, w.Hkv, w.D), dtype=np.uint16); V = np.zeros_like(K)
+    kp, vp = bits(prob.kv["k"]), bits(prob.kv["v"])                         # [pages][Hkv][ps][D]
+    for b in range(w.B):
+        for pg in range(w.tok_begin[b] // ps, -(-w.tok_end[b] // ps)):
+            n = min(ps, w.max_len - pg * ps)
+            K[b, pg * ps: pg * ps + n] = kp[int(table[b, pg])].transpose(1, 0, 2)[:n]
+            V[b, pg * ps: pg * ps + n] = vp[int(table[b, pg])].transpose(1, 0, 2)[:n]
+    q = bits(prob.q)
+    prob.step([])
+    torch.cuda.synchronize()
+    assert int(prob.status.item()) == hg.HG_DEV_OK
+    rm, rl, ro = O.chunked_partials(q, K, V, dtype, w.tok_begin, w.tok_end, w.chunk_tokens, prob.NC)
+    check_partials(prob.o_part.reshape(-1, w.D), prob.m_part.reshape(-1), prob.l_part.reshape(-1),
+                   rm.reshape(-1), rl.reshape(-1), ro.reshape(-1, w.D), "special values")
+    ref_out, ref_lse = O.full_batch(q, K, V, dtype, w.tok_begin, w.tok_end)
+    check_output(prob.out, prob.lse, ref_out, ref_lse, "special values")
+    assert np.abs(ref_out).max() > 1.0          # the large values do reach the output
+
+
 # ---- schedules: persistent-dynamic, persistent-static and one-CTA-per-item give the same bits --------------------
 
 @pytest.mark.parametrize("G", [1, 4])
