@@ -440,9 +440,10 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
 #endif
             const int page0 = first_page(cur);
             const int* const pages = &ctl.pages[(k & 1) * (MAX_CHUNK_PAGES / 2)];
-            // the next item (its index was requested one item ago) is looked at right after this item's first
-            // stage has been issued: the request for the item after it goes out, and the next item's page ids
-            // start loading (they are parked in shared memory once this item's loads have all been issued)
+            // the next item (its index was requested one item ago) is looked at the first time this item's loads have
+            // to wait for a ring slot (at the item's end at the latest): the request for the item after it goes out, and
+            // the next item's page ids start loading (they are parked in shared memory once this item's loads have all
+            // been issued)
             int i_nxt = n_items;
             bool has_next = false;
             Item nxt = cur;
@@ -473,46 +474,61 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
             const int g = cur.y / p.head_blocks;
             const int q_heads = GQA ? min(HPI, p.G - (cur.y % p.head_blocks) * HPI) : 1;
             const int q_head0 = GQA ? g * p.G + (cur.y % p.head_blocks) * HPI : g;
+            bool looked = false;                                   // the look-ahead for the next item has been done
             for (int it = 0; it < cur.ntiles; it += SUB) {         // one stage = SUB x (K tile + V tile of 64 tokens)
-                int okw = 1;
-#ifdef HG_TRACE
-                const long long tw0 = clock64();
-#endif
-                if (lane == 0) okw = mbar_wait(&ctl.empty[s], ph ^ 1u, abort_flag) ? 1 : 0;
-#ifdef HG_TRACE
-                trace_wait += clock64() - tw0;
-#endif
-                okw = __shfl_sync(0xffffffffu, okw, 0);
-                if (!okw) { alive = false; break; }
+                // Everything that does not need the ring slot comes first, so that a slot that frees up while this is
+                // computed is re-armed the moment the wait returns: the time a slot spends neither in flight nor in
+                // use comes straight off the bytes in flight (300 cycles more per stage cost the 16-token-page
+                // group-query workloads 2 - 2.6 % when it was tried).
                 const int t0j = (cur.tile0 + it + sub) * TILE_T + j * R;
+                const bool wanted = sub < SUB && it + sub < cur.ntiles && t0j < cur.hi && t0j + R > cur.lo;
                 int phys = -1;
-                if (sub < SUB && it + sub < cur.ntiles && t0j < cur.hi && t0j + R > cur.lo) phys = pages[(t0j >> p.page_shift) - page0];
+                if (wanted) phys = pages[(t0j >> p.page_shift) - page0];
                 const uint32_t nvalid = __popc(__ballot_sync(0xffffffffu, phys >= 0));   // K and V boxes
                 // boxes the item has tokens in but whose page id was refused: their rows must not enter the result
-                const bool wanted = sub < SUB && it + sub < cur.ntiles && t0j < cur.hi && t0j + R > cur.lo;
                 const uint32_t missing = __ballot_sync(0xffffffffu, wanted && phys < 0 && !isv) & 0xffffu;
                 // (items of 16 heads fetch their query rows themselves: the stage's q slot holds 8)
                 const uint32_t qbytes = (MODE != MODE_PROBE && NB == 1 && it == 0) ? (uint32_t)q_heads * D * 2u : 0u;
+                uint8_t* const dst = stage0_ptr + (size_t)s * STAGE_BYTES + sub * PAIR_BYTES + isv * TILE_BYTES + j * box_bytes;
+                const int c1 = t0j & (p.page_size - 1);
+
+                // the slot: if it is not free yet, the wait is the time for the next item's look-ahead
+                int ready = 1;
+                if (lane == 0) ready = mbar_try_wait(&ctl.empty[s], ph ^ 1u) ? 1 : 0;
+                ready = __shfl_sync(0xffffffffu, ready, 0);
+                if (!ready) {
+                    if (!looked && it > 0) { look_ahead(); looked = true; }
+                    int okw = 1;
+#ifdef HG_TRACE
+                    const long long tw0 = clock64();
+#endif
+                    if (lane == 0) okw = mbar_wait(&ctl.empty[s], ph ^ 1u, abort_flag) ? 1 : 0;
+#ifdef HG_TRACE
+                    trace_wait += clock64() - tw0;
+#endif
+                    okw = __shfl_sync(0xffffffffu, okw, 0);
+                    if (!okw) { alive = false; break; }
+                }
                 if (lane == 0) {
                     ctl.sdesc[s] = make_int2(i_cur, it | (int)(missing << 16));
                     if (it == 0) sitem[s] = cur;
                     mbar_arrive_expect_tx(&ctl.full[s], nvalid * box_bytes + qbytes);
                 }
-                __syncwarp();
+                // (no warp barrier here: bytes that land before the arrival above is counted cannot complete the phase,
+                // the arrival itself is still outstanding)
                 if (qbytes && lane == 31)        // the item's query rows travel with its first stage
                     bulk_load(stage0_ptr + (size_t)s * STAGE_BYTES + SUB * PAIR_BYTES,
                               reinterpret_cast<const uint16_t*>(p.q) + ((size_t)cur.b * p.Hq + q_head0) * D, qbytes, &ctl.full[s]);
-                if (phys >= 0) {
-                    uint8_t* dst = stage0_ptr + (size_t)s * STAGE_BYTES + sub * PAIR_BYTES + isv * TILE_BYTES + j * box_bytes;
-                    tma_load_5d(dst, isv ? &tmV : &tmK, &ctl.full[s], 0, t0j & (p.page_size - 1), 0, g, phys, policy);
-                }
+                if (phys >= 0) tma_load_5d(dst, isv ? &tmV : &tmK, &ctl.full[s], 0, c1, 0, g, phys, policy);
+#ifdef HG_PRODUCER_DELAY
+                { const long long d0 = clock64(); while (clock64() - d0 < HG_PRODUCER_DELAY) { } }
+#endif
                 if (issued == 0 && lane == 0) HG_TRACE_AT(2);
                 ++issued;
                 if (++s == p.stages) { s = 0; ph ^= 1u; }
-                if (it == 0) look_ahead();
             }
             if (!alive) break;
-            if (cur.ntiles == 0) look_ahead();
+            if (!looked) look_ahead();                             // the producer never had to wait during this item
             if (!has_next) break;
             int* const dstp = &ctl.pages[((k + 1) & 1) * (MAX_CHUNK_PAGES / 2)];
 #pragma unroll
