@@ -48,7 +48,6 @@ constexpr size_t logits_smem_bytes(int chunk) {
 
 template <int D, bool BF16>
 __global__ void __launch_bounds__(LG_THREADS, 3) logits_partial_kernel(const __grid_constant__ CUtensorMap tmV, const LogitsParams p) {
-    constexpr int HALVES = D / 64;
     constexpr int TILE_BYTES = LG_TILE * D * 2;
     constexpr int MT = D / 16;                        // 16-component blocks of D: one per warp of a set
     constexpr int SETS = LG_WARPS / MT;               // warp sets taking alternate 16-token steps (1 or 2)
@@ -101,7 +100,7 @@ __global__ void __launch_bounds__(LG_THREADS, 3) logits_partial_kernel(const __g
     for (int hb = 0; hb < head_blocks; ++hb) {
         const int h0 = g * p.G + hb * 8, nh = min(8, p.G - hb * 8);
         // ---- warp h: head h's logits -> m, l and the P fragments -------------------------------------------
-        if (hb > 0) __syncthreads();                                   // the previous block's fragments have been used
+        if (hb > 0) __syncthreads();          // the previous block's m and l have been written out (reached by all: see below)
         {
             // a lane owns token pairs (2u, 2u + 1), u = lane + 32 i: coalesced 8-byte loads, once for the maximum and
             // once more (out of the cache) for the weights
@@ -165,12 +164,16 @@ __global__ void __launch_bounds__(LG_THREADS, 3) logits_partial_kernel(const __g
             if (!ok) break;
             const uint32_t vbase = tile0 + s * TILE_BYTES;
             if ((ti + 1) * LG_TILE > nt) {
-                // rows past the chunk's last slot hold whatever lies behind it (other slots, NaN patterns): clear them
-                for (int u = tid; u < LG_TILE * 8 * HALVES; u += LG_THREADS) {
-                    const int r = u / (8 * HALVES), cc = u % (8 * HALVES);
-                    if (ti * LG_TILE + r >= nt) sts128_zero(vbase + (cc >> 3) * (128u * LG_TILE) + r * 128u + ((cc & 7) << 4));
+                // Rows past the chunk's last slot hold whatever lies behind it (other slots, NaN patterns).  Every warp
+                // clears the part of them that it reads itself - its two 16-byte columns of the rows of its own
+                // 16-token steps - so no warp depends on another here (a barrier inside this loop could be left
+                // waiting by a warp whose bounded wait ran out).
+                for (int u = lane; u < LG_TILE * 2; u += 32) {
+                    const int r = u >> 1, cc = 2 * mt + (u & 1);
+                    if (ti * LG_TILE + r >= nt && ((r >> 4) % SETS) == set)
+                        sts128_zero(vbase + (cc >> 3) * (128u * LG_TILE) + r * 128u + (((cc & 7) ^ (r & 7)) << 4));
                 }
-                __syncthreads();
+                __syncwarp();
             }
 #pragma unroll
             for (int k4 = set; k4 < LG_TILE / 16; k4 += SETS) {
@@ -187,13 +190,16 @@ __global__ void __launch_bounds__(LG_THREADS, 3) logits_partial_kernel(const __g
                 if (mbar_wait(&empty[s], (uint32_t)(it / LG_STAGES) & 1u, abort_flag)) { issue(it + LG_STAGES); ++issued; }
             }
         }
-        if (!ok) break;
         // ---- results: acc[0], acc[1]: component 16 mt + quad, heads 2tq, 2tq + 1; acc[2], acc[3]: component + 8 ----
+        float* const s_add = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(s_frag) +
+                                                      (size_t)((p.chunk + LG_TILE - 1) / LG_TILE * LG_TILE / 16) * 512);
         if constexpr (SETS == 2) {
-            float* const s_add = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(s_frag) +
-                                                          (size_t)((p.chunk + LG_TILE - 1) / LG_TILE * LG_TILE / 16) * 512);
             if (set == 1) *reinterpret_cast<float4*>(s_add + (mt * 32 + lane) * 4) = make_float4(acc[0], acc[1], acc[2], acc[3]);
-            __syncthreads();
+        }
+        // every warp gets here, whatever became of its waits: the verdict is made uniform at this barrier, so that
+        // all warps leave together or none does
+        if (!__syncthreads_and(ok ? 1 : 0)) break;
+        if constexpr (SETS == 2) {
             if (set == 0) {
                 const float4 x = *reinterpret_cast<const float4*>(s_add + (mt * 32 + lane) * 4);
                 acc[0] += x.x; acc[1] += x.y; acc[2] += x.z; acc[3] += x.w;
