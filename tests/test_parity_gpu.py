@@ -500,6 +500,49 @@ def test_chunks_with_many_pages_use_the_per_item_grid():
     run_and_check(w)
 
 
+@pytest.mark.parametrize("G,layout", [(1, "HND"), (4, "HND"), (4, "NHD")])
+def test_pages_above_four_gib_in_the_pool(G, layout):
+    # pools of 6 GiB each whose live pages are the last ones: page offsets need more than 32 bits, in bytes and in
+    # elements; everything below the live pages is uninitialised memory that no box may touch
+    w = wl(Hq=2 * G, Hkv=2, page_size=64, layout=layout, chunk_tokens=256, seq_lens=[1500, 777], tok_begin=[70, 0],
+           tok_end=[1500, 700], seed=79)
+    small = w.build_device_kv(DEV)
+    page_elems = small["page_stride"]
+    total_pages = (6 << 30) // (2 * page_elems)
+    shift = total_pages - small["num_pages"]
+    assert shift * page_elems > 2**31
+    kv = dict(small)
+    for which in ("k", "v"):
+        big = torch.empty((total_pages,) + tuple(small[which].shape[1:]), dtype=small[which].dtype, device=DEV)
+        big[:64].fill_(float("nan"))
+        big[shift:] = small[which]
+        kv[which] = big
+    table = small["block_table"]
+    kv["block_table"] = torch.where(table >= 0, table + shift, table)
+    kv["num_pages"] = total_pages
+    ref = OracleRef(w)
+    prob = DeviceProblem(w, DEV, kv=kv)
+    prob.partial()
+    prob.merge(ref.host_partials_device(DEV))
+    torch.cuda.synchronize()
+    assert int(prob.status.item()) == hg.HG_DEV_OK
+    rm, rl, ro = ref.chunk_partials(w.chunk_tokens, prob.NC)
+    check_partials(prob.o_part.reshape(-1, w.D), prob.m_part.reshape(-1), prob.l_part.reshape(-1),
+                   rm.reshape(-1), rl.reshape(-1), ro.reshape(-1, w.D))
+    check_output(prob.out, prob.lse, ref.out, ref.lse)
+    # the same through the read probe: the checksum of exactly the slice's bits
+    small_prob = DeviceProblem(w, DEV, kv=small)
+    sinks = []
+    for pr in (prob, small_prob):
+        sink = torch.zeros(w.B, w.Hkv, pr.NC, dtype=torch.int32, device=DEV)
+        pkg.hg_kv_read_probe(pr.kv["k"], pr.kv["v"], pr.seq_lens, pr.tok_begin, pr.tok_end, sink, pr.desc)
+        sinks.append(sink)
+    torch.cuda.synchronize()
+    assert torch.equal(sinks[0], sinks[1])
+    del prob, kv, big
+    torch.cuda.empty_cache()
+
+
 # ---- bounded waits: a stalled pipeline ends with a status code, not a hang -----------------------------------------
 
 @pytest.mark.parametrize("G", [1, 4])
