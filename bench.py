@@ -577,6 +577,9 @@ def measure_workload(name, args, R, sampler):
         rec["step_gbs"] = step_gbs
         rec["step_frac_of_8000"] = step_gbs / 8000.0
         rec["step_frac_of_probe"] = probe_us / (ms_step * 1e3) if probe_us else None
+        rec["probe"] = ("hg_kv_read_probe: the partial kernel's loads with every word XOR-folded instead of the attention "
+                        "arithmetic, K launches back to back after the other passes; above 1 when the board had reached its "
+                        "power cap by then (the fold is integer work on every word)")
         rec["roofline"] = {"bound": "hbm", "kernel": "partial_kernel", "achieved": achieved, "peak": peak,
                            "peak_kind": f"{peak_kind} copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
                            "frac_of_8000": achieved / 8000.0, "alg_bytes_per_launch": part_alg,
@@ -710,9 +713,10 @@ def main():
     if sampler:
         sampler.start()
         time.sleep(0.3)
+    # (the hand-off kernel's two short measurements come first for the same reason)
+    handoff = time_handoff(R.dev, args.steps) if args.workload == "all" and rank == 0 else None
     recs = {n: measure_workload(n, args, R, sampler) for n in names}
     shard_rec = measure_sharded(args, R) if (world > 1 or args.sharded) and args.workload == "all" else None
-    handoff = time_handoff(R.dev, args.steps) if args.workload == "all" and rank == 0 else None
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()

@@ -692,6 +692,44 @@ def test_sinks_plus_recent_window_as_two_ranges(G):
     check_output(prob.out, prob.lse, ref_out, ref_lse, "sinks + window")
 
 
+@pytest.mark.parametrize("G,page", [(1, 16), (4, 16), (8, 64)])
+def test_selected_pages_through_a_compacted_block_table(G, page):
+    """A page-granular token set (a Pre-QK^T choice of whole pages, say): the caller lists the chosen pages of each
+    sequence in a block table of their own, in token order, and attends the range [0, pages * page_size) of that
+    virtual sequence; the result is attention over exactly the chosen pages' tokens."""
+    from oracle import hg_oracle as O
+    L = [1500, 777]
+    w = wl(Hq=2 * G, Hkv=2, page_size=page, seq_lens=L, tok_begin=[0, 0], tok_end=L, chunk_tokens=256, seed=83)
+    prob = DeviceProblem(w, DEV)
+    rng = np.random.default_rng(83)
+    full_pages = [l // page for l in L]                      # the ragged last page stays out of the choice
+    chosen = [np.sort(rng.choice(n, size=max(1, n // 3), replace=False)) for n in full_pages]
+    chosen[1] = np.union1d(chosen[1], [0, full_pages[1] - 1])
+    width = max(len(c) for c in chosen)
+    table = torch.full((w.B, width), -1, dtype=torch.int32, device=DEV)
+    for b, c in enumerate(chosen):
+        table[b, :len(c)] = prob.kv["block_table"][b, torch.as_tensor(c, device=DEV)]
+    n_tok = [len(c) * page for c in chosen]
+    NC = (max(n_tok) + 255) // 256
+    prob.kv = dict(prob.kv, block_table=table, max_pages=width)
+    desc = prob.make_desc(256, NC)
+    lens = torch.tensor(n_tok, dtype=torch.int32, device=DEV)
+    o = torch.empty(w.B, w.Hq, NC, w.D, device=DEV); m = torch.empty(w.B, w.Hq, NC, device=DEV); l = torch.empty_like(m)
+    hg.hg_attn_partial(prob.q, prob.kv["k"], prob.kv["v"], lens, torch.zeros_like(lens), lens, o, m, l, desc)
+    hg.hg_attn_merge([(o, m, l)], prob.out, prob.lse, desc)
+    torch.cuda.synchronize()
+    assert int(prob.status.item()) == hg.HG_DEV_OK
+    q, K, V = bits(w.q()), bits(w.kv_logical("k")), bits(w.kv_logical("v"))
+    ref_out = np.empty((w.B, w.Hq, w.D)); ref_lse = np.empty((w.B, w.Hq))
+    for b in range(w.B):
+        idx = (chosen[b][:, None] * page + np.arange(page)[None, :]).reshape(-1).astype(np.int64)
+        for h in range(w.Hq):
+            g = h // G
+            ref_out[b, h], ref_lse[b, h] = O.full(q[b, h], np.ascontiguousarray(K[b, :, g]), np.ascontiguousarray(V[b, :, g]),
+                                                   w.dtype, idx=idx)
+    check_output(prob.out, prob.lse, ref_out, ref_lse, "selected pages")
+
+
 @pytest.mark.parametrize("G", [1, 4])
 def test_a_slice_longer_than_num_chunks_is_cut_to_its_first_chunks(G):
     """num_chunks bounds the work: tokens past the last chunk slot are not attended, and what is produced equals attention over the kept range."""
