@@ -98,6 +98,9 @@ typedef enum hg_dtype { HG_DTYPE_F16 = 0, HG_DTYPE_BF16 = 1 } hg_dtype;
  * K and V pools share this addressing.  Only pages that overlap [tok_begin, tok_end) are
  * dereferenced; other block-table entries may be -1.  Whole resident pages may be read,
  * including rows outside the slice, but such rows never influence a result.
+ * "Token t" is a position in the block-table row, nothing more: a row that lists only chosen pages of a
+ * sequence, in token order, with seq_lens / tok_end counted in that row's positions, gives attention over
+ * exactly those pages (a page-granular token selection, Section 4.5, needs no other entry point).
  * Requirements: head_dim in {64, 128}; page_size in {16, 32, 64, 128, 256}; pool base addresses
  * 16-byte aligned; every stride a multiple of 8 elements; chunk_tokens a multiple of 64 and of
  * page_size, at most 512 pages.
