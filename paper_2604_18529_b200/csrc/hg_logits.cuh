@@ -26,7 +26,12 @@ constexpr int LG_THREADS = 256;
 constexpr int LG_WARPS = LG_THREADS / 32;
 constexpr int LG_MAX_CHUNK = 1024;    // selected tokens per chunk
 constexpr int LG_TILE = 64;           // V rows per tile
-constexpr int LG_STAGES = 3;
+constexpr int LG_MIN_CTAS = 5;        // per SM
+// Tiles in flight per CTA: two of 16 KB (D = 128) or three of 8 KB (D = 64, where two and four measured slower).  A CTA streams nothing while it turns its
+// chunk's logits into fragments, so what keeps the V stream going is the number of CTAs that share an SM, not the
+// depth of one CTA's ring: five CTAs with two tiles each run 10-14 % faster than three with three.
+template <int D>
+__host__ __device__ constexpr int lg_stages() { return D == 128 ? 2 : 3; }
 
 struct LogitsParams {
     const float* logits;      // [B][Hq][K]
@@ -38,17 +43,18 @@ struct LogitsParams {
     int B, Hq, Hkv, G, K, chunk, NC;
 };
 
-// Dynamic shared memory: [LG_STAGES] V tiles (64 x D x 2 bytes, 1024-byte aligned), then the P fragments
+// Dynamic shared memory: [lg_stages<D>()] V tiles (64 x D x 2 bytes, 1024-byte aligned), then the P fragments
 // (chunk / 16 steps x 32 lanes x 4 words), then, at D = 64, the second warp set's accumulators.
 template <int D>
 constexpr size_t logits_smem_bytes(int chunk) {
-    return 1024 + (size_t)LG_STAGES * LG_TILE * D * 2 + (size_t)((chunk + LG_TILE - 1) / LG_TILE * LG_TILE / 16) * 512 +
+    return 1024 + (size_t)lg_stages<D>() * LG_TILE * D * 2 + (size_t)((chunk + LG_TILE - 1) / LG_TILE * LG_TILE / 16) * 512 +
            (D == 64 ? 4 * 32 * 4 * sizeof(float) : 0);
 }
 
 template <int D, bool BF16>
-__global__ void __launch_bounds__(LG_THREADS, 3) logits_partial_kernel(const __grid_constant__ CUtensorMap tmV, const LogitsParams p) {
+__global__ void __launch_bounds__(LG_THREADS, LG_MIN_CTAS) logits_partial_kernel(const __grid_constant__ CUtensorMap tmV, const LogitsParams p) {
     constexpr int TILE_BYTES = LG_TILE * D * 2;
+    constexpr int LG_STAGES = lg_stages<D>();
     constexpr int MT = D / 16;                        // 16-component blocks of D: one per warp of a set
     constexpr int SETS = LG_WARPS / MT;               // warp sets taking alternate 16-token steps (1 or 2)
     constexpr float LOG2E = 1.4426950408889634f;
