@@ -78,7 +78,8 @@ def test_gpus_n_starts_its_own_ranks():
     assert d == {"launch_check": True, "world": 2, "ranks_seen": [0, 1], "max_rank": 1.0}
 
 
-def test_gpus_n_without_cuda_fails_in_every_rank_after_the_spawn():
+def test_gpus_n_without_cuda_fails_in_the_ranks_after_the_spawn():
+    import re
     import torch
     if torch.cuda.is_available():
         import pytest
@@ -86,8 +87,11 @@ def test_gpus_n_without_cuda_fails_in_every_rank_after_the_spawn():
     out = _run_bench("--gpus", "2", "--steps", "1")
     assert out.returncode != 0
     assert "starting 2 ranks" in out.stderr
-    for r in (0, 1):
-        assert f"bench.py (rank {r} of 2) needs a CUDA device" in out.stderr
+    # the refusal comes from a rank of the spawned pair, not from the parent (the launcher ends the other rank as soon
+    # as the first one has failed, so not every rank gets to say it; that both ranks start and meet is what
+    # test_gpus_n_starts_its_own_ranks above asserts)
+    assert re.search(r"bench\.py \(rank [01] of 2\) needs a CUDA device", out.stderr)
+    assert "no CPU fallback" in out.stderr
     assert not [l for l in out.stdout.splitlines() if l.startswith("{")]
 
 
