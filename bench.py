@@ -473,6 +473,23 @@ def measure_workload(name, args, R, sampler):
     med = order[(len(order) - 1) // 2]       # the median repeat (the lower one of an even count)
     ms_step = rep_ms[med] / K
 
+    # the read probe: the partial kernel's own loads (same boxes, same ring, same schedule) with no arithmetic - what
+    # this access pattern can reach; K launches back to back between one pair of events, like the steps of pass A,
+    # and right after them (the board is then in the state the steps were timed in)
+    probe_us = None
+    if (w.kv_bytes() > 2 * 126e6 and not args.no_probe) or args.probe:
+        sink = torch.zeros(w.B, w.Hkv, prob.NC, dtype=torch.int32, device=dev)
+        probe = lambda: pkg.hg_kv_read_probe(prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end, sink, prob.desc)
+        for _ in range(3):
+            probe()
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        p0.record(stream)
+        for _ in range(K):
+            probe()
+        p1.record(stream)
+        torch.cuda.synchronize()
+        probe_us = p0.elapsed_time(p1) * 1e3 / K
+
     # ---- pass B: K more steps with an event around every kernel (roofline of the dominant kernel) ----------
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
     tb0 = time.time()
@@ -523,21 +540,6 @@ def measure_workload(name, args, R, sampler):
         sum(t.numel() * t.element_size() for src in host_h for t in src)
     d2h = out_h.numel() * 4 + lse_h.numel() * 4
 
-    # the read probe: the partial kernel's own loads (same boxes, same ring, same schedule) with no arithmetic - what
-    # this access pattern can reach; K launches back to back between one pair of events, like the steps of pass A
-    probe_us = None
-    if (w.kv_bytes() > 2 * 126e6 and not args.no_probe) or args.probe:
-        sink = torch.zeros(w.B, w.Hkv, prob.NC, dtype=torch.int32, device=dev)
-        probe = lambda: pkg.hg_kv_read_probe(prob.kv["k"], prob.kv["v"], prob.seq_lens, prob.tok_begin, prob.tok_end, sink, prob.desc)
-        for _ in range(3):
-            probe()
-        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        p0.record(stream)
-        for _ in range(K):
-            probe()
-        p1.record(stream)
-        torch.cuda.synchronize()
-        probe_us = p0.elapsed_time(p1) * 1e3 / K
     extras = time_extras(w, prob, dev, K) if args.extras and R.rank == 0 and name != "tiny" else None
     if int(prob.status.item()) != 0:
         raise SystemExit(f"{name}: device status {int(prob.status.item())} after the timed passes")
@@ -578,8 +580,7 @@ def measure_workload(name, args, R, sampler):
         rec["step_frac_of_8000"] = step_gbs / 8000.0
         rec["step_frac_of_probe"] = probe_us / (ms_step * 1e3) if probe_us else None
         rec["probe"] = ("hg_kv_read_probe: the partial kernel's loads with every word XOR-folded instead of the attention "
-                        "arithmetic, K launches back to back after the other passes; above 1 when the board had reached its "
-                        "power cap by then (the fold is integer work on every word)")
+                        "arithmetic, K launches back to back right after the timed steps")
         rec["roofline"] = {"bound": "hbm", "kernel": "partial_kernel", "achieved": achieved, "peak": peak,
                            "peak_kind": f"{peak_kind} copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
                            "frac_of_8000": achieved / 8000.0, "alg_bytes_per_launch": part_alg,
