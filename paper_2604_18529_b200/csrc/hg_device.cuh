@@ -72,7 +72,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     }
 }
 
-// All lanes wait; the verdict is made warp-uniform so that no lane leaves a loop alone.
+// All lanes wait; the outcome is made warp-uniform so that no lane leaves a loop alone.
 __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     const bool ok = mbar_wait(bar, parity, abort_flag);
     return __all_sync(0xffffffffu, ok);

@@ -202,7 +202,7 @@ __global__ void __launch_bounds__(LG_THREADS, LG_MIN_CTAS) logits_partial_kernel
         if constexpr (SETS == 2) {
             if (set == 1) *reinterpret_cast<float4*>(s_add + (mt * 32 + lane) * 4) = make_float4(acc[0], acc[1], acc[2], acc[3]);
         }
-        // every warp gets here, whatever became of its waits: the verdict is made uniform at this barrier, so that
+        // every warp gets here, whatever became of its waits: the outcome is made uniform at this barrier, so that
         // all warps leave together or none does
         if (!__syncthreads_and(ok ? 1 : 0)) break;
         if constexpr (SETS == 2) {
