@@ -109,7 +109,8 @@ __global__ void __launch_bounds__(LG_THREADS, LG_MIN_CTAS) logits_partial_kernel
         if (hb > 0) __syncthreads();          // the previous block's m and l have been written out (reached by all: see below)
         {
             // a lane owns token pairs (2u, 2u + 1), u = lane + 32 i: coalesced 8-byte loads, once for the maximum and
-            // once more (out of the cache) for the weights
+            // once more (out of the cache) for the weights; the first 256 slots - the whole chunk, at the usual chunk
+            // size - are kept in registers instead
             float mx = NEG_INF;
             const bool live = warp < nh;
             const float* row = p.logits + ((size_t)b * p.Hq + h0 + (live ? warp : 0)) * p.K + t0;
@@ -122,7 +123,12 @@ __global__ void __launch_bounds__(LG_THREADS, LG_MIN_CTAS) logits_partial_kernel
                 }
                 return v;
             };
-            for (int u0 = 0; 2 * u0 < nt; u0 += 128) {                 // four independent loads in flight per lane
+            float2 first[4];                                           // the chunk's first 256 slots stay in registers
+#pragma unroll
+            for (int j = 0; j < 4; ++j) first[j] = pair_at(lane + 32 * j);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) mx = fmaxf(mx, fmaxf(first[j].x, first[j].y));
+            for (int u0 = 128; 2 * u0 < nt; u0 += 128) {               // four independent loads in flight per lane
                 float2 v[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) v[j] = pair_at(u0 + lane + 32 * j);
@@ -137,7 +143,7 @@ __global__ void __launch_bounds__(LG_THREADS, LG_MIN_CTAS) logits_partial_kernel
             for (int u0 = 0; 2 * u0 < nsteps * 16; u0 += 128) {        // pair index u: step u / 8, position u % 8 in it
                 float2 sv[4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) sv[j] = pair_at(u0 + lane + 32 * j);
+                for (int j = 0; j < 4; ++j) sv[j] = u0 == 0 ? first[j] : pair_at(u0 + lane + 32 * j);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const int u = u0 + lane + 32 * j;
