@@ -701,6 +701,7 @@ def main():
     if world > 1:
         os.environ.setdefault("NCCL_DEBUG", "INFO")          # communicator lines (ranks, transport) stay visible
         os.environ.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+        os.environ.setdefault("NCCL_DEBUG_FILE", "/dev/stderr")   # standard output carries the one JSON line only
         dist.init_process_group("nccl", device_id=torch.device(R.dev))
 
     # the group-query configurations first: their consumer warps are the most clock-sensitive, and the 7.5 GB
