@@ -437,6 +437,17 @@ def test_result_does_not_depend_on_the_schedule(G):
             assert torch.equal(a, b)
 
 
+def test_a_ring_that_does_not_fit_shared_memory_is_refused_and_the_next_call_works():
+    w = wl(B=2, Hq=4, Hkv=2, seq_lens=[900, 333], tok_begin=[100, 0], tok_end=[900, 333], chunk_tokens=128)
+    prob = DeviceProblem(w, DEV)
+    prob.desc = prob.make_desc(w.chunk_tokens, prob.NC, tune_stages=8)         # 8 x 34 KB: more than an SM has
+    with pytest.raises(hg.HgError) as e:
+        prob.partial()
+    assert e.value.status == hg.HG_ERR_CUDA
+    torch.cuda.synchronize()                                                      # no error is left behind
+    run_and_check(w)
+
+
 @pytest.mark.parametrize("G", [1, 8])
 def test_every_call_leaves_the_work_counter_at_zero(G):
     """More items than resident CTAs, so the counter hands them out.  The last CTA to stop drawing clears both
