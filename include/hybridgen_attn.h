@@ -300,7 +300,13 @@ typedef struct hg_logits_desc {
     int32_t num_chunks;    /* NC >= ceil(K / chunk_tokens): partials per (sequence, head) */
     int32_t* status;       /* dev, optional (present when struct_size covers it): receives HG_DEV_WAIT_TIMEOUT if a
                               bounded on-chip wait of the kernel ran out */
+    uint32_t tune;         /* optional (present when struct_size covers it): HG_LOGITS_TUNE_* bits, 0 = defaults */
+    uint32_t reserved;     /* 0 */
 } hg_logits_desc;
+
+/* hg_logits_desc.tune: the same partials by another route (tests compare them; both are bit-reproducible) */
+#define HG_LOGITS_TUNE_WARP_MMA 1u   /* the contraction on warp-level MMAs (mma.sync) instead of tcgen05.mma with the
+                                        accumulator in tensor memory */
 
 /*
  * Softmax partials from host-computed logits and the matching V rows: the device side of the paper's

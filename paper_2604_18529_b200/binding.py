@@ -27,6 +27,7 @@ HG_FLAG_COUNTER_CLEAN = 4
 HG_STATIC_SCRATCH_BYTES = 8 << 20
 (HG_TUNE_NO_PERSISTENT, HG_TUNE_NO_DYNAMIC, HG_TUNE_NO_PDL, HG_TUNE_NO_MERGE_CLUSTER, HG_TUNE_NO_MERGE_ROWS,
  HG_TUNE_NO_GQA16, HG_TUNE_NO_HOST_DIRECT, HG_TUNE_NO_SPEC_PREFETCH) = 1, 2, 4, 8, 16, 32, 64, 128
+HG_LOGITS_TUNE_WARP_MMA = 1
 
 
 class HgError(RuntimeError):
@@ -74,6 +75,8 @@ class HgLogitsDesc(C.Structure):
         ("chunk_tokens", C.c_int32),
         ("num_chunks", C.c_int32),
         ("status", C.c_void_p),
+        ("tune", C.c_uint32),
+        ("reserved", C.c_uint32),
     ]
 
 
@@ -224,7 +227,8 @@ def hg_attn_partial(q, k_cache, v_cache, seq_lens, tok_begin, tok_end, o_part, m
 
 
 def logits_desc(*, batch: int, num_q_heads: int, num_kv_heads: int, head_dim: int, dtype, max_selected: int,
-                chunk_tokens: int = 256, num_chunks: int = 0, status: Optional[torch.Tensor] = None) -> HgLogitsDesc:
+                chunk_tokens: int = 256, num_chunks: int = 0, status: Optional[torch.Tensor] = None,
+                tune: int = 0) -> HgLogitsDesc:
     d = HgLogitsDesc()
     d.struct_size = C.sizeof(HgLogitsDesc)
     d.batch, d.num_q_heads, d.num_kv_heads, d.head_dim = batch, num_q_heads, num_kv_heads, head_dim
@@ -232,6 +236,7 @@ def logits_desc(*, batch: int, num_q_heads: int, num_kv_heads: int, head_dim: in
     d.max_selected, d.chunk_tokens = max_selected, chunk_tokens
     d.num_chunks = num_chunks or -(-max_selected // chunk_tokens)
     d.status = _dev(status, "status", torch.int32)
+    d.tune = tune
     d._keep = (status,)
     return d
 

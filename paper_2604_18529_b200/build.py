@@ -10,7 +10,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libhybridgen_attn.so")
 SOURCES = [os.path.join(CSRC, "hg_attn.cu"), os.path.join(CSRC, "hg_host.cpp")]
-DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("hg_device.cuh", "hg_partial.cuh", "hg_merge.cuh", "hg_logits.cuh", "hg_kvcache.cuh", "hg_stage.cuh")] + [
+DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("hg_device.cuh", "hg_partial.cuh", "hg_merge.cuh", "hg_logits.cuh", "hg_logits_tc.cuh", "hg_kvcache.cuh", "hg_stage.cuh")] + [
     os.path.join(ROOT, "include", "hybridgen_attn.h"), os.path.join(ROOT, "include", "hybridgen_host.h")]
 
 

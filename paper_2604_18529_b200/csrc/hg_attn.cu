@@ -17,6 +17,7 @@
 
 #include "hg_kvcache.cuh"
 #include "hg_logits.cuh"
+#include "hg_logits_tc.cuh"
 #include "hg_merge.cuh"
 #include "hg_partial.cuh"
 #include "hg_stage.cuh"
@@ -440,6 +441,15 @@ hg_status hg_attn_partial_from_logits(const float* logits, const void* v_rows, c
         kern<<<grid, LG_THREADS, smem, cs>>>(tv, p);
         return cudaGetLastError() == cudaSuccess ? HG_OK : HG_ERR_CUDA;
     };
+    const uint32_t ltune = d->struct_size >= offsetof(hg_logits_desc, tune) + sizeof(uint32_t) ? d->tune : 0u;
+    if (!(ltune & HG_LOGITS_TUNE_WARP_MMA)) {
+        // the contraction on tcgen05.mma, the accumulator in tensor memory
+        if (d->head_dim == 128)
+            return bf16 ? launch(logits_partial_tc_kernel<128, true>, logits_tc_smem_bytes<128>(p.chunk))
+                        : launch(logits_partial_tc_kernel<128, false>, logits_tc_smem_bytes<128>(p.chunk));
+        return bf16 ? launch(logits_partial_tc_kernel<64, true>, logits_tc_smem_bytes<64>(p.chunk))
+                    : launch(logits_partial_tc_kernel<64, false>, logits_tc_smem_bytes<64>(p.chunk));
+    }
     if (d->head_dim == 128)
         return bf16 ? launch(logits_partial_kernel<128, true>, logits_smem_bytes<128>(p.chunk))
                     : launch(logits_partial_kernel<128, false>, logits_smem_bytes<128>(p.chunk));
