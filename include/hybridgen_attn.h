@@ -304,9 +304,10 @@ typedef struct hg_logits_desc {
     uint32_t reserved;     /* 0 */
 } hg_logits_desc;
 
-/* hg_logits_desc.tune: the same partials by another route (tests compare them; both are bit-reproducible) */
-#define HG_LOGITS_TUNE_WARP_MMA 1u   /* the contraction on warp-level MMAs (mma.sync) instead of tcgen05.mma with the
-                                        accumulator in tensor memory */
+/* hg_logits_desc.tune: which of the two kernels computes the partials (0: the library's choice, the faster one
+   for the shape; tests compare the two; both are bit-reproducible) */
+#define HG_LOGITS_TUNE_WARP_MMA 1u   /* the contraction on warp-level MMAs (mma.sync), one CTA per chunk */
+#define HG_LOGITS_TUNE_TCGEN05 2u    /* the contraction on tcgen05.mma, the accumulator in tensor memory */
 
 /*
  * Softmax partials from host-computed logits and the matching V rows: the device side of the paper's

@@ -27,7 +27,7 @@ HG_FLAG_COUNTER_CLEAN = 4
 HG_STATIC_SCRATCH_BYTES = 8 << 20
 (HG_TUNE_NO_PERSISTENT, HG_TUNE_NO_DYNAMIC, HG_TUNE_NO_PDL, HG_TUNE_NO_MERGE_CLUSTER, HG_TUNE_NO_MERGE_ROWS,
  HG_TUNE_NO_GQA16, HG_TUNE_NO_HOST_DIRECT, HG_TUNE_NO_SPEC_PREFETCH) = 1, 2, 4, 8, 16, 32, 64, 128
-HG_LOGITS_TUNE_WARP_MMA = 1
+HG_LOGITS_TUNE_WARP_MMA, HG_LOGITS_TUNE_TCGEN05 = 1, 2
 
 
 class HgError(RuntimeError):

@@ -442,13 +442,33 @@ hg_status hg_attn_partial_from_logits(const float* logits, const void* v_rows, c
         return cudaGetLastError() == cudaSuccess ? HG_OK : HG_ERR_CUDA;
     };
     const uint32_t ltune = d->struct_size >= offsetof(hg_logits_desc, tune) + sizeof(uint32_t) ? d->tune : 0u;
-    if (!(ltune & HG_LOGITS_TUNE_WARP_MMA)) {
-        // the contraction on tcgen05.mma, the accumulator in tensor memory
+    const int tc_stages = d->head_dim == 128 ? lgtc_stages<128>(p.chunk) : lgtc_stages<64>(p.chunk);
+    const bool use_tc = (ltune & HG_LOGITS_TUNE_TCGEN05) != 0 && !(ltune & HG_LOGITS_TUNE_WARP_MMA) && tc_stages >= 2;
+    if (use_tc) {
+        // the contraction on tcgen05.mma, the accumulator in tensor memory: persistent CTAs, two per SM
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+            cudaGetLastError();
+            return HG_ERR_CUDA;
+        }
+        p.stages = tc_stages;
+        p.head_blocks = (p.G + 7) / 8;
+        p.items = (long long)p.B * p.Hkv * p.NC * p.head_blocks;
+        const long long resident = 2ll * sms;
+        const unsigned ctas = (unsigned)(p.items < resident ? p.items : resident);
+        auto launch_tc = [&](auto kern, size_t smem) -> hg_status {
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+                cudaGetLastError();
+                return HG_ERR_CUDA;
+            }
+            kern<<<ctas, LGTC_THREADS, smem, cs>>>(tv, p);
+            return cudaGetLastError() == cudaSuccess ? HG_OK : HG_ERR_CUDA;
+        };
         if (d->head_dim == 128)
-            return bf16 ? launch(logits_partial_tc_kernel<128, true>, logits_tc_smem_bytes<128>(p.chunk))
-                        : launch(logits_partial_tc_kernel<128, false>, logits_tc_smem_bytes<128>(p.chunk));
-        return bf16 ? launch(logits_partial_tc_kernel<64, true>, logits_tc_smem_bytes<64>(p.chunk))
-                    : launch(logits_partial_tc_kernel<64, false>, logits_tc_smem_bytes<64>(p.chunk));
+            return bf16 ? launch_tc(logits_partial_tc_kernel<128, true>, logits_tc_smem_bytes<128>(p.chunk))
+                        : launch_tc(logits_partial_tc_kernel<128, false>, logits_tc_smem_bytes<128>(p.chunk));
+        return bf16 ? launch_tc(logits_partial_tc_kernel<64, true>, logits_tc_smem_bytes<64>(p.chunk))
+                    : launch_tc(logits_partial_tc_kernel<64, false>, logits_tc_smem_bytes<64>(p.chunk));
     }
     if (d->head_dim == 128)
         return bf16 ? launch(logits_partial_kernel<128, true>, logits_smem_bytes<128>(p.chunk))

@@ -41,6 +41,9 @@ struct LogitsParams {
     float* l_part;
     int32_t* status;          // optional: HG_DEV_WAIT_TIMEOUT when a bounded wait ran out
     int B, Hq, Hkv, G, K, chunk, NC;
+    // the tcgen05 kernel only: V tiles in its ring, blocks of 8 heads per group, work items in all
+    int stages, head_blocks;
+    long long items;
 };
 
 // Dynamic shared memory: [lg_stages<D>()] V tiles (64 x D x 2 bytes, 1024-byte aligned), then the P fragments

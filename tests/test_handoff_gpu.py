@@ -16,6 +16,10 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
+# both kernels of the hand-off: warp-level MMAs, and tcgen05.mma with the accumulator in tensor memory
+KERNELS = [pytest.param(pkg.binding.HG_LOGITS_TUNE_WARP_MMA, id="warp_mma"), pytest.param(pkg.binding.HG_LOGITS_TUNE_TCGEN05, id="tcgen05")]
+
+
 def handoff_case(w, keep, chunk, seed=0):
     """keep: fraction of the host slice the host selects (top logits of the group's first head, per KV head)."""
     rng = np.random.default_rng(seed)
@@ -51,13 +55,14 @@ def handoff_case(w, keep, chunk, seed=0):
 
 @pytest.mark.parametrize("G,D,dtype", [(1, 128, "f16"), (4, 128, "f16"), (8, 64, "bf16"), (12, 128, "bf16")])
 @pytest.mark.parametrize("keep,chunk", [(1.0, 256), (0.25, 64), (0.05, 32)])
-def test_handoff_partials_and_merged_result(G, D, dtype, keep, chunk):
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_handoff_partials_and_merged_result(G, D, dtype, keep, chunk, kernel):
     w = W.AttnWorkload("handoff", 3, 2 * G, 2, D, dtype, [900, 400, 130], [500, 333, 0], [900, 400, 130],
                        page_size=16, chunk_tokens=128, seed=41 + G)
     q, K, V, logits, vrows, n_sel, chosen, Kpad = handoff_case(w, keep, chunk)
     NCs = -(-Kpad // chunk)
     desc = pkg.logits_desc(batch=w.B, num_q_heads=w.Hq, num_kv_heads=w.Hkv, head_dim=D, dtype=dtype,
-                           max_selected=Kpad, chunk_tokens=chunk, num_chunks=NCs)
+                           max_selected=Kpad, chunk_tokens=chunk, num_chunks=NCs, tune=kernel)
     lg = torch.from_numpy(logits).float().to(DEV)
     vr = torch.from_numpy(vrows.view(np.int16)).to(DEV)
     ns = torch.from_numpy(n_sel).to(DEV)
@@ -104,7 +109,8 @@ def test_handoff_partials_and_merged_result(G, D, dtype, keep, chunk):
 
 @pytest.mark.parametrize("G,D,dtype,K,chunk", [(1, 64, "f16", 77, 96), (16, 64, "bf16", 333, 96), (3, 128, "f16", 1025, 1024),
                                                (8, 128, "bf16", 2049, 160), (5, 128, "f16", 64, 64)])
-def test_handoff_odd_sizes(G, D, dtype, K, chunk):
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_handoff_odd_sizes(G, D, dtype, K, chunk, kernel):
     """Row lengths that are not a multiple of anything (logit rows at odd offsets take the scalar load path, V tiles
     straddle the end of a chunk and of the whole array), chunk sizes that are not a multiple of the 64-row tile, groups
     that fill one and a half or two head blocks, empty sequences and sequences that use every slot."""
@@ -122,7 +128,7 @@ def test_handoff_odd_sizes(G, D, dtype, K, chunk):
     NCs = -(-K // chunk)
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     desc = pkg.logits_desc(batch=B, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, dtype=dtype, max_selected=K,
-                           chunk_tokens=chunk, num_chunks=NCs, status=status)
+                           chunk_tokens=chunk, num_chunks=NCs, status=status, tune=kernel)
     lg = torch.from_numpy(logits).to(DEV)
     vr = torch.from_numpy(vbits.view(np.int16)).to(DEV)
     ho = torch.full((B, Hq, NCs, D), 5.0, device=DEV); hm = torch.full((B, Hq, NCs), 5.0, device=DEV); hl = torch.full_like(hm, 5.0)
