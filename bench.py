@@ -349,12 +349,14 @@ def time_handoff(dev, steps):
     import paper_2604_18529_b200 as pkg
     peak, peak_kind = measured_peak()
     out = []
-    for name, B, Hq, Hkv, K in (("mha", 8, 40, 40, 8192), ("gqa8", 1, 64, 8, 262144)):
+    # 256-slot chunks go to the warp-level kernel, 512-slot chunks to the tcgen05 kernel (the library's choice)
+    for name, B, Hq, Hkv, K, chunk in (("mha", 8, 40, 40, 8192, 256), ("gqa8", 1, 64, 8, 262144, 256),
+                                       ("mha_c512", 8, 40, 40, 8192, 512), ("gqa8_c512", 1, 64, 8, 262144, 512)):
         gen = torch.Generator(device=dev).manual_seed(11)
         logits = torch.randn(B, Hq, K, device=dev, generator=gen)
         vrows = torch.randn(B, Hkv, K, 128, device=dev, generator=gen).half()
         n_sel = torch.full((B,), K, dtype=torch.int32, device=dev)
-        ld = pkg.logits_desc(batch=B, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=128, dtype="f16", max_selected=K, chunk_tokens=256)
+        ld = pkg.logits_desc(batch=B, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=128, dtype="f16", max_selected=K, chunk_tokens=chunk)
         o = torch.empty(B, Hq, ld.num_chunks, 128, device=dev); m = torch.empty(B, Hq, ld.num_chunks, device=dev); l = torch.empty_like(m)
         call = lambda: pkg.hg_attn_partial_from_logits(logits, vrows, n_sel, o, m, l, ld)
         for _ in range(3):
@@ -368,7 +370,8 @@ def time_handoff(dev, steps):
         us = e0.elapsed_time(e1) * 1e3 / steps
         nbytes = logits.numel() * 4 + vrows.numel() * 2 + o.numel() * 4 + 2 * m.numel() * 4
         out.append({"shape": name, "batch": B, "q_heads": Hq, "kv_heads": Hkv, "head_dim": 128, "selected_per_seq": K,
-                    "chunk_tokens": 256, "us": us, "alg_bytes": nbytes, "gbs": nbytes / us / 1e3,
+                    "chunk_tokens": chunk, "kernel": "tcgen05.mma, accumulator in tensor memory" if chunk >= 512 else "mma.sync",
+                    "us": us, "alg_bytes": nbytes, "gbs": nbytes / us / 1e3,
                     "frac": nbytes / us / 1e3 / peak, "peak_kind": f"{peak_kind} copy bandwidth",
                     "frac_of_8000": nbytes / us / 1e3 / 8000.0})
         del logits, vrows, o, m, l

@@ -443,7 +443,12 @@ hg_status hg_attn_partial_from_logits(const float* logits, const void* v_rows, c
     };
     const uint32_t ltune = d->struct_size >= offsetof(hg_logits_desc, tune) + sizeof(uint32_t) ? d->tune : 0u;
     const int tc_stages = d->head_dim == 128 ? lgtc_stages<128>(p.chunk) : lgtc_stages<64>(p.chunk);
-    const bool use_tc = (ltune & HG_LOGITS_TUNE_TCGEN05) != 0 && !(ltune & HG_LOGITS_TUNE_WARP_MMA) && tc_stages >= 2;
+    const long long tc_items = (long long)p.B * p.Hkv * p.NC * ((p.G + 7) / 8);
+    // The library's choice: the tcgen05 kernel pays a hand-shake per work item and wins from 512-slot chunks on
+    // (6-14 % at D = 128); with 256-slot chunks and at D = 64 the warp-level kernel, one CTA per chunk, is 7-10 % ahead.
+    const bool tc_possible = tc_stages >= 2 && tc_items < 0x7fffffffll;
+    const bool use_tc = tc_possible && !(ltune & HG_LOGITS_TUNE_WARP_MMA) &&
+                        ((ltune & HG_LOGITS_TUNE_TCGEN05) != 0 || (d->head_dim == 128 && d->chunk_tokens >= 512));
     if (use_tc) {
         // the contraction on tcgen05.mma, the accumulator in tensor memory: persistent CTAs, two per SM
         int dev = 0, sms = 0;
@@ -454,7 +459,7 @@ hg_status hg_attn_partial_from_logits(const float* logits, const void* v_rows, c
         p.stages = tc_stages;
         p.head_blocks = (p.G + 7) / 8;
         p.items = (long long)p.B * p.Hkv * p.NC * p.head_blocks;
-        const long long resident = 2ll * sms;
+        const long long resident = (long long)LGTC_CTAS_PER_SM * sms;
         const unsigned ctas = (unsigned)(p.items < resident ? p.items : resident);
         auto launch_tc = [&](auto kern, size_t smem) -> hg_status {
             if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {

@@ -83,6 +83,7 @@ constexpr int LGTC_HEAD_WARPS = 8;
 constexpr int LGTC_LOAD_WARP = LGTC_HEAD_WARPS, LGTC_MMA_WARP = LGTC_HEAD_WARPS + 1;
 constexpr int LGTC_THREADS = (LGTC_HEAD_WARPS + 2) * 32;   // eight head warps, the loader and the tensor-core warp
 constexpr int LGTC_MAX_STAGES = 8;
+constexpr int LGTC_CTAS_PER_SM = 2;     // (three, with rings of three tiles, measured the same at D = 128)
 constexpr int LGTC_SMEM_BUDGET = 112 * 1024;               // dynamic shared memory of one of an SM's two CTAs
 
 __host__ __device__ constexpr size_t lgtc_p_bytes(int chunk) { return (size_t)((chunk + LG_TILE - 1) / LG_TILE * LG_TILE / 16) * 512; }
@@ -105,13 +106,16 @@ struct LgItem {
     int nt;          // slots of the chunk in use (0: an empty partial)
     int row_base;    // first V row of the chunk in the [B * Hkv * K][D] view
 };
-__device__ __forceinline__ LgItem lg_item(const LogitsParams& p, long long i) {
+constexpr int LGTC_NSEL_CACHE = 256;       // sequences whose slot counts are kept in shared memory
+// (every role decodes every item of its CTA: the decode must not wait for global memory, and the item index is 32 bits
+// wide - the host takes the other kernel for more than 2^31 items)
+__device__ __forceinline__ LgItem lg_item(const LogitsParams& p, const int* s_nsel, uint32_t i) {
     LgItem it;
-    it.hb = (int)(i % p.head_blocks); i /= p.head_blocks;
-    it.c = (int)(i % p.NC); i /= p.NC;
-    it.g = (int)(i % p.Hkv);
-    it.b = (int)(i / p.Hkv);
-    const int n = min(max(p.n_sel[it.b], 0), p.K);
+    it.hb = (int)(i % (uint32_t)p.head_blocks); i /= (uint32_t)p.head_blocks;
+    it.c = (int)(i % (uint32_t)p.NC); i /= (uint32_t)p.NC;
+    it.g = (int)(i % (uint32_t)p.Hkv);
+    it.b = (int)(i / (uint32_t)p.Hkv);
+    const int n = min(max(it.b < LGTC_NSEL_CACHE ? s_nsel[it.b] : p.n_sel[it.b], 0), p.K);
     const int t0 = it.c * p.chunk;
     it.nt = max(min(t0 + p.chunk, n) - t0, 0);
     it.row_base = (it.b * p.Hkv + it.g) * p.K + t0;
@@ -119,7 +123,7 @@ __device__ __forceinline__ LgItem lg_item(const LogitsParams& p, long long i) {
 }
 
 template <int D, bool BF16>
-__global__ void __launch_bounds__(LGTC_THREADS, 2) logits_partial_tc_kernel(const __grid_constant__ CUtensorMap tmV, const LogitsParams p) {
+__global__ void __launch_bounds__(LGTC_THREADS, LGTC_CTAS_PER_SM) logits_partial_tc_kernel(const __grid_constant__ CUtensorMap tmV, const LogitsParams p) {
     constexpr int TILE_BYTES = LG_TILE * D * 2;
     constexpr int HALVES = D / 64;                    // 64-component halves of a V row
     constexpr int HALF_BYTES = LG_TILE * 128;
@@ -138,6 +142,7 @@ __global__ void __launch_bounds__(LGTC_THREADS, 2) logits_partial_tc_kernel(cons
     __shared__ uint64_t full[LGTC_MAX_STAGES], empty[LGTC_MAX_STAGES], p_ready[2], done[2], acc_free[2];
     __shared__ int abort_flag_s;
     __shared__ uint32_t tmem_slot;
+    __shared__ int s_nsel[LGTC_NSEL_CACHE];
     const int S = p.stages;
     const uint32_t tile0 = (smem_u32(lg_raw) + 1023u) & ~1023u;
     uint8_t* const tile0_ptr = lg_raw + (tile0 - smem_u32(lg_raw));
@@ -155,6 +160,7 @@ __global__ void __launch_bounds__(LGTC_THREADS, 2) logits_partial_tc_kernel(cons
         abort_flag_s = 0;
         fence_barrier_init();
     }
+    for (int bb = tid; bb < p.B && bb < LGTC_NSEL_CACHE; bb += LGTC_THREADS) s_nsel[bb] = p.n_sel[bb];
     if (warp == LGTC_MMA_WARP) {
         tmem_alloc(&tmem_slot, LGTC_TMEM_COLS);
         tmem_relinquish();
@@ -172,8 +178,8 @@ __global__ void __launch_bounds__(LGTC_THREADS, 2) logits_partial_tc_kernel(cons
         // bandwidth, so the two are separate warps)
         if (lane == 0) {
             bool ok = true;
-            for (long long i = blockIdx.x; i < p.items && ok; i += gridDim.x) {
-                const LgItem cur = lg_item(p, i);
+            for (uint32_t i = blockIdx.x; i < (uint32_t)p.items && ok; i += gridDim.x) {
+                const LgItem cur = lg_item(p, s_nsel, i);
                 const int ntiles = (cur.nt + LG_TILE - 1) / LG_TILE;
                 for (int ti = 0; ti < ntiles; ++ti, ++issued) {
                     const int slot = issued % S;
@@ -191,8 +197,8 @@ __global__ void __launch_bounds__(LGTC_THREADS, 2) logits_partial_tc_kernel(cons
         // (all lanes follow the same control flow; lane 0 issues the products)
         int it = 0, kk = 0;                 // tiles handed to the tensor core, non-empty items begun
         bool ok = true;
-        for (long long i = blockIdx.x; i < p.items && ok; i += gridDim.x) {
-            const LgItem cur = lg_item(p, i);
+        for (uint32_t i = blockIdx.x; i < (uint32_t)p.items && ok; i += gridDim.x) {
+            const LgItem cur = lg_item(p, s_nsel, i);
             if (cur.nt == 0) continue;
             const int ntiles = (cur.nt + LG_TILE - 1) / LG_TILE, j = kk & 1;
             ok = warp_wait(&p_ready[j], (uint32_t)(kk >> 1) & 1u, abort_flag);     // P[j] is written ...
@@ -242,10 +248,10 @@ __global__ void __launch_bounds__(LGTC_THREADS, 2) logits_partial_tc_kernel(cons
         // accumulator that item k takes over); turn item k's logits - requested one item earlier, so they are in
         // registers by now - into m, l and P[k & 1] and tell the driver; request item k + 1's logits; read item k - 2's
         // accumulator out and tell the driver that it is free.
-        long long cur_i = blockIdx.x;
+        uint32_t cur_i = blockIdx.x;
         auto next_item = [&](LgItem& out) -> bool {           // the CTA's next non-empty item; empty ones are written on the way
-            while (cur_i < p.items) {
-                const LgItem t = lg_item(p, cur_i);
+            while (cur_i < (uint32_t)p.items) {
+                const LgItem t = lg_item(p, s_nsel, cur_i);
                 cur_i += gridDim.x;
                 if (t.nt > 0) { out = t; return true; }
                 const int nh = min(8, p.G - t.hb * 8);

@@ -59,6 +59,6 @@ def test_default_line_covers_every_configuration_and_headlines_the_largest():
     assert d["ms_per_step"] == head["ms_per_step"] and d["value"] == head["kv_tokens_per_s"]
     assert d["roofline"] == head["roofline"] and d["e2e"] == head["e2e"]
     assert c["min_step_frac_of_8000"] == min(r["step_frac_of_8000"] for r in c["workloads"] if r["workload"] != "tiny")
-    assert [h["shape"] for h in c["handoff"]] == ["mha", "gqa8"] and all(h["gbs"] > 1000 for h in c["handoff"])
+    assert [h["shape"] for h in c["handoff"]] == ["mha", "gqa8", "mha_c512", "gqa8_c512"] and all(h["gbs"] > 1000 for h in c["handoff"])
     s = d["sharded"]
     assert s["ranks"] == 1 and s["gpu_tokens_total"] == 419430 and s["tokens_this_rank"] == 419430 and s["ms_per_step"] > 0
