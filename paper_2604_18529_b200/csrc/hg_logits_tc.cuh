@@ -4,7 +4,7 @@
 // accumulator in tensor memory.  This contraction suits the asynchronous tensor core well: the chunk maximum is known
 // before the first product (the logits come from the host), so the accumulator is never rescaled and nothing but the
 // final read-out has to leave tensor memory; and the V tile, as the TMA tensor load leaves it (64 token rows of 128
-// bytes per 64-component half, 128-byte swizzled), IS the canonical "M-major" A operand - M = 64 components, K = tokens
+// bytes per 64-component half, 128-byte swizzled), IS the canonical "M-major" A operand - M = the D components of a row, K = tokens
 // - so no warp ever touches a V element.  That frees the warps for the one thing that used to stop the stream - the
 // chunk's logits - and lets it run beside the stream instead of in front of it:
 //
@@ -14,8 +14,8 @@
 //     products' completion free the tile's slot (tcgen05.commit on the slot's "empty" barrier) and, after an item's
 //     last tile, announce the item ("done");
 //   * head warp h meanwhile turns head h's logits of the NEXT item into m, l and P, stored (hi + lo 16-bit terms)
-//     as the K-major B operand [8 heads x 16 tokens] of every 16-token step, then reads the PREVIOUS item's
-//     accumulator out of tensor memory (tcgen05.ld) and writes the partial.  P, the accumulator and their barriers
+//     as the K-major B operand [16 rows x 16 tokens] of every 16-token step; warps 0-3 then read the accumulator of
+//     the item before the previous one out of tensor memory (tcgen05.ld) and write the partial.  P, the accumulator and their barriers
 //     are double-buffered by item parity.
 //
 // One product per 16-token step: M = D, N = 16 (the 8 heads' hi terms and their 8 lo terms side by side; the read-out
