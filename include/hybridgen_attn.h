@@ -205,10 +205,11 @@ hg_status hg_attn_merge(const hg_partial_src* partials, int32_t n_src, float* ou
 /*
  * A chunk size for a problem of `total_tokens` GPU-resident token positions (summed over the
  * sequences; an estimate will do) with the given head counts and page size: a multiple of 64 and of
- * page_size between 128 and 2048 tokens that gives the resident CTAs of the device a few work items
- * each.  Chunk size is the caller's choice (the paper has no chunks); this is the rule the measured
- * workloads of this library follow: large problems run best at 1024-2048 tokens, small ones need
- * short chunks to spread over the SMs.  Returns 0 for invalid arguments.  No CUDA call is made.
+ * page_size between 128 and 1024 tokens that gives every resident CTA of the device about fifteen
+ * work items.  Chunk size is the caller's choice (the paper has no chunks); this is the rule the
+ * measured workloads of this library follow: work items of 256-400 KB of K and V ran fastest at every
+ * size (the last items of a launch end spread over one item's duration), small problems need short
+ * chunks to spread over the SMs.  Returns 0 for invalid arguments.  No CUDA call is made.
  */
 int32_t hg_attn_suggest_chunk(int64_t total_tokens, int32_t num_q_heads, int32_t num_kv_heads, int32_t page_size);
 

@@ -488,11 +488,14 @@ int32_t hg_attn_suggest_chunk(int64_t total_tokens, int32_t num_q_heads, int32_t
     if (shift < 4 || shift > 8) return 0;
     const int G = num_q_heads / num_kv_heads;
     const int64_t rows = (int64_t)num_kv_heads * (G <= 8 ? 1 : (G + 15) / 16);     // items per chunk of one sequence
-    const int64_t target_items = 2000;            // about seven per resident CTA of a 148-SM device
+    // about fifteen items per resident CTA of a 148-SM device: items of 256-400 KB were the fastest at every size
+    // measured (the last wave of work items ends spread over about one item's duration, so short items keep the tail
+    // short; below that the per-item epilogues and the longer merge rows cost more than the tail gives back)
+    const int64_t target_items = 4400;
     const int unit = page_size > TILE_T ? page_size : TILE_T;
     int64_t chunk = total_tokens * rows / target_items;
     chunk = (chunk + unit - 1) / unit * unit;
-    const int64_t lo = 128 > unit ? 128 : unit, hi = 2048;
+    const int64_t lo = 128 > unit ? 128 : unit, hi = 1024 > unit ? 1024 : unit;
     if (chunk < lo) chunk = lo;
     if (chunk > hi) chunk = hi;
     return (int32_t)chunk;

@@ -834,6 +834,9 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
             const int v_row = row0 + (lane & 7) + (lane >> 4) * 8;         // V^T: matrices (d lo, d hi) x (tok, tok+8)
             const int v_dc = (lane >> 3) & 1;
             const uint32_t a_off = row_off(a_row), v_off = row_off(v_row);
+            // item epilogue: vectors of four parked per (head, lane), see there
+            constexpr int V4 = KSTEPS / 2;
+            auto park_swz = [](int f, int pair) -> int { return D == 128 ? (f ^ pair) : (f ^ (pair & 1) ^ ((pair >> 1) << 2)); };
 
             for (;;) {
                 int2 d;
@@ -1020,25 +1023,30 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
                         ctl.red_m[par][e] = m_run[nb][0]; ctl.red_m[par][e + 1] = m_run[nb][1];
                         ctl.red_l[par][e] = l_run[nb][0]; ctl.red_l[par][e + 1] = l_run[nb][1];
                     }
-                    // this warp's [8 heads][D] of the block into its own rows; heads 2tq and 2tq+1 sit in the same 2 KB part
-                    float* const lane_base = warp_scratch(s, warp, (nb * 8 + 2 * tq) * D + quad);
+                    // This warp's [8 heads][D] of the block into its own rows.  A lane holds 2 x KSTEPS components of
+                    // each of its two heads (d = 16 mt + quad and that + 8): they are parked as V4 = KSTEPS / 2 vectors
+                    // of four per head, vector quad * V4 + i of the head's D / 4 holding d = 32 i + 8 kk + quad
+                    // (kk = 0..3), at an index XOR-ed with the lane's head pair so that the eight lanes of a store
+                    // phase hit eight different 16-byte bank groups.
 #pragma unroll
-                    for (int mt = 0; mt < KSTEPS; ++mt) {
-                        lane_base[mt * 16] = oacc[nb][mt][0];
-                        lane_base[D + mt * 16] = oacc[nb][mt][1];
-                        lane_base[mt * 16 + 8] = oacc[nb][mt][2];
-                        lane_base[D + mt * 16 + 8] = oacc[nb][mt][3];
+                    for (int hsel = 0; hsel < 2; ++hsel) {
+                        float4* const head_base = reinterpret_cast<float4*>(warp_scratch(s, warp, (nb * 8 + 2 * tq + hsel) * D));
+#pragma unroll
+                        for (int i = 0; i < V4; ++i)
+                            head_base[park_swz(quad * V4 + i, tq)] =
+                                make_float4(oacc[nb][2 * i][hsel], oacc[nb][2 * i][2 + hsel], oacc[nb][2 * i + 1][hsel], oacc[nb][2 * i + 1][2 + hsel]);
                     }
                 }
 #ifdef HG_TRACE
                 ctrace_park += clock64() - te0;
 #endif
                 if (!consumer_sync()) break;
-                // thread -> (head, D/16 consecutive components): the four warp states of one head, weighted
+                // thread -> (head, D/16 components: the parked vectors r and, at D = 128, r + 16 of the head): the four
+                // warp states of one head, weighted
 #pragma unroll
                 for (int nb = 0; nb < NB; ++nb) {
                     constexpr int PER = D / 16;
-                    const int hh = nb * 8 + (tid >> 4), dbase = (tid & 15) * PER;
+                    const int hh = nb * 8 + (tid >> 4), r = tid & 15, pair = (tid >> 4) >> 1;
                     if (hh < nheads) {
                         float mw[CONSUMER_WARPS], M = NEG_INF, lsum = 0.f;
 #pragma unroll
@@ -1051,20 +1059,23 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
                         for (int w2 = 0; w2 < CONSUMER_WARPS; ++w2) {
                             const float w = fast_exp2(mw[w2] - Ms);
                             lsum = fmaf(w, ctl.red_l[par][w2 * HPI + hh], lsum);
-                            const float4* src = reinterpret_cast<const float4*>(warp_scratch(s, w2, hh * D + dbase));
+                            const float4* src = reinterpret_cast<const float4*>(warp_scratch(s, w2, hh * D));
 #pragma unroll
                             for (int v4 = 0; v4 < PER / 4; ++v4) {
-                                const float4 x = src[v4];
+                                const float4 x = src[park_swz(r + 16 * v4, pair)];
                                 accv[v4 * 4 + 0] = fmaf(w, x.x, accv[v4 * 4 + 0]); accv[v4 * 4 + 1] = fmaf(w, x.y, accv[v4 * 4 + 1]);
                                 accv[v4 * 4 + 2] = fmaf(w, x.z, accv[v4 * 4 + 2]); accv[v4 * 4 + 3] = fmaf(w, x.w, accv[v4 * 4 + 3]);
                             }
                         }
                         const size_t oslot = ((size_t)cur.b * p.Hq + h0 + hh) * p.NC + cur.c;
-                        float4* dst = reinterpret_cast<float4*>(p.o_part + oslot * D + dbase);
+                        float* const dst = p.o_part + oslot * D;
 #pragma unroll
-                        for (int v4 = 0; v4 < PER / 4; ++v4)
-                            dst[v4] = make_float4(accv[v4 * 4 + 0], accv[v4 * 4 + 1], accv[v4 * 4 + 2], accv[v4 * 4 + 3]);
-                        if ((tid & 15) == 0) { p.m_part[oslot] = M * LN2; p.l_part[oslot] = lsum; }
+                        for (int v4 = 0; v4 < PER / 4; ++v4) {
+                            const int f = r + 16 * v4, d0 = 32 * (f % V4) + f / V4;      // component kk of vector f: d0 + 8 kk
+#pragma unroll
+                            for (int kk = 0; kk < 4; ++kk) dst[d0 + 8 * kk] = accv[v4 * 4 + kk];
+                        }
+                        if (r == 0) { p.m_part[oslot] = M * LN2; p.l_part[oslot] = lsum; }
                     }
                 }
                 release(s, true);

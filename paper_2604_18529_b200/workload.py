@@ -315,7 +315,7 @@ def make_workload(name: str) -> AttnWorkload:
     if name == "llama70b":
         L = [1048576]
         tb, te = _suffix(L, [0.4])
-        return AttnWorkload("llama70b", 1, 64, 8, 128, "f16", L, tb, te, page_size=16, chunk_tokens=2048,
+        return AttnWorkload("llama70b", 1, 64, 8, 128, "f16", L, tb, te, page_size=16, chunk_tokens=768,
                             sigma_kv=0.5, seed=1004)
     if name == "ragged":
         key = tensor_key(1005, TENSOR_LENS)
@@ -324,7 +324,7 @@ def make_workload(name: str) -> AttnWorkload:
         L = [4096 + int(u[i] * (65536 - 4096 + 1)) for i in range(16)]
         shares = [0.1 + 0.8 * u[16 + i] for i in range(16)]
         tb, te = _suffix(L, shares)
-        return AttnWorkload("ragged", 16, 32, 8, 128, "f16", L, tb, te, page_size=16, chunk_tokens=1024, seed=1005)
+        return AttnWorkload("ragged", 16, 32, 8, 128, "f16", L, tb, te, page_size=16, chunk_tokens=512, seed=1005)
     raise KeyError(name)
 
 

@@ -162,9 +162,10 @@ def test_suggested_chunk_is_always_a_legal_one():
         for tokens in (0, 1, 1000, 157_280, 419_430, 10**9):
             for hq, hkv in ((8, 8), (32, 8), (64, 8), (64, 4), (96, 8)):
                 c = pkg.hg_attn_suggest_chunk(tokens, hq, hkv, page)
-                assert c % 64 == 0 and c % page == 0 and max(128, page) <= c <= 2048
+                assert c % 64 == 0 and c % page == 0 and max(128, page) <= c <= 1024
     assert pkg.hg_attn_suggest_chunk(2048, 64, 8, 16) == 128           # a small problem is cut fine
-    assert pkg.hg_attn_suggest_chunk(10**7, 64, 8, 16) == 2048          # a large one coarse
+    assert pkg.hg_attn_suggest_chunk(10**7, 64, 8, 16) == 1024          # a large one coarse
+    assert pkg.hg_attn_suggest_chunk(278_000, 32, 8, 16) == 512 and pkg.hg_attn_suggest_chunk(419_430, 64, 8, 16) == 768
     for bad in ((-1, 8, 8, 16), (100, 8, 3, 16), (100, 8, 8, 48), (100, 0, 1, 16)):
         with pytest.raises(pkg.HgError):
             pkg.hg_attn_suggest_chunk(*bad)
