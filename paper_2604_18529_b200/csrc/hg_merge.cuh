@@ -18,6 +18,25 @@ namespace hg {
 
 constexpr int MERGE_MAX_SRC = 8;
 
+// The o rows are read with the hint their producer wrote them with (keep the lines in the L2): partials are scratch
+// that the next step overwrites in place, and a line that stays resident is neither written out to DRAM nor
+// allocated again.
+__device__ __forceinline__ uint64_t merge_keep_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ float4 ld_keep_v4(const float* p, uint64_t pol) {
+    float4 v;
+    asm volatile("ld.global.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p), "l"(pol));
+    return v;
+}
+__device__ __forceinline__ float2 ld_keep_v2(const float* p, uint64_t pol) {
+    float2 v;
+    asm volatile("ld.global.L2::cache_hint.v2.f32 {%0, %1}, [%2], %3;" : "=f"(v.x), "=f"(v.y) : "l"(p), "l"(pol));
+    return v;
+}
+
 struct MergeParams {
     const float* o[MERGE_MAX_SRC];
     const float* m[MERGE_MAX_SRC];
@@ -49,6 +68,7 @@ __global__ void __launch_bounds__(THREADS_) merge_kernel(const MergeParams p) {
     cudaTriggerProgrammaticLaunchCompletion();  // a partial kernel launched as a dependent may set up meanwhile
     cudaGridDependencySynchronize();            // partials may come from the kernel launched just before
 #endif
+    const uint64_t keep = merge_keep_policy();
 
     // ---- one sweep: every warp keeps a running maximum and rescales its sums when it grows ----------
     float acc[VEC];
@@ -71,10 +91,10 @@ __global__ void __launch_bounds__(THREADS_) merge_kernel(const MergeParams p) {
                 const bool live = in && mi[u] != NEG_INF;      // an empty partial's o is not read
                 const float* orow = os + (size_t)(in ? i : 0) * D + lane * VEC;
                 if constexpr (VEC == 4) {
-                    const float4 v = live ? *reinterpret_cast<const float4*>(orow) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    const float4 v = live ? ld_keep_v4(orow, keep) : make_float4(0.f, 0.f, 0.f, 0.f);
                     ov[u][0] = v.x; ov[u][1] = v.y; ov[u][2] = v.z; ov[u][3] = v.w;
                 } else {
-                    const float2 v = live ? *reinterpret_cast<const float2*>(orow) : make_float2(0.f, 0.f);
+                    const float2 v = live ? ld_keep_v2(orow, keep) : make_float2(0.f, 0.f);
                     ov[u][0] = v.x; ov[u][1] = v.y;
                 }
             }
@@ -160,6 +180,7 @@ __global__ void __launch_bounds__(256) merge_rows_kernel(const MergeParams p, in
     cudaGridDependencySynchronize();
 #endif
     if (row >= rows) return;
+    const uint64_t keep = merge_keep_policy();
     float acc[VEC];
 #pragma unroll
     for (int v = 0; v < VEC; ++v) acc[v] = 0.f;
@@ -185,10 +206,10 @@ __global__ void __launch_bounds__(256) merge_rows_kernel(const MergeParams p, in
                     li[u] = in ? ls[i] : 0.f;
                     const float* orow = os + (size_t)i * D + lane * VEC;
                     if constexpr (VEC == 4) {
-                        const float4 v = in ? *reinterpret_cast<const float4*>(orow) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        const float4 v = in ? ld_keep_v4(orow, keep) : make_float4(0.f, 0.f, 0.f, 0.f);
                         ov[u][0] = v.x; ov[u][1] = v.y; ov[u][2] = v.z; ov[u][3] = v.w;
                     } else {
-                        const float2 v = in ? *reinterpret_cast<const float2*>(orow) : make_float2(0.f, 0.f);
+                        const float2 v = in ? ld_keep_v2(orow, keep) : make_float2(0.f, 0.f);
                         ov[u][0] = v.x; ov[u][1] = v.y;
                     }
                 }

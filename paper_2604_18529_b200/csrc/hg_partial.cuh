@@ -818,7 +818,7 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
                         lsum = fmaf(w, ctl.red_l[par][sidx], lsum);
                     }
                     const size_t oslot = ((size_t)cur.b * p.Hq + h0) * p.NC + cur.c;
-                    p.o_part[oslot * D + tid] = accv;
+                    st_global_hint(p.o_part + oslot * D + tid, accv, l2_evict_last_policy());      // the merge reads these lines next
                     if (tid == 0) { p.m_part[oslot] = M * LN2; p.l_part[oslot] = lsum; }
                 }
                 release(s, true);
@@ -1069,11 +1069,12 @@ __global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_consta
                         }
                         const size_t oslot = ((size_t)cur.b * p.Hq + h0 + hh) * p.NC + cur.c;
                         float* const dst = p.o_part + oslot * D;
+                        const uint64_t keep = l2_evict_last_policy();      // the merge reads these lines next
 #pragma unroll
                         for (int v4 = 0; v4 < PER / 4; ++v4) {
                             const int f = r + 16 * v4, d0 = 32 * (f % V4) + f / V4;      // component kk of vector f: d0 + 8 kk
 #pragma unroll
-                            for (int kk = 0; kk < 4; ++kk) dst[d0 + 8 * kk] = accv[v4 * 4 + kk];
+                            for (int kk = 0; kk < 4; ++kk) st_global_hint(dst + d0 + 8 * kk, accv[v4 * 4 + kk], keep);
                         }
                         if (r == 0) { p.m_part[oslot] = M * LN2; p.l_part[oslot] = lsum; }
                     }
