@@ -227,8 +227,9 @@ __global__ void __launch_bounds__(LG_THREADS, LG_MIN_CTAS) logits_partial_kernel
                 const int hh = 2 * tq + j;
                 if (hh < nh) {
                     const size_t slot = ((size_t)b * p.Hq + h0 + hh) * p.NC + c;
-                    p.o_part[slot * D + d] = acc[j];
-                    p.o_part[slot * D + d + 8] = acc[2 + j];
+                    const uint64_t keep = l2_evict_last_policy();      // the merge reads these lines next
+                    st_global_hint(p.o_part + slot * D + d, acc[j], keep);
+                    st_global_hint(p.o_part + slot * D + d + 8, acc[2 + j], keep);
                     if (mt == 0 && quad == 0) { p.m_part[slot] = s_m[hh]; p.l_part[slot] = s_l[hh]; }
                 }
             }

@@ -290,11 +290,12 @@ __global__ void __launch_bounds__(LGTC_THREADS, LGTC_CTAS_PER_SM) logits_partial
                 const int h0 = im.g * p.G + im.hb * 8, nh = min(8, p.G - im.hb * 8);
                 const int d = D == 128 ? warp * 32 + lane : warp * 16 + lane;
                 if (D == 128 || lane < 16) {
+                    const uint64_t keep = l2_evict_last_policy();      // the merge reads these lines next
 #pragma unroll
                     for (int hh = 0; hh < 8; ++hh)
                         if (hh < nh)
-                            p.o_part[(((size_t)im.b * p.Hq + h0 + hh) * p.NC + im.c) * D + d] =
-                                __uint_as_float(r[hh]) + __uint_as_float(r[8 + hh]);
+                            st_global_hint(p.o_part + (((size_t)im.b * p.Hq + h0 + hh) * p.NC + im.c) * D + d,
+                                           __uint_as_float(r[hh]) + __uint_as_float(r[8 + hh]), keep);
                 }
             }
         };
