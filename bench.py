@@ -41,9 +41,9 @@ LARGE = ("opt13b", "opt30b", "llama70b", "ragged")
 # capture of the first sequences is scaled to the full launch.
 NCU_TRAFFIC_BYTES = {
     "opt13b": 4 * (805_556_224 + 4_392_704),          # two of the eight sequences captured, x 4
-    "llama70b": 1_718_240_000 + 8_749_568,            # the full launch captured
+    "llama70b": 1_718_243_000 + 4_194_048,            # the full launch captured
     "opt30b": 4 * (1_879_137_000 + 3_563_520),        # one of the four sequences captured, x 4
-    "ragged": 951_518_976 + 7_020_800,                # the full launch captured
+    "ragged": 951_552_512 + 4_044_288,                # the full launch captured
 }
 
 

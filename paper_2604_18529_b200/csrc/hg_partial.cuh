@@ -181,8 +181,11 @@ __device__ __forceinline__ Item decode_item(const PartialParams& p, const Contro
     return it;
 }
 
+// (Register budget: two CTAs per SM are what the shared memory allows; the group-query kernel with items of 8 heads is
+// held to the registers of three per SM - 128 instead of 163, nothing spilled, the tile loop is not on the critical
+// path - so that CTAs of a kernel launched as a dependent find room beside it earlier.)
 template <int D, bool BF16, int MODE>
-__global__ void __launch_bounds__(THREADS, 2) partial_kernel(const __grid_constant__ CUtensorMap tmK,
+__global__ void __launch_bounds__(THREADS, MODE == MODE_GQA ? 3 : 2) partial_kernel(const __grid_constant__ CUtensorMap tmK,
                                                           const __grid_constant__ CUtensorMap tmV,
                                                           const PartialParams p) {
     constexpr int HALVES = D / 64;
