@@ -52,7 +52,7 @@ def test_default_line_covers_every_configuration_and_headlines_the_largest():
             assert "step_frac_of_8000" not in r and r["us_per_step"] > 0
         else:
             ro = r["roofline"]
-            assert 0.3 < r["step_frac_of_8000"] < 1.05 and ro["traffic"] > 0.99 * ro["alg_bytes_per_launch"]
+            assert 0.3 < r["step_frac_of_8000"] < 1.05 and ro["traffic"] > 0.98 * ro["alg_bytes_per_launch"]     # (partials that stay in the L2 never reach DRAM)
             assert abs(ro["frac"] - ro["achieved"] / ro["peak"]) < 1e-9
             assert r["probe_us"] > 0 and 0.3 < r["step_frac_of_probe"] < 1.5     # the bare loads are the ceiling
     head = [r for r in c["workloads"] if r["workload"] == "opt30b"][0]
