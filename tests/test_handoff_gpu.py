@@ -215,3 +215,38 @@ def test_cpu_stage_feeds_the_gpu_stage(strategy, G):
     assert np.abs(out - ref_out).max() <= OUT_MAX_ABS
     assert np.linalg.norm(out - ref_out) / np.linalg.norm(ref_out) <= OUT_REL_L2
     assert np.abs(lse - ref_lse).max() <= LSE_ABS
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,K,chunk", [(8, 40, 40, 8192, 256), (1, 64, 8, 262144, 256), (8, 40, 40, 8192, 512), (1, 64, 8, 262144, 512)])
+def test_handoff_at_the_sizes_and_launch_configurations_the_bench_times(B, Hq, Hkv, K, chunk):
+    """The four hand-off measurements of bench.py (0.6 - 0.7 GB each, the library's own choice of kernel: warp-level MMAs
+    at 256-slot chunks, tcgen05 at 512): sampled (sequence, head, chunk) partials against the oracle, and properties
+    that hold for every partial."""
+    D, G = 128, Hq // Hkv
+    gen = torch.Generator(device=DEV).manual_seed(11)
+    logits = torch.randn(B, Hq, K, device=DEV, generator=gen)
+    vrows = torch.randn(B, Hkv, K, D, device=DEV, generator=gen).half()
+    n_sel = torch.full((B,), K, dtype=torch.int32, device=DEV)
+    n_sel[-1] = K - 37                                             # a ragged last chunk in the last sequence
+    ld = pkg.logits_desc(batch=B, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, dtype="f16", max_selected=K, chunk_tokens=chunk)
+    NC = ld.num_chunks
+    o = torch.full((B, Hq, NC, D), 7.0, device=DEV); m = torch.full((B, Hq, NC), 7.0, device=DEV); l = torch.full((B, Hq, NC), 7.0, device=DEV)
+    pkg.hg_attn_partial_from_logits(logits, vrows, n_sel, o, m, l, ld)
+    torch.cuda.synchronize()
+    # every partial: the maximum is the chunk's largest logit, 1 <= l <= slots in use, nothing left unwritten
+    ref_m = logits.view(B, Hq, NC, chunk).amax(dim=3)
+    ref_m[-1, :, -1] = logits[-1, :, (NC - 1) * chunk:K - 37].amax(dim=1)
+    assert torch.equal(m, ref_m)
+    assert bool((l >= 1.0).all()) and bool((l <= chunk).all()) and bool(torch.isfinite(o).all())
+    # sampled partials against the oracle (first and last chunk of the ragged sequence among them)
+    rng = np.random.default_rng(5)
+    picks = [(B - 1, Hq - 1, NC - 1), (B - 1, 0, NC - 1), (0, 0, 0)] + [(int(rng.integers(B)), int(rng.integers(Hq)), int(rng.integers(NC))) for _ in range(45)]
+    got_o, got_m, got_l, rm, rl, ro = [], [], [], [], [], []
+    for b, h, c in picks:
+        a, e = c * chunk, min((c + 1) * chunk, int(n_sel[b]))
+        lg = logits[b, h, a:e].double().cpu().numpy()
+        vr = vrows[b, h // G, a:e].contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+        mm, ll, oo = O.partial_from_logits(lg, vr, "f16")
+        rm.append(mm); rl.append(ll); ro.append(oo)
+        got_o.append(o[b, h, c]); got_m.append(m[b, h, c]); got_l.append(l[b, h, c])
+    check_partials(torch.stack(got_o), torch.stack(got_m), torch.stack(got_l), np.array(rm), np.array(rl), np.stack(ro))
