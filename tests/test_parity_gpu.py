@@ -939,3 +939,37 @@ def test_the_readme_decode_flow():
                        ref.host_partials_device(DEV), out, lse, ws, desc)
     torch.cuda.synchronize()
     check_output(out, lse, ref.out, ref.lse, "readme")
+
+
+@pytest.mark.parametrize("rows,slots", [(8, 65), (24, 700), (48, 300), (64, 548), (100, 131), (128, 700), (200, 300), (320, 40), (512, 70)])
+def test_merge_launch_shapes_against_the_oracle(rows, slots):
+    """hg_attn_merge alone on synthetic partials, over the launch shapes it chooses between (clusters of 8, 4 and 2 CTAs,
+    one CTA of 8 or of 32 warps per row), with and without clusters: against the oracle's MERGE."""
+    from oracle import hg_oracle as O
+    D, B = 128, 1
+    g = torch.Generator(device=DEV).manual_seed(rows * 1000 + slots)
+    o = torch.randn(B, rows, slots, D, device=DEV, generator=g)
+    m = torch.randn(B, rows, slots, device=DEV, generator=g) * 3.0
+    l = torch.rand(B, rows, slots, device=DEV, generator=g) * 50.0 + 1.0
+    m[:, :, slots // 2:] = float("-inf")                                     # trailing empty slots ...
+    m[:, ::3, : slots // 4] = float("-inf"); m[:, 1, :] = float("-inf")      # ... holes, and a row with nothing at all
+    host = (torch.randn(B, rows, 1, D, device=DEV, generator=g), torch.randn(B, rows, 1, device=DEV, generator=g) + 2.0,
+            torch.rand(B, rows, 1, device=DEV, generator=g) + 1.0)
+    host[1][:, 1] = float("-inf")
+    outs = []
+    for tune in (0, hg.HG_TUNE_NO_MERGE_CLUSTER):
+        desc = pkg.attn_desc(batch=B, num_q_heads=rows, num_kv_heads=rows, head_dim=D, dtype=torch.float16, page_size=16, num_pages=1,
+                             page_stride=16 * rows * D, head_stride=16 * D, tok_stride=D, block_table=None, max_pages=1,
+                             chunk_tokens=64, num_chunks=slots, tune=tune)
+        out = torch.full((B, rows, D), 9.0, device=DEV); lse = torch.full((B, rows), 9.0, device=DEV)
+        pkg.hg_attn_merge([(o, m, l), host], out, lse, desc)
+        torch.cuda.synchronize()
+        outs.append((out, lse))
+    mm = torch.cat([m, host[1]], dim=2).double().cpu().numpy(); ll = torch.cat([l, host[2]], dim=2).double().cpu().numpy()
+    oo = torch.cat([o, host[0]], dim=2).double().cpu().numpy()
+    ref_out, ref_lse = O.merge_batch(mm, ll, oo)
+    for out, lse in outs:
+        got, gl = out.double().cpu().numpy(), lse.double().cpu().numpy()
+        assert np.all(got[0, 1] == 0.0) and gl[0, 1] == -np.inf                 # the empty row
+        keep = np.isfinite(ref_lse)
+        assert np.abs(got[keep] - ref_out[keep]).max() <= 1e-4 and np.abs(gl[keep] - ref_lse[keep]).max() <= 1e-4
